@@ -1,0 +1,194 @@
+/*
+ * pp.h -- exact min-bottleneck partition-and-placement on one NVIDIA B200 (sm_100a).
+ *
+ * Problem (paper, Section 1 and Section 3.2).  A chain of L layers is cut into m >= 1
+ * contiguous non-empty segments; segment j runs on its own edge node n_j, all nodes
+ * different; a segment fits when the bytes of its layers are <= the node's capacity.  The
+ * tensor that crosses cut j is the output of the last layer of segment j; its latency is
+ *        gamma_j = bits[e_j] / bw[n_j][n_{j+1}]            (Eq. 3, data / bandwidth)
+ * and a plan's bottleneck latency is
+ *        beta = max_j gamma_j                              (Eq. 2),   beta = +0.0 if m = 1.
+ * The library finds beta* = min over all plans, returns one canonical optimal plan, and
+ * scores arbitrary candidate plans in bulk.
+ *
+ * Arithmetic contract.  gamma is ONE IEEE-754 binary64 round-to-nearest division of the
+ * integer bit count by the integer kbps, so beta is in milliseconds.  The search only
+ * compares and selects gamma values (min / max); beta* is bit-for-bit one of them, or +0.0,
+ * or +inf.  A link of 0 kbps is unusable (gamma = +inf); the diagonal of bw is ignored.
+ *
+ * Canonical plan.  Among all plans with beta == beta*, the lexicographically smallest key
+ *        (m, mask, n_m, e_{m-1}, n_{m-1}, ..., e_1, n_1),   mask = sum_j 2^{n_j}:
+ * fewest segments, then lowest node-set mask, then lowest last node, then, walking
+ * backwards, lowest cut and lowest node id.
+ *
+ * Conventions for every entry point:
+ *  - "host" / "device" on a pointer says where the memory must live.  The library never
+ *    frees or keeps caller memory; inputs of pp_problem_create are copied.
+ *  - Errors are return codes only.  On PP_ERR_* the outputs are untouched.
+ *  - All work of a problem runs on its CUDA stream (default: the legacy default stream).
+ *    The *_dev entry points are asynchronous on that stream; the host entry points
+ *    synchronise it before returning.
+ *  - Layers are 0..L-1, nodes 0..k-1.  A cut value e means "the segment ends with layer e".
+ *  - There is no CPU fallback: without a CUDA device every compute entry point fails with
+ *    PP_ERR_CUDA.
+ */
+#ifndef PP_H
+#define PP_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PP_MAX_K 20   /* nodes; the state table has k * 2^k rows */
+#define PP_MAX_L 1024 /* layers */
+#define PP_MAX_BITS (1ull << 40) /* layer_out_bits must be below this */
+#define PP_MAX_KBPS (1u << 24)   /* bw_kbps must be below this */
+
+typedef struct pp_problem pp_problem; /* opaque; owns host and device copies of the inputs */
+
+typedef enum {
+    PP_OK = 0,
+    PP_INFEASIBLE = 1, /* not an error: no plan exists; beta = +inf, m = 0 */
+    PP_ERR_ARG = -1,   /* null pointer, L < 1, k < 1, B < 0 */
+    PP_ERR_LIMIT = -2, /* k > PP_MAX_K, L > PP_MAX_L, value above PP_MAX_BITS / PP_MAX_KBPS,
+                          or (batched solve) a state table that does not fit shared memory */
+    PP_ERR_NOMEM = -3, /* host or device allocation failed, or workspace too small */
+    PP_ERR_CUDA = -4,  /* a CUDA runtime call failed (includes "no device") */
+    PP_ERR_TIMEOUT = -5 /* reserved */
+} pp_status;
+
+/* plan_status bit flags written by the evaluator (0 = valid plan) */
+#define PP_PLAN_BAD_NSEG 1   /* nseg == 0 or nseg > min(k, L); nothing else is checked */
+#define PP_PLAN_BAD_ENDS 2   /* a cut outside [0, L-2] or cuts not strictly increasing */
+#define PP_PLAN_BAD_NODE 4   /* a node outside [0, k-1] or used twice */
+#define PP_PLAN_MEMORY 8     /* some segment exceeds its node's capacity */
+#define PP_PLAN_DEAD_LINK 16 /* two consecutive nodes joined by a 0 kbps link */
+
+/* Result record of the exact search as the device writes it. */
+typedef struct {
+    double beta_ms;              /* beta*, +inf if infeasible */
+    int32_t status;              /* PP_OK or PP_INFEASIBLE */
+    int32_t m;                   /* number of segments, 0 if infeasible */
+    int32_t cuts[PP_MAX_K];      /* e_1 .. e_{m-1}; unused slots are -1 */
+    int32_t placement[PP_MAX_K]; /* n_1 .. n_m;     unused slots are -1 */
+} pp_solution;
+
+/* Device-time breakdown of the last pp_solve_exact / pp_solve_exact_dev of a problem. */
+typedef struct {
+    float ms_rank;     /* gamma table and rank compression (Eq. 3) */
+    float ms_sweep;    /* base frontier plus all popcount levels of the (min,max) sweep */
+    float ms_finalize; /* final choice and backtrack */
+    float ms_total;
+    int32_t sweep_launches;  /* kernels launched for the sweep, base frontier included */
+    int32_t total_launches;  /* all kernels of the solve */
+    int32_t state_bytes;     /* bytes of one state element: 2 (16-bit ranks) or 4 */
+    int32_t fast_path;       /* 1 if the register-tiled sweep kernel ran, 0 if the generic one */
+} pp_profile;
+
+/*
+ * Problem set-up (Section 3: inputs are the chain and the weighted communication graph).
+ *   layer_out_bits  host [L]    output size of each layer in bits (transfer size of a cut after it)
+ *   layer_mem_bytes host [L]    memory of each layer in bytes
+ *   node_mem_bytes  host [k]    capacity of each node in bytes (heterogeneous; the paper's
+ *                               homogeneous case is all entries equal)
+ *   bw_kbps         host [k*k]  row-major, [v*k + w] = bandwidth of the link v -> w; 0 = no link
+ * Validates, builds the uint64 memory prefix sums and the per-node window table (for each
+ * node w and segment end c', the earliest segment start that still fits), uploads them.
+ * *out receives the handle; free it with pp_problem_destroy.
+ */
+pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
+                            const uint64_t *layer_mem_bytes, int32_t k,
+                            const uint64_t *node_mem_bytes, const uint32_t *bw_kbps,
+                            pp_problem **out);
+
+/* Frees the handle and every device buffer the library allocated for it (not a caller
+ * workspace).  NULL is allowed. */
+void pp_problem_destroy(pp_problem *p);
+
+/* Use `cuda_stream` (a cudaStream_t, e.g. torch.cuda.current_stream().cuda_stream) for all
+ * later work of this problem.  NULL selects the legacy default stream. */
+pp_status pp_problem_set_stream(pp_problem *p, void *cuda_stream);
+
+/* Bytes of device scratch the exact search needs (state table, gamma and rank tables). */
+pp_status pp_problem_workspace_bytes(const pp_problem *p, uint64_t *bytes);
+
+/* Hand the library a caller-owned device buffer (256-byte aligned, at least
+ * pp_problem_workspace_bytes) to use instead of allocating its own at the first solve.
+ * The caller keeps ownership and must keep it alive while the problem is used. */
+pp_status pp_problem_set_workspace(pp_problem *p, void *device_buffer, uint64_t bytes);
+
+/*
+ * Exact search (Eq. 2 minimised over every cut set and every injective placement) by a
+ * (min,max) dynamic programme over (used-node mask, last node, last cut layer), swept by
+ * popcount of the mask; then the canonical plan by backtracking.
+ *   beta_ms   host [1]    beta* in milliseconds, +inf if infeasible
+ *   m         host [1]    number of segments, 0 if infeasible
+ *   cuts      host [k-1]  e_1..e_{m-1}, rest -1   (may be NULL when k == 1)
+ *   placement host [k]    n_1..n_m, rest -1
+ * Returns PP_OK, PP_INFEASIBLE or an error.  Synchronous.
+ */
+pp_status pp_solve_exact(pp_problem *p, double *beta_ms, int32_t *m, int32_t *cuts,
+                         int32_t *placement);
+
+/* Same search; the result record is written to device memory `solution_dev` (device,
+ * sizeof(pp_solution), 8-byte aligned) by work queued on the problem's stream.  Returns as
+ * soon as the work is queued; feasibility is in solution_dev->status. */
+pp_status pp_solve_exact_dev(pp_problem *p, pp_solution *solution_dev);
+
+/*
+ * Batched beta evaluator (Eq. 3 per cut, Eq. 2 per plan) for B candidate plans of one problem.
+ *   nseg        [B]    number of segments of each plan
+ *   ends        [B*k]  row b: cuts e_1..e_{nseg-1} (only the first nseg-1 entries are read;
+ *                      the last segment always ends at L-1)
+ *   nodes       [B*k]  row b: n_1..n_nseg (only the first nseg entries are read)
+ *   beta_ms     [B]    out: beta of the plan, +inf if any flag is set
+ *   plan_status [B]    out: PP_PLAN_* flags.  BAD_NSEG stops all other checks; MEMORY and
+ *                      DEAD_LINK are only evaluated when ENDS and NODE are clean.
+ * pp_eval_plans takes host pointers and is synchronous; pp_eval_plans_dev takes device
+ * pointers and is asynchronous on the problem's stream.  B == 0 is a no-op.
+ */
+pp_status pp_eval_plans(pp_problem *p, int64_t B, const uint8_t *nseg, const int32_t *ends,
+                        const int32_t *nodes, double *beta_ms, uint8_t *plan_status);
+pp_status pp_eval_plans_dev(pp_problem *p, int64_t B, const uint8_t *nseg, const int32_t *ends,
+                            const int32_t *nodes, double *beta_ms, uint8_t *plan_status);
+
+/*
+ * Many independent instances of the same shape (L, k) in one call; each instance is the
+ * exact search above, done by one thread block with its whole state table in shared memory.
+ *   out_bits [B*L], mem [B*L], node_mem [B*k], bw [B*k*k]   inputs, instance-major
+ *   beta_ms [B], m [B], cuts [B*(k-1)], placement [B*k], status [B] (PP_OK / PP_INFEASIBLE,
+ *   or PP_ERR_LIMIT for an instance with a value above the limits)
+ * Returns PP_ERR_LIMIT without touching outputs when k * 2^(k-1) * L doubles plus the gamma
+ * table exceed the shared memory of one block.  Host variant is synchronous and uses the
+ * legacy default stream; the _dev variant takes device pointers and a stream and is
+ * asynchronous.  cuts may be NULL when k == 1.
+ */
+pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                               const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
+                               double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
+                               int8_t *status);
+pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                                   const uint64_t *mem, const uint64_t *node_mem,
+                                   const uint32_t *bw, double *beta_ms, int32_t *m, int32_t *cuts,
+                                   int32_t *placement, int8_t *status, void *cuda_stream);
+
+/* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream. */
+pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out);
+
+/* Test hook: after a solve, copy one row of the state table to the host as latencies:
+ * row_out[c] = value of state (mask, v, c) in milliseconds (+inf if unreachable), c = 0..L-1.
+ * `mask` must contain node v.  Synchronous. */
+pp_status pp_debug_read_state_row(pp_problem *p, uint32_t mask, int32_t v, double *row_out);
+
+/* Force (1) or forbid (0) the generic sweep kernel; -1 restores the automatic choice.
+ * Meant for tests that want both kernels checked on the same instance. */
+pp_status pp_problem_force_generic(pp_problem *p, int32_t mode);
+
+const char *pp_status_str(pp_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PP_H */

@@ -1,0 +1,252 @@
+"""Thin ctypes binding of libpp.so: argument marshalling only, same names as include/pp.h.
+
+Every step of the search and of the evaluator runs inside the library's CUDA kernels.  There is
+no Python or CPU fallback: if libpp.so is missing or fails to load, importing the library
+handle raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libpp.so")
+
+PP_MAX_K, PP_MAX_L = 20, 1024
+PP_OK, PP_INFEASIBLE = 0, 1
+PP_ERR_ARG, PP_ERR_LIMIT, PP_ERR_NOMEM, PP_ERR_CUDA, PP_ERR_TIMEOUT = -1, -2, -3, -4, -5
+PP_PLAN_BAD_NSEG, PP_PLAN_BAD_ENDS, PP_PLAN_BAD_NODE, PP_PLAN_MEMORY, PP_PLAN_DEAD_LINK = 1, 2, 4, 8, 16
+
+EXPORTS = (
+    "pp_problem_create", "pp_problem_destroy", "pp_problem_set_stream",
+    "pp_problem_workspace_bytes", "pp_problem_set_workspace", "pp_solve_exact",
+    "pp_solve_exact_dev", "pp_eval_plans", "pp_eval_plans_dev", "pp_solve_exact_batch",
+    "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row",
+    "pp_problem_force_generic", "pp_status_str",
+)
+
+
+class pp_solution(ctypes.Structure):
+    _fields_ = [("beta_ms", ctypes.c_double), ("status", ctypes.c_int32), ("m", ctypes.c_int32),
+                ("cuts", ctypes.c_int32 * PP_MAX_K), ("placement", ctypes.c_int32 * PP_MAX_K)]
+
+
+class pp_profile(ctypes.Structure):
+    _fields_ = [("ms_rank", ctypes.c_float), ("ms_sweep", ctypes.c_float),
+                ("ms_finalize", ctypes.c_float), ("ms_total", ctypes.c_float),
+                ("sweep_launches", ctypes.c_int32), ("total_launches", ctypes.c_int32),
+                ("state_bytes", ctypes.c_int32), ("fast_path", ctypes.c_int32)]
+
+
+class PPError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_str(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library.  Raises if it has not been built (run __graft_entry__.build())."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: build the CUDA library first "
+                               "(python -m paper_2210_12219_b200.build); there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64
+        L.pp_problem_create.argtypes = [i32, vp, vp, i32, vp, vp, ctypes.POINTER(vp)]
+        L.pp_problem_destroy.argtypes = [vp]
+        L.pp_problem_destroy.restype = None
+        L.pp_problem_set_stream.argtypes = [vp, vp]
+        L.pp_problem_workspace_bytes.argtypes = [vp, ctypes.POINTER(u64)]
+        L.pp_problem_set_workspace.argtypes = [vp, vp, u64]
+        L.pp_solve_exact.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32), vp, vp]
+        L.pp_solve_exact_dev.argtypes = [vp, vp]
+        L.pp_eval_plans.argtypes = [vp, i64, vp, vp, vp, vp, vp]
+        L.pp_eval_plans_dev.argtypes = [vp, i64, vp, vp, vp, vp, vp]
+        L.pp_solve_exact_batch.argtypes = [i64, i32, i32] + [vp] * 9
+        L.pp_solve_exact_batch_dev.argtypes = [i64, i32, i32] + [vp] * 10
+        L.pp_last_solve_profile.argtypes = [vp, ctypes.POINTER(pp_profile)]
+        L.pp_debug_read_state_row.argtypes = [vp, ctypes.c_uint32, i32, vp]
+        L.pp_problem_force_generic.argtypes = [vp, i32]
+        L.pp_status_str.argtypes = [ctypes.c_int]
+        L.pp_status_str.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name not in ("pp_problem_destroy", "pp_status_str"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_str(status: int) -> str:
+    return lib().pp_status_str(int(status)).decode()
+
+
+def _host(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a, ctypes.c_void_p(a.ctypes.data)
+
+
+def _check(status: int, where: str, ok=(PP_OK,)):
+    if status not in ok:
+        raise PPError(status, where)
+    return status
+
+
+@dataclass
+class Solution:
+    status: int
+    beta_ms: float
+    m: int
+    cuts: np.ndarray
+    placement: np.ndarray
+
+    def plan(self):
+        return (self.m, tuple(int(x) for x in self.cuts[: max(self.m - 1, 0)]),
+                tuple(int(x) for x in self.placement[: self.m]))
+
+
+class Problem:
+    """Owner of a pp_problem handle.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, L, layer_out_bits, layer_mem_bytes, k, node_mem_bytes, bw_kbps):
+        self.L, self.k = int(L), int(k)
+        self._h = ctypes.c_void_p()
+        keep = [_host(layer_out_bits, np.uint64), _host(layer_mem_bytes, np.uint64),
+                _host(node_mem_bytes, np.uint64), _host(bw_kbps, np.uint32)]
+        st = lib().pp_problem_create(self.L, keep[0][1], keep[1][1], self.k, keep[2][1], keep[3][1],
+                                     ctypes.byref(self._h))
+        _check(st, "pp_problem_create")
+        self._workspace = None
+
+    @classmethod
+    def from_instance(cls, inst):
+        return cls(inst.L, inst.layer_out_bits, inst.layer_mem_bytes, inst.k, inst.node_mem_bytes,
+                   inst.bw_kbps)
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().pp_problem_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- plumbing ------------------------------------------------------------------------
+    def set_stream(self, cuda_stream: int):
+        _check(lib().pp_problem_set_stream(self._h, ctypes.c_void_p(cuda_stream)), "pp_problem_set_stream")
+
+    def workspace_bytes(self) -> int:
+        n = ctypes.c_uint64()
+        _check(lib().pp_problem_workspace_bytes(self._h, ctypes.byref(n)), "pp_problem_workspace_bytes")
+        return int(n.value)
+
+    def set_workspace(self, tensor):
+        """Use a torch CUDA tensor (uint8) as the search scratch; it is kept alive by this object."""
+        _check(lib().pp_problem_set_workspace(self._h, ctypes.c_void_p(tensor.data_ptr()),
+                                              tensor.numel() * tensor.element_size()),
+               "pp_problem_set_workspace")
+        self._workspace = tensor
+
+    def force_generic(self, mode: int):
+        _check(lib().pp_problem_force_generic(self._h, int(mode)), "pp_problem_force_generic")
+
+    # -- exact search --------------------------------------------------------------------
+    def solve_exact(self) -> Solution:
+        beta = ctypes.c_double()
+        m = ctypes.c_int32()
+        cuts = np.full(max(self.k - 1, 1), -1, dtype=np.int32)
+        placement = np.full(self.k, -1, dtype=np.int32)
+        st = lib().pp_solve_exact(self._h, ctypes.byref(beta), ctypes.byref(m),
+                                  ctypes.c_void_p(cuts.ctypes.data), ctypes.c_void_p(placement.ctypes.data))
+        _check(st, "pp_solve_exact", ok=(PP_OK, PP_INFEASIBLE))
+        return Solution(st, beta.value, int(m.value), cuts[: max(self.k - 1, 0)], placement)
+
+    def solve_exact_dev(self, solution_ptr: int):
+        """Queue the search; the pp_solution record is written at device address solution_ptr."""
+        _check(lib().pp_solve_exact_dev(self._h, ctypes.c_void_p(solution_ptr)), "pp_solve_exact_dev")
+
+    def last_solve_profile(self) -> pp_profile:
+        prof = pp_profile()
+        _check(lib().pp_last_solve_profile(self._h, ctypes.byref(prof)), "pp_last_solve_profile")
+        return prof
+
+    def debug_read_state_row(self, mask: int, v: int) -> np.ndarray:
+        row = np.empty(self.L, dtype=np.float64)
+        _check(lib().pp_debug_read_state_row(self._h, int(mask), int(v), ctypes.c_void_p(row.ctypes.data)),
+               "pp_debug_read_state_row")
+        return row
+
+    # -- evaluator -----------------------------------------------------------------------
+    def eval_plans(self, nseg, ends, nodes):
+        """Host arrays in, host arrays out: (beta_ms float64 [B], plan_status uint8 [B])."""
+        nseg, p0 = _host(nseg, np.uint8)
+        B = nseg.shape[0]
+        ends, p1 = _host(ends, np.int32)
+        nodes, p2 = _host(nodes, np.int32)
+        assert ends.size == B * self.k and nodes.size == B * self.k
+        beta = np.empty(B, dtype=np.float64)
+        status = np.empty(B, dtype=np.uint8)
+        _check(lib().pp_eval_plans(self._h, B, p0, p1, p2, ctypes.c_void_p(beta.ctypes.data),
+                                   ctypes.c_void_p(status.ctypes.data)), "pp_eval_plans")
+        return beta, status
+
+    def eval_plans_dev(self, B, nseg_ptr, ends_ptr, nodes_ptr, beta_ptr, status_ptr):
+        _check(lib().pp_eval_plans_dev(self._h, int(B), *(ctypes.c_void_p(x) for x in
+                                       (nseg_ptr, ends_ptr, nodes_ptr, beta_ptr, status_ptr))),
+               "pp_eval_plans_dev")
+
+
+@dataclass
+class BatchSolution:
+    beta_ms: np.ndarray  # float64 [B]
+    m: np.ndarray  # int32 [B]
+    cuts: np.ndarray  # int32 [B, k-1]
+    placement: np.ndarray  # int32 [B, k]
+    status: np.ndarray  # int8 [B]
+
+    def plan(self, b):
+        m = int(self.m[b])
+        return (m, tuple(int(x) for x in self.cuts[b, : max(m - 1, 0)]),
+                tuple(int(x) for x in self.placement[b, :m]))
+
+
+def solve_exact_batch(L, k, out_bits, mem, node_mem, bw) -> BatchSolution:
+    """Host arrays [B, L], [B, L], [B, k], [B, k, k] -> BatchSolution (synchronous)."""
+    out_bits, p0 = _host(out_bits, np.uint64)
+    B = out_bits.shape[0]
+    mem, p1 = _host(mem, np.uint64)
+    node_mem, p2 = _host(node_mem, np.uint64)
+    bw, p3 = _host(bw, np.uint32)
+    assert out_bits.size == B * L and mem.size == B * L and node_mem.size == B * k and bw.size == B * k * k
+    beta = np.empty(B, dtype=np.float64)
+    m = np.empty(B, dtype=np.int32)
+    cuts = np.full((B, max(k - 1, 1)), -1, dtype=np.int32)
+    placement = np.empty((B, k), dtype=np.int32)
+    status = np.empty(B, dtype=np.int8)
+    st = lib().pp_solve_exact_batch(B, L, k, p0, p1, p2, p3, *(ctypes.c_void_p(a.ctypes.data) for a in
+                                    (beta, m, cuts, placement, status)))
+    _check(st, "pp_solve_exact_batch")
+    return BatchSolution(beta, m, cuts[:, : max(k - 1, 0)] if k > 1 else cuts[:, :0], placement, status)
+
+
+def solve_exact_batch_dev(B, L, k, bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr,
+                          placement_ptr, status_ptr, cuda_stream: int = 0):
+    st = lib().pp_solve_exact_batch_dev(int(B), int(L), int(k), *(ctypes.c_void_p(x) for x in (
+        bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr, placement_ptr, status_ptr,
+        cuda_stream)))
+    _check(st, "pp_solve_exact_batch_dev")

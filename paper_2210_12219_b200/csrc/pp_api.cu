@@ -1,0 +1,505 @@
+// C-ABI of libpp (see include/pp.h) and the host orchestration behind it: validation,
+// memory prefix sums, window table, mask lists, launch sequence, result download.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <limits>
+#include <map>
+#include <new>
+#include <vector>
+
+#include "pp_internal.cuh"
+
+using namespace pp;
+
+struct pp_problem {
+    int L = 0, k = 0, Lpad = 0, U = 0, elem = 2;
+    std::vector<uint64_t> bits, mem, cap, M;
+    std::vector<uint32_t> bw, ubw, masks, level_off;
+    std::vector<int16_t> lo, pair_u;
+    unsigned char *d_inputs = nullptr;  // one allocation for all small device arrays
+    unsigned char *d_work = nullptr;    // exact-search scratch (own or caller's)
+    uint64_t work_bytes = 0;
+    bool own_work = false;
+    cudaStream_t stream = nullptr;
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    pp_solution *h_sol = nullptr;  // pinned
+    pp_solution *d_sol = nullptr;
+    int32_t *h_err = nullptr;      // pinned
+    Dev d{};
+    bool solved = false;
+    int sweep_launches = 0, total_launches = 0, fast_used = 0;
+    int force_generic = -1;
+};
+
+namespace {
+
+pp_status from_cuda(cudaError_t e)
+{
+    if (e == cudaSuccess) return PP_OK;
+    cudaGetLastError();  // clear the sticky-less error state
+    return e == cudaErrorMemoryAllocation ? PP_ERR_NOMEM : PP_ERR_CUDA;
+}
+
+#define PP_CUDA(call)                                   \
+    do {                                                \
+        cudaError_t e__ = (call);                       \
+        if (e__ != cudaSuccess) return from_cuda(e__);  \
+    } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WorkLayout {
+    size_t pos, order, gu, rk, rank, table, total;
+};
+
+WorkLayout work_layout(int L, int k, int Lpad, int U, int elem)
+{
+    WorkLayout w;
+    size_t o = 0;
+    w.pos = o;   o = align_up(o + (size_t)L * 2, 256);
+    w.order = o; o = align_up(o + (size_t)L * 2, 256);
+    w.gu = o;    o = align_up(o + (size_t)std::max(U, 1) * L * 8, 256);
+    w.rk = o;    o = align_up(o + (size_t)std::max(U, 1) * L * 4, 256);
+    w.rank = o;  o = align_up(o + (size_t)k * k * Lpad * elem, 256);
+    w.table = o; o = align_up(o + ((size_t)k << k) * Lpad * elem, 256);
+    w.total = o;
+    return w;
+}
+
+pp_status validate(int32_t L, const uint64_t *bits, const uint64_t *mem, int32_t k,
+                   const uint64_t *cap, const uint32_t *bw)
+{
+    if (!bits || !mem || !cap || !bw) return PP_ERR_ARG;
+    if (L < 1 || k < 1) return PP_ERR_ARG;
+    if (L > PP_MAX_L || k > PP_MAX_K) return PP_ERR_LIMIT;
+    for (int i = 0; i < L; ++i)
+        if (bits[i] >= PP_MAX_BITS) return PP_ERR_LIMIT;
+    for (int i = 0; i < k * k; ++i)
+        if (bw[i] >= PP_MAX_KBPS) return PP_ERR_LIMIT;
+    uint64_t acc = 0;
+    for (int i = 0; i < L; ++i) {
+        if (mem[i] > std::numeric_limits<uint64_t>::max() - acc) return PP_ERR_LIMIT;
+        acc += mem[i];
+    }
+    return PP_OK;
+}
+
+void bind_work(pp_problem *p)
+{
+    WorkLayout w = work_layout(p->L, p->k, p->Lpad, p->U, p->elem);
+    unsigned char *b = p->d_work;
+    p->d.pos = reinterpret_cast<int16_t *>(b + w.pos);
+    p->d.order = reinterpret_cast<int16_t *>(b + w.order);
+    p->d.gu = reinterpret_cast<double *>(b + w.gu);
+    p->d.rk = reinterpret_cast<uint32_t *>(b + w.rk);
+    p->d.rank = b + w.rank;
+    p->d.table = b + w.table;
+}
+
+pp_status ensure_work(pp_problem *p)
+{
+    if (p->d_work) return PP_OK;
+    WorkLayout w = work_layout(p->L, p->k, p->Lpad, p->U, p->elem);
+    void *ptr = nullptr;
+    PP_CUDA(cudaMalloc(&ptr, w.total));
+    p->d_work = static_cast<unsigned char *>(ptr);
+    p->work_bytes = w.total;
+    p->own_work = true;
+    bind_work(p);
+    return PP_OK;
+}
+
+pp_status queue_solve(pp_problem *p, pp_solution *sol_dev)
+{
+    pp_status st = ensure_work(p);
+    if (st != PP_OK) return st;
+    cudaStream_t s = p->stream;
+    const Dev &d = p->d;
+    int launches = 0;
+    PP_CUDA(cudaEventRecord(p->ev[0], s));
+    PP_CUDA(launch_rank_build(d, s, &launches));
+    PP_CUDA(cudaEventRecord(p->ev[1], s));
+    PP_CUDA(launch_base(d, s));
+    int sweep = 1;
+    const int top = std::min(p->k, p->L);
+    bool fast = fast_sweep_supported(d);
+    if (p->force_generic == 1) fast = false;
+    for (int level = 2; level <= top; ++level) {
+        PP_CUDA(fast ? launch_sweep_fast(d, level, s) : launch_sweep_generic(d, level, s));
+        ++sweep;
+    }
+    PP_CUDA(cudaEventRecord(p->ev[2], s));
+    PP_CUDA(launch_finalize(d, sol_dev, s));
+    PP_CUDA(cudaEventRecord(p->ev[3], s));
+    p->sweep_launches = sweep;
+    p->total_launches = launches + sweep + 1;
+    p->fast_used = fast ? 1 : 0;
+    p->solved = true;
+    return PP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *pp_status_str(pp_status s)
+{
+    switch (s) {
+        case PP_OK: return "ok";
+        case PP_INFEASIBLE: return "infeasible: no plan exists";
+        case PP_ERR_ARG: return "bad argument";
+        case PP_ERR_LIMIT: return "size or value above the library limits";
+        case PP_ERR_NOMEM: return "out of memory";
+        case PP_ERR_CUDA: return "CUDA runtime error";
+        case PP_ERR_TIMEOUT: return "timeout";
+    }
+    return "unknown status";
+}
+
+pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
+                            const uint64_t *layer_mem_bytes, int32_t k,
+                            const uint64_t *node_mem_bytes, const uint32_t *bw_kbps,
+                            pp_problem **out)
+{
+    if (!out) return PP_ERR_ARG;
+    pp_status st = validate(L, layer_out_bits, layer_mem_bytes, k, node_mem_bytes, bw_kbps);
+    if (st != PP_OK) return st;
+    pp_problem *p = new (std::nothrow) pp_problem();
+    if (!p) return PP_ERR_NOMEM;
+    try {
+        p->L = L;
+        p->k = k;
+        p->bits.assign(layer_out_bits, layer_out_bits + L);
+        p->mem.assign(layer_mem_bytes, layer_mem_bytes + L);
+        p->cap.assign(node_mem_bytes, node_mem_bytes + k);
+        p->bw.assign(bw_kbps, bw_kbps + (size_t)k * k);
+        // memory prefix sums: segment first..last needs M[last+1] - M[first] bytes
+        p->M.assign(L + 1, 0);
+        for (int i = 0; i < L; ++i) p->M[i + 1] = p->M[i] + p->mem[i];
+        // window table: lo[w][c'] = earliest previous cut c >= 0 such that layers c+1..c' fit on
+        // w; c' itself when not even layer c' alone fits.  Non-decreasing in c'.
+        p->lo.assign((size_t)k * L, 0);
+        for (int w = 0; w < k; ++w) {
+            int c = 0;
+            for (int c2 = 0; c2 < L; ++c2) {
+                while (c < c2 && p->M[c2 + 1] - p->M[c + 1] > p->cap[w]) ++c;
+                p->lo[(size_t)w * L + c2] = (int16_t)c;
+            }
+        }
+        // distinct usable bandwidths
+        std::map<uint32_t, int> seen;
+        p->pair_u.assign((size_t)k * k, -1);
+        for (int v = 0; v < k; ++v)
+            for (int w = 0; w < k; ++w) {
+                uint32_t b = p->bw[(size_t)v * k + w];
+                if (v == w || b == 0) continue;
+                auto it = seen.find(b);
+                if (it == seen.end()) {
+                    it = seen.emplace(b, (int)p->ubw.size()).first;
+                    p->ubw.push_back(b);
+                }
+                p->pair_u[(size_t)v * k + w] = (int16_t)it->second;
+            }
+        p->U = (int)p->ubw.size();
+        if (p->ubw.empty()) p->ubw.push_back(0);  // keep the upload non-empty; U stays 0
+        // 16-bit ranks when 0, 1..L*U and the +inf code all fit
+        p->elem = ((uint64_t)L * (uint64_t)std::max(p->U, 1) + 1 <= 65534) ? 2 : 4;
+        const int per32 = 32 / p->elem;
+        p->Lpad = (L + per32 - 1) / per32 * per32;
+        // masks by (popcount, value)
+        const uint32_t nm = 1u << k;
+        p->level_off.assign(k + 2, 0);
+        for (uint32_t S = 1; S < nm; ++S) p->level_off[__builtin_popcount(S) + 1]++;
+        for (int j = 1; j <= k + 1; ++j) p->level_off[j] += p->level_off[j - 1];
+        p->masks.assign(nm - 1, 0);
+        {
+            std::vector<uint32_t> at(p->level_off.begin(), p->level_off.end());
+            for (uint32_t S = 1; S < nm; ++S) p->masks[at[__builtin_popcount(S)]++] = S;
+        }
+    } catch (const std::bad_alloc &) {
+        delete p;
+        return PP_ERR_NOMEM;
+    }
+
+    // upload the small arrays in one allocation
+    struct Part { const void *src; size_t bytes; size_t off; };
+    std::vector<Part> parts = {
+        {p->bits.data(), p->bits.size() * 8, 0},       {p->M.data(), p->M.size() * 8, 0},
+        {p->cap.data(), p->cap.size() * 8, 0},         {p->bw.data(), p->bw.size() * 4, 0},
+        {p->lo.data(), p->lo.size() * 2, 0},           {p->pair_u.data(), p->pair_u.size() * 2, 0},
+        {p->ubw.data(), p->ubw.size() * 4, 0},
+        {p->masks.data(), p->masks.size() * 4, 0},     {p->level_off.data(), p->level_off.size() * 4, 0},
+        {nullptr, 8, 0} /* best */,                    {nullptr, 4, 0} /* err */,
+        {nullptr, sizeof(pp_solution), 0} /* solution */};
+    size_t total = 0;
+    for (auto &q : parts) { q.off = total; total = align_up(total + q.bytes, 256); }
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&p->d_inputs), total);
+    if (e == cudaSuccess) e = cudaMemset(p->d_inputs, 0, total);
+    for (auto &q : parts)
+        if (e == cudaSuccess && q.src && q.bytes)
+            e = cudaMemcpy(p->d_inputs + q.off, q.src, q.bytes, cudaMemcpyHostToDevice);
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreate(&p->ev[i]);
+    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->h_sol), sizeof(pp_solution));
+    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->h_err), sizeof(int32_t));
+    if (e != cudaSuccess) {
+        pp_status rc = from_cuda(e);
+        pp_problem_destroy(p);
+        return rc;
+    }
+    unsigned char *b = p->d_inputs;
+    Dev &d = p->d;
+    d.L = L; d.k = k; d.Lpad = p->Lpad; d.U = p->U; d.elem = p->elem;
+    d.bits = reinterpret_cast<uint64_t *>(b + parts[0].off);
+    d.M = reinterpret_cast<uint64_t *>(b + parts[1].off);
+    d.cap = reinterpret_cast<uint64_t *>(b + parts[2].off);
+    d.bw = reinterpret_cast<uint32_t *>(b + parts[3].off);
+    d.lo = reinterpret_cast<int16_t *>(b + parts[4].off);
+    d.pair_u = reinterpret_cast<int16_t *>(b + parts[5].off);
+    d.ubw = reinterpret_cast<uint32_t *>(b + parts[6].off);
+    d.masks = reinterpret_cast<uint32_t *>(b + parts[7].off);
+    d.level_off = reinterpret_cast<uint32_t *>(b + parts[8].off);
+    d.best = reinterpret_cast<unsigned long long *>(b + parts[9].off);
+    d.err = reinterpret_cast<int32_t *>(b + parts[10].off);
+    p->d_sol = reinterpret_cast<pp_solution *>(b + parts[11].off);
+    *out = p;
+    return PP_OK;
+}
+
+void pp_problem_destroy(pp_problem *p)
+{
+    if (!p) return;
+    if (p->own_work && p->d_work) cudaFree(p->d_work);
+    if (p->d_inputs) cudaFree(p->d_inputs);
+    for (auto &e : p->ev)
+        if (e) cudaEventDestroy(e);
+    if (p->h_sol) cudaFreeHost(p->h_sol);
+    if (p->h_err) cudaFreeHost(p->h_err);
+    delete p;
+}
+
+pp_status pp_problem_set_stream(pp_problem *p, void *cuda_stream)
+{
+    if (!p) return PP_ERR_ARG;
+    p->stream = static_cast<cudaStream_t>(cuda_stream);
+    return PP_OK;
+}
+
+pp_status pp_problem_workspace_bytes(const pp_problem *p, uint64_t *bytes)
+{
+    if (!p || !bytes) return PP_ERR_ARG;
+    *bytes = work_layout(p->L, p->k, p->Lpad, p->U, p->elem).total;
+    return PP_OK;
+}
+
+pp_status pp_problem_set_workspace(pp_problem *p, void *device_buffer, uint64_t bytes)
+{
+    if (!p || !device_buffer) return PP_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(device_buffer) % 256) return PP_ERR_ARG;
+    if (bytes < work_layout(p->L, p->k, p->Lpad, p->U, p->elem).total) return PP_ERR_NOMEM;
+    if (p->own_work && p->d_work) {
+        cudaStreamSynchronize(p->stream);
+        cudaFree(p->d_work);
+    }
+    p->d_work = static_cast<unsigned char *>(device_buffer);
+    p->work_bytes = bytes;
+    p->own_work = false;
+    p->solved = false;
+    bind_work(p);
+    return PP_OK;
+}
+
+pp_status pp_problem_force_generic(pp_problem *p, int32_t mode)
+{
+    if (!p || mode < -1 || mode > 1) return PP_ERR_ARG;
+    p->force_generic = mode;
+    return PP_OK;
+}
+
+pp_status pp_solve_exact_dev(pp_problem *p, pp_solution *solution_dev)
+{
+    if (!p || !solution_dev) return PP_ERR_ARG;
+    return queue_solve(p, solution_dev);
+}
+
+pp_status pp_solve_exact(pp_problem *p, double *beta_ms, int32_t *m, int32_t *cuts,
+                         int32_t *placement)
+{
+    if (!p || !beta_ms || !m || !placement || (!cuts && p->k > 1)) return PP_ERR_ARG;
+    PP_CUDA(cudaMemsetAsync(p->d.err, 0, sizeof(int32_t), p->stream));
+    pp_status st = queue_solve(p, p->d_sol);
+    if (st != PP_OK) return st;
+    PP_CUDA(cudaMemcpyAsync(p->h_sol, p->d_sol, sizeof(pp_solution), cudaMemcpyDeviceToHost, p->stream));
+    PP_CUDA(cudaMemcpyAsync(p->h_err, p->d.err, sizeof(int32_t), cudaMemcpyDeviceToHost, p->stream));
+    PP_CUDA(cudaStreamSynchronize(p->stream));
+    if (*p->h_err) return PP_ERR_CUDA;
+    *beta_ms = p->h_sol->beta_ms;
+    *m = p->h_sol->m;
+    for (int j = 0; j < p->k - 1; ++j) cuts[j] = p->h_sol->cuts[j];
+    for (int j = 0; j < p->k; ++j) placement[j] = p->h_sol->placement[j];
+    return static_cast<pp_status>(p->h_sol->status);
+}
+
+pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out)
+{
+    if (!p || !out || !p->solved) return PP_ERR_ARG;
+    PP_CUDA(cudaStreamSynchronize(p->stream));
+    PP_CUDA(cudaEventElapsedTime(&out->ms_rank, p->ev[0], p->ev[1]));
+    PP_CUDA(cudaEventElapsedTime(&out->ms_sweep, p->ev[1], p->ev[2]));
+    PP_CUDA(cudaEventElapsedTime(&out->ms_finalize, p->ev[2], p->ev[3]));
+    PP_CUDA(cudaEventElapsedTime(&out->ms_total, p->ev[0], p->ev[3]));
+    out->sweep_launches = p->sweep_launches;
+    out->total_launches = p->total_launches;
+    out->state_bytes = p->elem;
+    out->fast_path = p->fast_used;
+    return PP_OK;
+}
+
+pp_status pp_eval_plans_dev(pp_problem *p, int64_t B, const uint8_t *nseg, const int32_t *ends,
+                            const int32_t *nodes, double *beta_ms, uint8_t *plan_status)
+{
+    if (!p || B < 0) return PP_ERR_ARG;
+    if (B == 0) return PP_OK;
+    if (!nseg || !ends || !nodes || !beta_ms || !plan_status) return PP_ERR_ARG;
+    PP_CUDA(launch_eval(p->d, B, nseg, ends, nodes, beta_ms, plan_status, p->stream));
+    return PP_OK;
+}
+
+pp_status pp_eval_plans(pp_problem *p, int64_t B, const uint8_t *nseg, const int32_t *ends,
+                        const int32_t *nodes, double *beta_ms, uint8_t *plan_status)
+{
+    if (!p || B < 0) return PP_ERR_ARG;
+    if (B == 0) return PP_OK;
+    if (!nseg || !ends || !nodes || !beta_ms || !plan_status) return PP_ERR_ARG;
+    const size_t k = p->k;
+    const size_t b_nseg = (size_t)B, b_rows = (size_t)B * k * 4, b_beta = (size_t)B * 8;
+    size_t o_ends = align_up(b_nseg, 256), o_nodes = align_up(o_ends + b_rows, 256);
+    size_t o_beta = align_up(o_nodes + b_rows, 256), o_st = align_up(o_beta + b_beta, 256);
+    size_t total = o_st + (size_t)B;
+    unsigned char *buf = nullptr;
+    PP_CUDA(cudaMalloc(reinterpret_cast<void **>(&buf), total));
+    cudaStream_t s = p->stream;
+    cudaError_t e = cudaMemcpyAsync(buf, nseg, b_nseg, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_ends, ends, b_rows, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_nodes, nodes, b_rows, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+        e = launch_eval(p->d, B, buf, reinterpret_cast<int32_t *>(buf + o_ends),
+                        reinterpret_cast<int32_t *>(buf + o_nodes),
+                        reinterpret_cast<double *>(buf + o_beta), buf + o_st, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(beta_ms, buf + o_beta, b_beta, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(plan_status, buf + o_st, (size_t)B, cudaMemcpyDeviceToHost, s);
+    cudaError_t e2 = cudaStreamSynchronize(s);
+    cudaFree(buf);
+    if (e != cudaSuccess) return from_cuda(e);
+    return from_cuda(e2);
+}
+
+pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                                   const uint64_t *mem, const uint64_t *node_mem,
+                                   const uint32_t *bw, double *beta_ms, int32_t *m, int32_t *cuts,
+                                   int32_t *placement, int8_t *status, void *cuda_stream)
+{
+    if (B < 0 || L < 1 || k < 1) return PP_ERR_ARG;
+    if (L > PP_MAX_L || k > PP_MAX_K) return PP_ERR_LIMIT;
+    if (B == 0) return PP_OK;
+    if (!out_bits || !mem || !node_mem || !bw || !beta_ms || !m || !placement || !status ||
+        (!cuts && k > 1))
+        return PP_ERR_ARG;
+    int dev = 0, max_sm = 0;
+    PP_CUDA(cudaGetDevice(&dev));
+    PP_CUDA(cudaDeviceGetAttribute(&max_sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    if (batch_smem_bytes(L, k) + 1024 > (size_t)max_sm) return PP_ERR_LIMIT;
+    PP_CUDA(launch_batch(B, L, k, out_bits, mem, node_mem, bw, beta_ms, m, cuts, placement, status,
+                         static_cast<cudaStream_t>(cuda_stream)));
+    return PP_OK;
+}
+
+pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                               const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
+                               double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
+                               int8_t *status)
+{
+    if (B < 0 || L < 1 || k < 1) return PP_ERR_ARG;
+    if (L > PP_MAX_L || k > PP_MAX_K) return PP_ERR_LIMIT;
+    if (B == 0) return PP_OK;
+    if (!out_bits || !mem || !node_mem || !bw || !beta_ms || !m || !placement || !status ||
+        (!cuts && k > 1))
+        return PP_ERR_ARG;
+    const size_t nB = (size_t)B;
+    const size_t sz[9] = {nB * L * 8, nB * L * 8, nB * k * 8, nB * k * k * 4, nB * 8,
+                          nB * 4,     nB * (size_t)std::max(k - 1, 1) * 4, nB * k * 4, nB};
+    size_t off[10];
+    off[0] = 0;
+    for (int i = 0; i < 9; ++i) off[i + 1] = align_up(off[i] + sz[i], 256);
+    unsigned char *buf = nullptr;
+    PP_CUDA(cudaMalloc(reinterpret_cast<void **>(&buf), off[9]));
+    cudaStream_t s = nullptr;
+    const void *src[4] = {out_bits, mem, node_mem, bw};
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i)
+        e = cudaMemcpyAsync(buf + off[i], src[i], sz[i], cudaMemcpyHostToDevice, s);
+    pp_status st = PP_OK;
+    if (e == cudaSuccess)
+        st = pp_solve_exact_batch_dev(B, L, k, reinterpret_cast<uint64_t *>(buf + off[0]),
+                                      reinterpret_cast<uint64_t *>(buf + off[1]),
+                                      reinterpret_cast<uint64_t *>(buf + off[2]),
+                                      reinterpret_cast<uint32_t *>(buf + off[3]),
+                                      reinterpret_cast<double *>(buf + off[4]),
+                                      reinterpret_cast<int32_t *>(buf + off[5]),
+                                      reinterpret_cast<int32_t *>(buf + off[6]),
+                                      reinterpret_cast<int32_t *>(buf + off[7]),
+                                      reinterpret_cast<int8_t *>(buf + off[8]), s);
+    if (e == cudaSuccess && st == PP_OK) {
+        void *dst[5] = {beta_ms, m, cuts, placement, status};
+        for (int i = 0; i < 5 && e == cudaSuccess; ++i) {
+            if (!dst[i]) continue;
+            size_t n = (i == 2) ? nB * (size_t)(k - 1) * 4 : sz[4 + i];
+            if (n) e = cudaMemcpyAsync(dst[i], buf + off[4 + i], n, cudaMemcpyDeviceToHost, s);
+        }
+    }
+    cudaError_t e2 = cudaStreamSynchronize(s);
+    cudaFree(buf);
+    if (st != PP_OK) return st;
+    if (e != cudaSuccess) return from_cuda(e);
+    return from_cuda(e2);
+}
+
+pp_status pp_debug_read_state_row(pp_problem *p, uint32_t mask, int32_t v, double *row_out)
+{
+    if (!p || !row_out || !p->solved) return PP_ERR_ARG;
+    if (v < 0 || v >= p->k || mask >= (1u << p->k) || !((mask >> v) & 1u)) return PP_ERR_ARG;
+    PP_CUDA(cudaStreamSynchronize(p->stream));
+    const int L = p->L, U = p->U;
+    std::vector<uint32_t> rk((size_t)std::max(U, 1) * L);
+    std::vector<double> gu((size_t)std::max(U, 1) * L);
+    if (U > 0) {
+        PP_CUDA(cudaMemcpy(rk.data(), p->d.rk, (size_t)U * L * 4, cudaMemcpyDeviceToHost));
+        PP_CUDA(cudaMemcpy(gu.data(), p->d.gu, (size_t)U * L * 8, cudaMemcpyDeviceToHost));
+    }
+    std::map<uint32_t, double> val;
+    for (size_t i = 0; i < (size_t)U * L; ++i) val[rk[i]] = gu[i];
+    const size_t row = ((size_t)mask * p->k + v) * p->Lpad;
+    std::vector<uint32_t> raw(L);
+    if (p->elem == 2) {
+        std::vector<uint16_t> r16(L);
+        PP_CUDA(cudaMemcpy(r16.data(), static_cast<uint16_t *>(p->d.table) + row, (size_t)L * 2,
+                           cudaMemcpyDeviceToHost));
+        for (int c = 0; c < L; ++c) raw[c] = r16[c] == 0xFFFFu ? 0xFFFFFFFFu : r16[c];
+    } else {
+        PP_CUDA(cudaMemcpy(raw.data(), static_cast<uint32_t *>(p->d.table) + row, (size_t)L * 4,
+                           cudaMemcpyDeviceToHost));
+    }
+    for (int c = 0; c < L; ++c) {
+        if (raw[c] == 0) row_out[c] = 0.0;
+        else if (raw[c] == 0xFFFFFFFFu) row_out[c] = std::numeric_limits<double>::infinity();
+        else {
+            auto it = val.find(raw[c]);
+            if (it == val.end()) return PP_ERR_CUDA;
+            row_out[c] = it->second;
+        }
+    }
+    return PP_OK;
+}
+
+}  // extern "C"

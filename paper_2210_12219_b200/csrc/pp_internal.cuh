@@ -1,0 +1,60 @@
+// Internal declarations shared by the translation units of libpp (host launchers + device view).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pp.h"
+
+namespace pp {
+
+// Device view of one problem.  Ranks are an order-preserving recoding of the gamma doubles:
+// 0 stands for +0.0, the all-ones value of the element type for +inf, 1..N for the gamma
+// values in increasing order (equal doubles share a rank).  min/max/compare on ranks give the
+// same selections as on the doubles (the sweep never does arithmetic on values).
+struct Dev {
+    int L, k, Lpad;            // Lpad: row stride in elements (32-byte multiple)
+    int U;                     // number of distinct non-zero off-diagonal bandwidth values
+    int elem;                  // bytes per state element: 2 or 4
+    const uint64_t *bits;      // [L]
+    const uint64_t *M;         // [L+1] prefix sums of layer memory
+    const uint64_t *cap;       // [k]
+    const uint32_t *bw;        // [k*k]
+    const int16_t *lo;         // [k*L] lo[w*L+c'] = first c >= 0 whose successor segment c+1..c' fits w
+                               //        (= c' when even the single layer c' does not fit)
+    const int16_t *pair_u;     // [k*k] index into ubw of the pair's bandwidth, -1 if unusable
+    const uint32_t *ubw;       // [U] distinct bandwidth values
+    const uint32_t *masks;     // [2^k - 1] all non-empty masks sorted by (popcount, value)
+    const uint32_t *level_off; // [k+2] masks of popcount j are masks[level_off[j] .. level_off[j+1])
+    int16_t *pos;              // [L] position of layer c in the ascending order of bits
+    int16_t *order;            // [L] layer at each position
+    double *gu;                // [U*L] gu[u*L+i] = bits[order[i]] / ubw[u]  (ascending in i)
+    uint32_t *rk;              // [U*L] rank of gu[u*L+i]
+    void *rank;                // [k*k*Lpad] rank[(w*k+v)*Lpad + c] of gamma[c][v][w], element type
+    void *table;               // [2^k * k * Lpad] state rows, row (S, v) at (S*k+v)*Lpad
+    unsigned long long *best;  // packed (rank, popcount, mask, v) of the best final state
+    int32_t *err;              // device error word (0 = fine)
+};
+
+static constexpr unsigned long long kNoBest = ~0ull;
+
+// final-state key: smaller is better; rank in the high bits, then popcount, mask, node
+__host__ __device__ inline unsigned long long pack_best(uint32_t rank, int popc, uint32_t mask, int v)
+{
+    return ((unsigned long long)rank << 30) | ((unsigned long long)popc << 25) |
+           ((unsigned long long)mask << 5) | (unsigned long long)v;
+}
+
+cudaError_t launch_rank_build(const Dev &d, cudaStream_t s, int *launches);
+cudaError_t launch_base(const Dev &d, cudaStream_t s);
+cudaError_t launch_sweep_generic(const Dev &d, int level, cudaStream_t s);
+bool fast_sweep_supported(const Dev &d);
+cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s);
+cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s);
+cudaError_t launch_eval(const Dev &d, int64_t B, const uint8_t *nseg, const int32_t *ends,
+                        const int32_t *nodes, double *beta, uint8_t *status, cudaStream_t s);
+size_t batch_smem_bytes(int L, int k);
+cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                         const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
+                         int32_t *cuts, int32_t *placement, int8_t *status, cudaStream_t s);
+
+}  // namespace pp

@@ -1,0 +1,253 @@
+"""GPU parity: the CUDA library (through its C-ABI) against the CPU oracle, bit for bit.
+
+beta is an fp64 quotient selected by min/max on both sides, plans are integers: every
+comparison here is exact equality (tolerance 0)."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2210_12219_b200 as pp
+from paper_2210_12219_b200 import build
+from paper_2210_12219_b200 import workloads as W
+from tests.helpers import make_instance, parse_golden
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+    pp.lib()
+
+
+def gpu_solve(inst, generic=None):
+    with pp.Problem.from_instance(inst) as p:
+        if generic is not None:
+            p.force_generic(1 if generic else 0)
+        return p.solve_exact()
+
+
+def assert_same(inst, got, want):
+    assert got.status == want.status, inst.name
+    assert got.beta_ms == want.beta_ms or (np.isinf(got.beta_ms) and np.isinf(want.beta_ms)), inst.name
+    assert got.plan() == want.plan(), inst.name
+    k = inst.k
+    assert (got.cuts[max(got.m - 1, 0):] == -1).all() and (got.placement[got.m:] == -1).all()
+    assert len(got.cuts) == k - 1 and len(got.placement) == k
+
+
+def test_hand_worked_fixtures():
+    _, cases = parse_golden()
+    for inst, plans, optimum in cases:
+        want_beta, m, cuts, nodes = optimum
+        got = gpu_solve(inst)
+        assert got.beta_ms == want_beta and got.plan() == (m, tuple(cuts), tuple(nodes))
+        assert got.status == (pp.PP_INFEASIBLE if m == 0 else pp.PP_OK)
+        with pp.Problem.from_instance(inst) as p:
+            B = len(plans)
+            nseg = np.array([q[0] for q in plans], dtype=np.uint8)
+            ends = np.full((B, inst.k), -1, dtype=np.int32)
+            nd = np.full((B, inst.k), -1, dtype=np.int32)
+            for b, (ns, cu, no, _, _) in enumerate(plans):
+                ends[b, :min(len(cu), inst.k)] = cu[:inst.k]
+                nd[b, :min(len(no), inst.k)] = no[:inst.k]
+            beta, status = p.eval_plans(nseg, ends, nd)
+            for b, (_, _, _, wb, wf) in enumerate(plans):
+                assert status[b] == wf and beta[b] == wb
+
+
+def test_tiny_config_matches_bruteforce_and_dp():
+    inst = W.config_tiny()
+    got = gpu_solve(inst)
+    assert_same(inst, got, oracle.bruteforce(inst))
+    assert_same(inst, got, oracle.dp_naive(inst))
+
+
+@pytest.mark.parametrize("generic", [True, False])
+def test_random_small_instances(generic):
+    n_inf = 0
+    seed = 0
+    for L, k, n in ((1, 1, 2), (1, 4, 2), (2, 2, 4), (5, 3, 20), (7, 4, 30), (12, 6, 30), (9, 5, 30),
+                    (3, 6, 10), (17, 5, 20), (33, 4, 10), (16, 7, 10), (40, 3, 6)):
+        for i in range(n):
+            kind = i % 4
+            inst = W.random_small(20000 + seed, L, k, tight=(kind == 1), ties=(kind == 2),
+                                  dead_links=0.3 if kind == 3 else 0.0)
+            seed += 1
+            want = oracle.dp_naive(inst)
+            assert_same(inst, gpu_solve(inst, generic), want)
+            n_inf += want.status == oracle.INFEASIBLE
+    assert seed >= 170 and n_inf >= 5
+
+
+def _compare_rows(inst, p, rows):
+    want = oracle.dp_fact(inst, 4, want_table=True).table
+    for S, v in rows:
+        got = p.debug_read_state_row(S, v)
+        assert np.array_equal(got, want[S, v]), (inst.name, S, v)
+
+
+@pytest.mark.parametrize("generic", [True, False])
+def test_state_table_element_by_element(generic):
+    # every state of small instances, sampled rows of configs 2 and 3 (several tiles of masks,
+    # ragged rows: L = 12, 50, 100 are not multiples of the 16-element row padding)
+    rng = np.random.default_rng(3)
+    for inst in (W.config_tiny(), W.random_small(30000, 19, 5, tight=True),
+                 W.random_small(30001, 8, 6, dead_links=0.3)):
+        with pp.Problem.from_instance(inst) as p:
+            p.force_generic(1 if generic else 0)
+            p.solve_exact()
+            rows = [(S, v) for S in range(1, 1 << inst.k) for v in range(inst.k)
+                    if S >> v & 1 and bin(S).count("1") <= inst.L]
+            _compare_rows(inst, p, rows)
+    for inst in (W.config_resnet50_shaped(), W.config_deeper_cnn()):
+        with pp.Problem.from_instance(inst) as p:
+            p.force_generic(1 if generic else 0)
+            want = oracle.dp_fact(inst, 8)
+            assert_same(inst, p.solve_exact(), want)
+            rows = []
+            while len(rows) < 120:
+                S = int(rng.integers(1, 1 << inst.k))
+                vs = [v for v in range(inst.k) if S >> v & 1]
+                rows.append((S, int(rng.choice(vs))))
+            rows.append(((1 << inst.k) - 1, inst.k - 1))
+            _compare_rows(inst, p, rows)
+
+
+def test_named_configs_2_and_3():
+    for inst in (W.config_resnet50_shaped(), W.config_deeper_cnn()):
+        want = oracle.dp_fact(inst, 8)
+        got = gpu_solve(inst)
+        assert_same(inst, got, want)
+        assert oracle.eval_plan(inst, *got.plan()) == (got.beta_ms, 0)
+
+
+def _sub_instance(inst, nodes):
+    idx = np.array(nodes)
+    return make_instance(inst.layer_out_bits, inst.layer_mem_bytes, inst.node_mem_bytes[idx],
+                         inst.bw_kbps[np.ix_(idx, idx)], f"{inst.name}-sub")
+
+
+def test_large_config_full_size():
+    # config 5 (k = 18, L = 200) in the launch configuration the benchmark times.  The oracle
+    # solves the whole instance for beta* and the plan; single states are checked on sampled
+    # rows: the states of a node subset are exactly the table of the instance restricted to
+    # those nodes, which the oracle can afford for up to 8 nodes.
+    inst = W.config_large()
+    want = oracle.dp_fact(inst, oracle.max_threads())
+    with pp.Problem.from_instance(inst) as p:
+        got = p.solve_exact()
+        assert_same(inst, got, want)
+        assert oracle.eval_plan(inst, *got.plan()) == (got.beta_ms, 0)
+        prof = p.last_solve_profile()
+        assert prof.state_bytes == 2
+        rng = np.random.default_rng(9)
+        for size in (1, 2, 3, 5, 7, 8):
+            nodes = sorted(int(x) for x in rng.choice(inst.k, size=size, replace=False))
+            sub = _sub_instance(inst, nodes)
+            table = oracle.dp_fact(sub, 4, want_table=True).table
+            S = sum(1 << n for n in nodes)
+            for j, n in enumerate(nodes):
+                assert np.array_equal(p.debug_read_state_row(S, n), table[(1 << size) - 1, j])
+        # second solve on the same handle gives the same answer (scratch is reused)
+        assert_same(inst, p.solve_exact(), want)
+
+
+def test_32bit_rank_path():
+    # enough distinct gamma values that 16-bit ranks do not fit: L * U + 1 > 65534
+    L, k = 700, 11
+    base = W.random_small(40000, L, k)
+    cap = np.full(k, int(base.layer_mem_bytes.sum()) // 4, dtype=np.uint64)
+    bw = base.bw_kbps.copy()
+    bw[np.triu_indices(k, 1)] += np.arange(k * (k - 1) // 2, dtype=np.uint32) + 1  # directed links
+    inst = make_instance(base.layer_out_bits, base.layer_mem_bytes, cap, bw)
+    assert len({int(x) for x in inst.bw_kbps.ravel() if x}) * L + 1 > 65534
+    want = oracle.dp_fact(inst, oracle.max_threads())
+    with pp.Problem.from_instance(inst) as p:
+        got = p.solve_exact()
+        assert p.last_solve_profile().state_bytes == 4
+    assert_same(inst, got, want)
+
+
+def test_evaluator_against_oracle():
+    for inst, B in ((W.config_tiny(), 3000), (W.config_resnet50_shaped(), 3000),
+                    (W.random_small(50000, 14, 7, dead_links=0.2), 2000), (W.config_large(), 5000)):
+        nseg, ends, nodes = W.random_plans(inst, B, seed=B + inst.k, invalid_fraction=0.15)
+        want_beta, want_status = oracle.eval_plans(inst, nseg, ends, nodes)
+        with pp.Problem.from_instance(inst) as p:
+            beta, status = p.eval_plans(nseg, ends, nodes)
+            assert np.array_equal(status, want_status)
+            assert np.array_equal(beta, want_beta)  # inf == inf
+            assert (status == 0).sum() > 10 and (status != 0).sum() > 10
+            # the optimum scores as itself
+            sol = p.solve_exact()
+            if sol.status == pp.PP_OK:
+                e = np.full((1, inst.k), -1, np.int32)
+                n = np.full((1, inst.k), -1, np.int32)
+                e[0, :sol.m - 1] = sol.cuts[:sol.m - 1]
+                n[0, :sol.m] = sol.placement[:sol.m]
+                b1, s1 = p.eval_plans(np.array([sol.m], np.uint8), e, n)
+                assert s1[0] == 0 and b1[0] == sol.beta_ms
+            assert p.eval_plans(np.zeros(0, np.uint8), np.zeros((0, inst.k), np.int32),
+                                np.zeros((0, inst.k), np.int32))[0].shape == (0,)
+
+
+def _stack(insts):
+    return (np.stack([i.layer_out_bits for i in insts]), np.stack([i.layer_mem_bytes for i in insts]),
+            np.stack([i.node_mem_bytes for i in insts]), np.stack([i.bw_kbps for i in insts]))
+
+
+def test_batched_solve_full_config():
+    insts = W.config_batched()
+    assert len(insts) == 4096
+    got = pp.solve_exact_batch(24, 8, *_stack(insts))
+    n_inf = 0
+    for b, inst in enumerate(insts):
+        want = oracle.dp_fact(inst)
+        assert got.status[b] == want.status, b
+        assert got.beta_ms[b] == want.beta_ms or (np.isinf(got.beta_ms[b]) and np.isinf(want.beta_ms))
+        assert got.plan(b) == want.plan(), b
+        assert (got.cuts[b, max(want.m - 1, 0):] == -1).all() and (got.placement[b, want.m:] == -1).all()
+        n_inf += want.status == oracle.INFEASIBLE
+    assert 0 < n_inf < 4096
+
+
+def test_batched_solve_odd_shapes():
+    for L, k, n in ((1, 1, 3), (5, 2, 9), (13, 5, 40), (3, 6, 12), (30, 7, 10)):
+        insts = [W.random_small(60000 + 100 * L + i, L, k, tight=(i % 3 == 1), ties=(i % 3 == 2),
+                                dead_links=0.25 if i % 4 == 3 else 0.0) for i in range(n)]
+        got = pp.solve_exact_batch(L, k, *_stack(insts))
+        for b, inst in enumerate(insts):
+            want = oracle.dp_naive(inst)
+            assert got.status[b] == want.status
+            assert got.plan(b) == want.plan()
+            assert got.beta_ms[b] == want.beta_ms or np.isinf(want.beta_ms)
+    # a table that cannot fit one block's shared memory is refused, not mis-solved
+    with pytest.raises(pp.PPError) as ei:
+        pp.solve_exact_batch(200, 12, np.ones((1, 200), np.uint64), np.ones((1, 200), np.uint64),
+                             np.ones((1, 12), np.uint64), np.ones((1, 12, 12), np.uint32))
+    assert ei.value.status == pp.PP_ERR_LIMIT
+
+
+def test_workspace_and_stream_from_torch():
+    import torch
+    inst = W.config_resnet50_shaped()
+    want = oracle.dp_fact(inst, 4)
+    stream = torch.cuda.Stream()
+    with pp.Problem.from_instance(inst) as p:
+        ws = torch.empty(p.workspace_bytes(), dtype=torch.uint8, device="cuda")
+        p.set_workspace(ws)
+        p.set_stream(stream.cuda_stream)
+        sol = torch.zeros(24, dtype=torch.float64, device="cuda")  # 192 bytes >= sizeof(pp_solution)
+        p.solve_exact_dev(sol.data_ptr())
+        stream.synchronize()
+        raw = sol.cpu().numpy().tobytes()
+        rec = pp.pp_solution.from_buffer_copy(raw[:176])
+        assert rec.beta_ms == want.beta_ms and rec.status == want.status and rec.m == want.m
+        assert tuple(rec.cuts[:want.m - 1]) == want.plan()[1]
+        assert tuple(rec.placement[:want.m]) == want.plan()[2]
+        small = torch.empty(16, dtype=torch.uint8, device="cuda")
+        with pytest.raises(pp.PPError):
+            p.set_workspace(small)
