@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the exact partition-and-placement path on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+  1. exact search on the Large instance (k = 18 nodes, L = 200 layers): gamma/rank tables,
+     base frontier, every popcount level of the (min,max) sweep, final choice, backtrack;
+  2. the batched many-instance search on 4096 instances (k = 8, L = 24);
+  3. the batched beta evaluator on 262144 candidate plans of the Large instance.
+The headline number is DP relaxations per second, where one relaxation is
+g = min(g, max(dp, gamma)) and an instance has k(k-1)2^(k-2) L of them (a closed form of
+the sizes, not of the data).
+
+`value` is measured with the inputs resident in device memory; `e2e` goes through the
+host-pointer C entry points, host<->device copies inside the timed region.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2210_12219_b200 import workloads as W  # noqa: E402
+
+METRIC = "exact-plan DP relaxations/s"
+UNIT = "relaxations/s"
+N_PLANS = 262144
+N_BATCH = 4096
+BATCH_L, BATCH_K = 24, 8
+WORKLOAD = ("Large: k=18 nodes, L=200 layers (exact search) + Batched: 4096 x (k=8, L=24) + "
+            "262144 candidate plans scored")
+
+
+def n_relax(k: int, L: int) -> int:
+    return k * (k - 1) * (1 << (k - 2)) * L if k >= 2 else 0
+
+
+def n_states(k: int, L: int) -> int:
+    return k * (1 << (k - 1)) * L
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle sampling in the background while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def __enter__(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            time.sleep(0.3)  # let the first sample land before the timed region starts
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        if self.proc is None or not self.path or not os.path.exists(self.path):
+            return None
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        with open(self.path) as f:
+            for line in f:
+                t = [x.strip() for x in line.split(",")]
+                if len(t) < 7:
+                    continue
+                try:
+                    sm.append(float(t[0]))
+                    mx.append(float(t[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, t[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def stack(insts):
+    return (np.stack([i.layer_out_bits for i in insts]), np.stack([i.layer_mem_bytes for i in insts]),
+            np.stack([i.node_mem_bytes for i in insts]), np.stack([i.bw_kbps for i in insts]))
+
+
+def run_ours(args):
+    import torch
+
+    import paper_2210_12219_b200 as pp
+    from paper_2210_12219_b200 import build as pp_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pp_build.build()
+    pp.lib()
+    dev = torch.device("cuda", local)
+
+    # ---- synthetic inputs (every rank works on its own replica of the same workload) ----
+    large = W.config_large()
+    batch = W.config_batched(N_BATCH, BATCH_L, BATCH_K)
+    b_bits, b_mem, b_cap, b_bw = stack(batch)
+    nseg, ends, nodes = W.random_plans(large, N_PLANS, seed=77, invalid_fraction=0.05)
+    k, L = large.k, large.L
+    relax_large = n_relax(k, L)
+    relax_batch = N_BATCH * n_relax(BATCH_K, BATCH_L)
+    relax_step = relax_large + relax_batch
+
+    stream = torch.cuda.Stream(device=dev)
+    prob = pp.Problem.from_instance(large)
+    prob.set_stream(stream.cuda_stream)
+    ws = torch.empty(prob.workspace_bytes(), dtype=torch.uint8, device=dev)
+    prob.set_workspace(ws)
+    tt = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    d_nseg, d_ends, d_nodes = tt(nseg), tt(ends), tt(nodes)
+    d_beta = torch.empty(N_PLANS, dtype=torch.float64, device=dev)
+    d_pstat = torch.empty(N_PLANS, dtype=torch.uint8, device=dev)
+    d_bb, d_bm, d_bc, d_bbw = tt(b_bits), tt(b_mem), tt(b_cap), tt(b_bw)
+    o_beta = torch.empty(N_BATCH, dtype=torch.float64, device=dev)
+    o_m = torch.empty(N_BATCH, dtype=torch.int32, device=dev)
+    o_cuts = torch.empty(N_BATCH * (BATCH_K - 1), dtype=torch.int32, device=dev)
+    o_place = torch.empty(N_BATCH * BATCH_K, dtype=torch.int32, device=dev)
+    o_stat = torch.empty(N_BATCH, dtype=torch.int8, device=dev)
+    d_sol = torch.zeros(ctypes.sizeof(pp.pp_solution) // 8, dtype=torch.float64, device=dev)
+
+    def batch_device():
+        pp.solve_exact_batch_dev(N_BATCH, BATCH_L, BATCH_K, d_bb.data_ptr(), d_bm.data_ptr(),
+                                 d_bc.data_ptr(), d_bbw.data_ptr(), o_beta.data_ptr(), o_m.data_ptr(),
+                                 o_cuts.data_ptr(), o_place.data_ptr(), o_stat.data_ptr(),
+                                 stream.cuda_stream)
+
+    def eval_device():
+        prob.eval_plans_dev(N_PLANS, d_nseg.data_ptr(), d_ends.data_ptr(), d_nodes.data_ptr(),
+                            d_beta.data_ptr(), d_pstat.data_ptr())
+
+    def step_device():
+        prob.solve_exact_dev(d_sol.data_ptr())
+        batch_device()
+        eval_device()
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- warm-up, then the timed region (device-resident inputs) ----
+    warmup = max(args.warmup, 3)
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            step_device()
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(local) as clocks:
+            ev0.record(stream)
+            for _ in range(args.steps):
+                step_device()
+            ev1.record(stream)
+            barrier()
+        ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+        clk = clocks.summary()
+        prof = prob.last_solve_profile()
+        launches_per_step = prof.total_launches + 2
+
+        # per-part device times (same launch configuration, measured after the timed region)
+        sweep_ms, rank_ms, fin_ms, solve_ms = [], [], [], []
+        for _ in range(7):
+            prob.solve_exact_dev(d_sol.data_ptr())
+            pr = prob.last_solve_profile()
+            sweep_ms.append(pr.ms_sweep)
+            rank_ms.append(pr.ms_rank)
+            fin_ms.append(pr.ms_finalize)
+            solve_ms.append(pr.ms_total)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        batch_ms, eval_ms = [], []
+        for _ in range(7):
+            e0.record(stream)
+            batch_device()
+            e1.record(stream)
+            eval_device()
+            e2.record(stream)
+            stream.synchronize()
+            batch_ms.append(e0.elapsed_time(e1))
+            eval_ms.append(e1.elapsed_time(e2))
+
+    sol_rec = pp.pp_solution.from_buffer_copy(d_sol.cpu().numpy().tobytes())
+    ms_per_step = ms_total / args.steps
+    value = world * relax_step / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-pointer entry points ----
+    h2d = (large.layer_out_bits.nbytes + large.layer_mem_bytes.nbytes + large.node_mem_bytes.nbytes
+           + large.bw_kbps.nbytes + nseg.nbytes + ends.nbytes + nodes.nbytes
+           + b_bits.nbytes + b_mem.nbytes + b_cap.nbytes + b_bw.nbytes)
+    d2h = (ctypes.sizeof(pp.pp_solution) + N_PLANS * 9
+           + N_BATCH * (8 + 4 + 4 * (BATCH_K - 1) + 4 * BATCH_K + 1))
+
+    def step_host():
+        with pp.Problem.from_instance(large) as p2:
+            p2.set_workspace(ws)
+            s = p2.solve_exact()
+            bsol = pp.solve_exact_batch(BATCH_L, BATCH_K, b_bits, b_mem, b_cap, b_bw)
+            beta, pstat = p2.eval_plans(nseg, ends, nodes)
+        return s, bsol, beta, pstat
+
+    for _ in range(2):
+        host_out = step_host()
+    barrier()
+    t0 = time.perf_counter()
+    e2e_steps = max(2, min(args.steps, 10))
+    for _ in range(e2e_steps):
+        host_out = step_host()
+    barrier()
+    e2e_s = max_over_ranks((time.perf_counter() - t0) / e2e_steps)
+    e2e_value = world * relax_step / e2e_s
+    assert host_out[0].beta_ms == sol_rec.beta_ms and host_out[0].m == sol_rec.m
+
+    # ---- roofline of the dominant kernel (the popcount sweep of the Large instance) ----
+    peaks, which = measured_peaks()
+    elem = prof.state_bytes
+    sweep_t = statistics.median(sweep_ms) * 1e-3
+    alg_bytes = 2 * n_states(k, L) * elem  # every state written once and read once
+    achieved = alg_bytes / sweep_t / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": which,
+                "kernel": "sweep (%d launches per solve, base frontier included)" % prof.sweep_launches,
+                "algorithmic_bytes_per_solve": alg_bytes, "sweep_ms": sweep_t * 1e3}
+
+    med = statistics.median
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u16" if elem == 2 else "u32",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD,
+                   "relaxations_per_step": relax_step, "states_large": n_states(k, L),
+                   "l2": "state table of %.2f GB per solve exceeds the 126 MB L2; no explicit flush"
+                         % (alg_bytes / 2 / 1e9),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "gpu_launches": launches_per_step * args.steps,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_s * 1e3},
+        "clocks": clk,
+        "roofline": roofline,
+        "breakdown": {
+            "large_solve_ms": med(solve_ms), "rank_build_ms": med(rank_ms),
+            "sweep_ms": med(sweep_ms), "finalize_ms": med(fin_ms),
+            "large_relaxations_per_s": relax_large / (med(solve_ms) * 1e-3),
+            "batch_ms": med(batch_ms), "instances_per_s": N_BATCH / (med(batch_ms) * 1e-3),
+            "eval_ms": med(eval_ms), "plans_per_s": N_PLANS / (med(eval_ms) * 1e-3),
+            "fast_path": prof.fast_path, "beta_ms": sol_rec.beta_ms, "segments": sol_rec.m,
+        },
+    }
+    if rank == 0 and world == 1 and not args.no_cpu:
+        out["cpu_baseline"] = cpu_baseline(large)
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(large):
+    """The oracle as it stands, timed on the host cores on the Large instance (one full solve)."""
+    import oracle
+    threads = oracle.max_threads()
+    t0 = time.perf_counter()
+    sol = oracle.dp_fact(large, threads)
+    dt = time.perf_counter() - t0
+    return {"value": n_relax(large.k, large.L) / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "one full factorised-DP solve of the Large instance (k=18, L=200), OpenMP",
+            "seconds": dt, "beta_ms": sol.beta_ms}
+
+
+def run_reference(args):
+    """CPU oracle arm: each step is a bounded sample of the step above -- the Large instance
+    restricted to its first 15 nodes, 64 of the batched instances, 2048 of the candidate plans."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    large = W.config_large()
+    ksub = 15
+    sub = W.Instance(large.L, ksub, large.layer_out_bits, large.layer_mem_bytes,
+                     large.node_mem_bytes[:ksub].copy(),
+                     np.ascontiguousarray(large.bw_kbps[:ksub, :ksub]), "large[:15 nodes]")
+    batch = W.config_batched(64, BATCH_L, BATCH_K)
+    nseg, ends, nodes = W.random_plans(large, 2048, seed=77, invalid_fraction=0.05)
+    threads = oracle.max_threads()
+    relax_step = n_relax(ksub, large.L) + 64 * n_relax(BATCH_K, BATCH_L)
+
+    def step():
+        oracle.dp_fact(sub, threads)
+        for inst in batch:
+            oracle.dp_fact(inst, 1)
+        oracle.eval_plans(large, nseg, ends, nodes)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = relax_step / dt
+    sample = ("per step: factorised DP on the Large instance restricted to its first 15 nodes, "
+              "64 batched instances, 2048 candidate plans")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
