@@ -186,6 +186,43 @@ pp_status pp_debug_read_state_row(pp_problem *p, uint32_t mask, int32_t v, doubl
  * Meant for tests that want both kernels checked on the same instance. */
 pp_status pp_problem_force_generic(pp_problem *p, int32_t mode);
 
+/*
+ * Exact search that allocates nothing (the paper has no counterpart; this entry point exists
+ * for the library's users, not for the method).
+ *
+ * Who needs it: code that must not, or cannot, call cudaMalloc at this point -- a process
+ * whose whole device heap was handed to a framework's caching allocator at start-up, a
+ * serving loop that cannot afford the device-wide synchronisation an allocation implies, a
+ * plug-in that is only allowed to launch work.  pp_problem_create / pp_solve_exact allocate
+ * device and pinned memory; this call does not.  It performs the same search with the same
+ * kernels (the generic sweep) and gives bit-identical results, but every byte of device
+ * scratch (inputs copy, gamma and rank tables, state table) comes from one array of
+ * PP_STATIC_SCRATCH_BYTES that is compiled into the library.  Every GPU that loads the library
+ * holds that array until the process exits, whether or not this call is ever made.
+ *
+ *   layer_out_bits, layer_mem_bytes  host [L];  node_mem_bytes host [k];  bw_kbps host [k*k]
+ *   solution_dev   device, sizeof(pp_solution), 8-byte aligned: receives the result record
+ *   cuda_stream    a cudaStream_t (NULL = legacy default stream); the inputs are copied from
+ *                  pageable host memory with cudaMemcpyAsync (the host buffers may be reused
+ *                  as soon as the call returns); kernels are queued on the stream and the call
+ *                  returns without waiting for them.
+ * Limits: k <= 14, L <= PP_MAX_L, and the scratch the instance needs (dominated by the state
+ * table, k * 2^k rows of L elements of 2 or 4 bytes) must fit PP_STATIC_SCRATCH_BYTES; anything
+ * larger returns PP_ERR_LIMIT before any work is queued (k = 10, L = 50 needs about 1.1 MB;
+ * k = 14, L = 100 about 52 MB).  Host-side preparation uses about 100 KB of stack.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress,
+ * with that device current) and caches it; make that first call outside any stream capture.
+ * All calls share the one array and it keeps the previous call's contents; the library resets
+ * the words that must start clean itself.  Two calls whose GPU work overlaps (different
+ * streams, or different host threads) race on the array: serialise them.
+ * No cudaMalloc, cudaFree, cudaMallocHost or other allocating routine is called.
+ */
+#define PP_STATIC_SCRATCH_BYTES (64u << 20)
+pp_status pp_solve_exact_static(int32_t L, const uint64_t *layer_out_bits,
+                                const uint64_t *layer_mem_bytes, int32_t k,
+                                const uint64_t *node_mem_bytes, const uint32_t *bw_kbps,
+                                pp_solution *solution_dev, void *cuda_stream);
+
 const char *pp_status_str(pp_status s);
 
 #ifdef __cplusplus

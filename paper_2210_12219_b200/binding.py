@@ -25,7 +25,7 @@ EXPORTS = (
     "pp_problem_workspace_bytes", "pp_problem_set_workspace", "pp_solve_exact",
     "pp_solve_exact_dev", "pp_eval_plans", "pp_eval_plans_dev", "pp_solve_exact_batch",
     "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row",
-    "pp_problem_force_generic", "pp_status_str",
+    "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str",
 )
 
 
@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
         L.pp_last_solve_profile.argtypes = [vp, ctypes.POINTER(pp_profile)]
         L.pp_debug_read_state_row.argtypes = [vp, ctypes.c_uint32, i32, vp]
         L.pp_problem_force_generic.argtypes = [vp, i32]
+        L.pp_solve_exact_static.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp]
         L.pp_status_str.argtypes = [ctypes.c_int]
         L.pp_status_str.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -250,3 +251,13 @@ def solve_exact_batch_dev(B, L, k, bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta
         bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr, placement_ptr, status_ptr,
         cuda_stream)))
     _check(st, "pp_solve_exact_batch_dev")
+
+
+def solve_exact_static(L, layer_out_bits, layer_mem_bytes, k, node_mem_bytes, bw_kbps,
+                       solution_ptr: int, cuda_stream: int = 0) -> int:
+    """pp_solve_exact_static: host input arrays, device address of the pp_solution record.
+    Returns the status code instead of raising, so callers can test the limit check."""
+    keep = [_host(layer_out_bits, np.uint64), _host(layer_mem_bytes, np.uint64),
+            _host(node_mem_bytes, np.uint64), _host(bw_kbps, np.uint32)]
+    return lib().pp_solve_exact_static(int(L), keep[0][1], keep[1][1], int(k), keep[2][1], keep[3][1],
+                                       ctypes.c_void_p(solution_ptr), ctypes.c_void_p(cuda_stream))
