@@ -223,6 +223,17 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         return PP_ERR_NOMEM;
     }
 
+    // constants of the register-tiled sweep, when the instance is inside its envelope
+    std::vector<unsigned char> fmeta;
+    bool has_fast = false;
+    try {
+        fmeta.resize(fast_meta_bytes());
+        has_fast = p->elem == 2 && p->Lpad <= 256 && k >= 2 &&
+                   fast_meta_build(L, k, p->lo.data(), fmeta.data());
+    } catch (const std::bad_alloc &) {
+        delete p;
+        return PP_ERR_NOMEM;
+    }
     // upload the small arrays in one allocation
     struct Part { const void *src; size_t bytes; size_t off; };
     std::vector<Part> parts = {
@@ -232,7 +243,8 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         {p->ubw.data(), p->ubw.size() * 4, 0},
         {p->masks.data(), p->masks.size() * 4, 0},     {p->level_off.data(), p->level_off.size() * 4, 0},
         {nullptr, 8, 0} /* best */,                    {nullptr, 4, 0} /* err */,
-        {nullptr, sizeof(pp_solution), 0} /* solution */};
+        {nullptr, sizeof(pp_solution), 0} /* solution */,
+        {fmeta.data(), fmeta.size(), 0}};
     size_t total = 0;
     for (auto &q : parts) { q.off = total; total = align_up(total + q.bytes, 256); }
     cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&p->d_inputs), total);
@@ -263,6 +275,7 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     d.best = reinterpret_cast<unsigned long long *>(b + parts[9].off);
     d.err = reinterpret_cast<int32_t *>(b + parts[10].off);
     p->d_sol = reinterpret_cast<pp_solution *>(b + parts[11].off);
+    d.fast_meta = has_fast ? b + parts[12].off : nullptr;
     *out = p;
     return PP_OK;
 }

@@ -33,6 +33,7 @@ struct Dev {
     void *table;               // [2^k * k * Lpad] state rows, row (S, v) at (S*k+v)*Lpad
     unsigned long long *best;  // packed (rank, popcount, mask, v) of the best final state
     int32_t *err;              // device error word (0 = fine)
+    const void *fast_meta;     // per-node window constants of the register-tiled sweep, or null
 };
 
 static constexpr unsigned long long kNoBest = ~0ull;
@@ -47,6 +48,8 @@ __host__ __device__ inline unsigned long long pack_best(uint32_t rank, int popc,
 cudaError_t launch_rank_build(const Dev &d, cudaStream_t s, int *launches);
 cudaError_t launch_base(const Dev &d, cudaStream_t s);
 cudaError_t launch_sweep_generic(const Dev &d, int level, cudaStream_t s);
+size_t fast_meta_bytes();
+bool fast_meta_build(int L, int k, const int16_t *lo, void *out);
 bool fast_sweep_supported(const Dev &d);
 cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s);
 cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s);

@@ -214,6 +214,20 @@ def random_small(seed: int, L: int, k: int, *, tight: bool = False, dead_links: 
     return Instance(L, k, bits, mem, cap, bw, f"small[{seed}]")
 
 
+def uniform_memory_small(seed: int, L: int, k: int, wmin: int = 8, wmax: int | None = None, *,
+                         ties: bool = False, dead_links: float = 0.0) -> Instance:
+    """Small instance whose layers all need the same memory (a stack of identical blocks), so
+    that node w holds any run of at most W_w consecutive layers; W_w is drawn from [wmin, wmax]."""
+    base = random_small(seed, L, k, ties=ties, dead_links=dead_links)
+    wmax = wmax if wmax is not None else L + 4
+    unit = 1_000_000
+    widths = stream(10, seed, F_CAP).uniform_int(wmin, max(wmin, wmax), k)
+    slack = stream(10, seed, F_AUX).uniform_int(0, unit - 1, k)
+    cap = widths * np.uint64(unit) + slack
+    mem = np.full(L, unit, dtype=np.uint64)
+    return Instance(L, k, base.layer_out_bits, mem, cap, base.bw_kbps, f"uniform[{seed}]")
+
+
 def random_plans(inst: Instance, count: int, seed: int, invalid_fraction: float = 0.1):
     """Candidate plans for the batched evaluator: random segment counts, random strictly
     increasing segment ends, random distinct nodes; a fraction is corrupted on purpose

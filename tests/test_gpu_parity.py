@@ -116,6 +116,43 @@ def test_state_table_element_by_element(generic):
             _compare_rows(inst, p, rows)
 
 
+def test_register_tiled_sweep_on_uniform_memory_chains():
+    # chains of identical layers take the register-tiled sweep kernel; rows of every raggedness
+    # (L not a multiple of 8 or 16, one lane up to all 32 lanes), every window remainder r = W % 8
+    # and block count q = W // 8, windows wider than the chain, ties and dead links
+    n_fast = 0
+    seed = 0
+    for L, k, wmin, wmax, n in ((9, 3, 8, 9, 6), (12, 5, 8, 10, 10), (17, 6, 8, 13, 10), (31, 4, 8, 16, 12),
+                                (40, 6, 8, 30, 10), (64, 5, 9, 40, 8), (100, 7, 8, 60, 6),
+                                (129, 4, 8, 70, 6), (200, 6, 21, 85, 4), (255, 3, 8, 140, 6),
+                                (256, 4, 15, 300, 4), (23, 2, 8, 14, 6), (50, 5, 8, 60, 6)):
+        for i in range(n):
+            inst = W.uniform_memory_small(80000 + seed, L, k, wmin, wmax, ties=(i % 3 == 1),
+                                          dead_links=0.25 if i % 3 == 2 else 0.0)
+            seed += 1
+            want = oracle.dp_fact(inst, 4, want_table=(L * (1 << k) <= 16384))
+            with pp.Problem.from_instance(inst) as p:
+                got = p.solve_exact()
+                assert p.last_solve_profile().fast_path == 1, inst.name
+                n_fast += 1
+                assert_same(inst, got, want)
+                if want.table is not None:
+                    for S in range(1, 1 << k):
+                        for v in range(k):
+                            if S >> v & 1 and bin(S).count("1") <= L:
+                                assert np.array_equal(p.debug_read_state_row(S, v), want.table[S, v]), \
+                                    (inst.name, S, v)
+                p.force_generic(1)
+                assert_same(inst, p.solve_exact(), want)
+                assert p.last_solve_profile().fast_path == 0
+    assert n_fast >= 80
+    # a node whose window is narrower than 8 layers sends the instance to the generic kernel
+    inst = W.uniform_memory_small(81000, 30, 4, 3, 7)
+    with pp.Problem.from_instance(inst) as p:
+        assert_same(inst, p.solve_exact(), oracle.dp_fact(inst))
+        assert p.last_solve_profile().fast_path == 0
+
+
 def test_named_configs_2_and_3():
     for inst in (W.config_resnet50_shaped(), W.config_deeper_cnn()):
         want = oracle.dp_fact(inst, 8)
@@ -142,7 +179,7 @@ def test_large_config_full_size():
         assert_same(inst, got, want)
         assert oracle.eval_plan(inst, *got.plan()) == (got.beta_ms, 0)
         prof = p.last_solve_profile()
-        assert prof.state_bytes == 2
+        assert prof.state_bytes == 2 and prof.fast_path == 1
         rng = np.random.default_rng(9)
         for size in (1, 2, 3, 5, 7, 8):
             nodes = sorted(int(x) for x in rng.choice(inst.k, size=size, replace=False))
