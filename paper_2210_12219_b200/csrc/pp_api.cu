@@ -228,7 +228,7 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     bool has_fast = false;
     try {
         fmeta.resize(fast_meta_bytes());
-        has_fast = p->elem == 2 && p->Lpad <= 256 && k >= 2 &&
+        has_fast = p->elem == 2 && p->Lpad <= 240 && k >= 2 &&
                    fast_meta_build(L, k, p->lo.data(), fmeta.data());
     } catch (const std::bad_alloc &) {
         delete p;

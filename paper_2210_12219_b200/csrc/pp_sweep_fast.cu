@@ -1,19 +1,22 @@
 // Register-tiled sweep of one popcount level for 16-bit ranks.
 //
-// Envelope: 16-bit state elements, Lpad <= 256, the whole rank table in shared memory, and for
-// every node w a sliding window of constant width:  lo_w(c') = max(0, c' - W_w), W_w >= 8 (chains
-// whose layers all need the same memory, e.g. stacks of identical blocks).  Anything else runs on
-// the generic kernel.
+// Envelope: 16-bit state elements, Lpad <= 240 (rows occupy at most 30 lanes), the whole rank
+// table in shared memory, and for every node w a sliding window of constant width:
+// lo_w(c') = max(0, c' - W_w), W_w >= 8 (chains whose layers all need the same memory, e.g.
+// stacks of identical blocks).  Anything else runs on the generic kernel.
 //
 // Mapping: one warp per source mask S.  Lane l owns the 8 consecutive cut positions 8l..8l+7 of
 // every row, as four packed u16x2 registers (one 16-byte vector).  The |S| source rows
-// dp[S][v][.] are loaded once into registers; for every target node w not in S the warp
+// dp[S][v][.] are loaded once into registers; then, two target nodes w not in S at a time (their
+// instruction streams interleaved so that one's shuffle latency hides behind the other), the warp
 //   1. relaxes   g[c] = min_v max(dp[S][v][c], rank[w][v][c])    (one 128-bit shared-memory load
 //      and eight packed min/max per (v, w) and lane),
 //   2. takes the window minimum  out[c'] = min g[c'-W .. c'-1]   with blocks of 8 = lanes:
 //      window = tail of the block that holds c'-W  (in-lane suffix minima, fetched by shuffles)
-//             + whole blocks in between            (sliding minimum over the 32 block minima)
+//             + whole blocks in between            (sliding minimum over the block minima)
 //             + head of the own block              (in-lane exclusive prefix minima),
+//      all of it branch-free: what a node does not need is a shuffle from distance 31, which
+//      finds no source lane and leaves the accumulator alone,
 //   3. writes row dp[S + w][w][.] with one 16-byte store per lane.
 // Row (S + w, w) has the single source mask S, so no two warps ever write the same row.
 #include "pp_internal.cuh"
@@ -25,15 +28,18 @@ namespace {
 constexpr int kFastThreads = 512;
 constexpr uint32_t kInf2 = 0xFFFFFFFFu;
 
-// per-target-node constants of the window step, precomputed on the host side of the launch
-struct WMeta {
-    int q, r;        // W = 8q + r
+// Per-target-node constants of the window step (W = 8q + r, e = r >> 1), built on the host.
+// A shuffle distance of 31 means "nothing": rows occupy at most 30 lanes, so no lane that holds
+// data finds a source and +inf (or the untouched accumulator) results.
+struct alignas(16) WMeta {
+    int de[4];       // source distance of suffix register j: q, or q + 1 when j < e
+    int dx;          // q + 1: the extra register that an odd r needs
     int sh16;        // 16 if r is odd else 0
-    int rr;          // r >> 1
-    int jm;          // index of the register that mixes two source lanes (r odd), else -1
-    int n1;          // q - 1: whole blocks between, for outputs at in-block positions >= r
-    int s;           // floor(log2(n1)) when n1 >= 1
-    int d2;          // 1 + n1 - 2^s
+    int rot1, rot2;  // e & 1, e & 2: rotate the suffix registers by e before they travel
+    int dd[4];       // doubling distances 1, 2, 4, 8 for the first s steps, then 31
+    int d1, d2;      // T1 = min(D << d1, D << d2): 1 and 1 + n1 - 2^s, or 31 when n1 = q - 1 = 0
+    int dq;          // q: the one more block that positions below r need
+    int pad;
     uint32_t sel[4]; // byte selectors that pick T(q) or T(q-1) per half of each register
 };
 
@@ -53,11 +59,93 @@ __device__ __forceinline__ uint32_t vmax2(uint32_t a, uint32_t b)
     asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
     return r;
 }
-// shuffle up by delta lanes, +inf shifted in from below lane 0
-__device__ __forceinline__ uint32_t shfl_up_inf(uint32_t x, int delta, int lane)
+// shuffle up by delta (<= 31) lanes, +inf shifted in from below lane 0
+__device__ __forceinline__ uint32_t shfl_up_inf(uint32_t x, int delta)
 {
-    uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, delta > 31 ? 31 : delta);
-    return lane >= delta ? y : kInf2;
+    uint32_t y;
+    asm volatile("{ .reg .pred p; shfl.sync.up.b32 %0|p, %1, %2, 0, 0xffffffff; @!p mov.b32 %0, 0xffffffff; }"
+                 : "=r"(y) : "r"(x), "r"(delta));
+    return y;
+}
+// acc = min(acc, x shifted up by delta lanes); lanes without a source keep acc
+__device__ __forceinline__ void min_shfl_up(uint32_t &acc, uint32_t x, int delta)
+{
+    asm volatile("{ .reg .pred p; .reg .b32 t; shfl.sync.up.b32 t|p, %1, %2, 0, 0xffffffff; @p min.u16x2 %0, %0, t; }"
+                 : "+r"(acc) : "r"(x), "r"(delta));
+}
+
+constexpr int NT = 2;  // target nodes processed together
+
+// Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].
+__device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mp,
+                                           uint32_t (&o)[NT][4])
+{
+    uint32_t z[NT][4], B[NT];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+        // pair minima replicated in both halves, their prefix (q*) and suffix (t*) minima
+        const uint32_t m0 = vmin2(r[t][0], __byte_perm(r[t][0], 0, 0x1032));
+        const uint32_t m1 = vmin2(r[t][1], __byte_perm(r[t][1], 0, 0x1032));
+        const uint32_t m2 = vmin2(r[t][2], __byte_perm(r[t][2], 0, 0x1032));
+        const uint32_t m3 = vmin2(r[t][3], __byte_perm(r[t][3], 0, 0x1032));
+        const uint32_t q1 = vmin2(m0, m1), q2 = vmin2(q1, m2);
+        const uint32_t t2 = vmin2(m2, m3), t1 = vmin2(m1, t2);
+        B[t] = vmin2(q2, m3);
+        // exclusive in-lane prefix minima: (min g[0..2j-1], min g[0..2j])
+        o[t][0] = __byte_perm(r[t][0], kInf2, 0x1044);
+        o[t][1] = vmin2(m0, __byte_perm(r[t][1], kInf2, 0x1044));
+        o[t][2] = vmin2(q1, __byte_perm(r[t][2], kInf2, 0x1044));
+        o[t][3] = vmin2(q2, __byte_perm(r[t][3], kInf2, 0x1044));
+        // inclusive in-lane suffix minima: (min g[2j..7], min g[2j+1..7])
+        const uint32_t s0 = vmin2(__byte_perm(m0, r[t][0], 0x7610), t1);
+        const uint32_t s1 = vmin2(__byte_perm(m1, r[t][1], 0x7610), t2);
+        const uint32_t s2 = vmin2(__byte_perm(m2, r[t][2], 0x7610), m3);
+        const uint32_t s3 = __byte_perm(m3, r[t][3], 0x7610);
+        // rotate the four suffix registers right by e = r >> 1 so that register j is the one
+        // output register j needs, whichever lane it comes from
+        const bool p1 = mp[t]->rot1 != 0, p2 = mp[t]->rot2 != 0;
+        const uint32_t a0 = p1 ? s3 : s0, a1 = p1 ? s0 : s1, a2 = p1 ? s1 : s2, a3 = p1 ? s2 : s3;
+        z[t][0] = p2 ? a2 : a0;
+        z[t][1] = p2 ? a3 : a1;
+        z[t][2] = p2 ? a0 : a2;
+        z[t][3] = p2 ? a1 : a3;
+    }
+    // tail of the block that holds c' - W: registers from lane l-q (or l-q-1 for j < e); for an
+    // odd r every output register straddles two of them and is funnel-shifted by 16 bits
+    uint32_t f[NT][5];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) f[t][0] = shfl_up_inf(z[t][3], mp[t]->dx);
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int t = 0; t < NT; ++t) f[t][j + 1] = shfl_up_inf(z[t][j], mp[t]->de[j]);
+    // whole blocks in between: D = min B[l-2^s+1 .. l], T1 = min B[l-n1 .. l-1], T2 = min B[l-q .. l-1]
+    uint32_t D[NT], T1[NT], T2[NT];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) D[t] = B[t];
+#pragma unroll
+    for (int st = 0; st < 4; ++st)
+#pragma unroll
+        for (int t = 0; t < NT; ++t) min_shfl_up(D[t], D[t], mp[t]->dd[st]);
+#pragma unroll
+    for (int t = 0; t < NT; ++t) T1[t] = shfl_up_inf(D[t], mp[t]->d1);
+#pragma unroll
+    for (int t = 0; t < NT; ++t) min_shfl_up(T1[t], D[t], mp[t]->d2);
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+        T2[t] = T1[t];
+        min_shfl_up(T2[t], B[t], mp[t]->dq);
+    }
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+        const int sh = mp[t]->sh16;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t e = __funnelshift_l(f[t][j], f[t][j + 1], sh);
+            const uint32_t mid = __byte_perm(T2[t], T1[t], mp[t]->sel[j]);
+            o[t][j] = vmin2(vmin2(o[t][j], e), mid);
+        }
+    }
 }
 
 template <int NV>
@@ -74,7 +162,8 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(d.rank);
         for (int i = threadIdx.x; i < rank_elems / 8; i += kFastThreads) smem4[i] = src[i];
-        for (int i = threadIdx.x; i < 32; i += kFastThreads) smem4[rank_elems / 8 + i] = make_uint4(kInf2, kInf2, kInf2, kInf2);
+        for (int i = threadIdx.x; i < 32; i += kFastThreads)
+            smem4[rank_elems / 8 + i] = make_uint4(kInf2, kInf2, kInf2, kInf2);
         const int *ms = reinterpret_cast<const int *>(meta_g);
         int *md = reinterpret_cast<int *>(wm);
         for (int i = threadIdx.x; i < (int)(sizeof(WMeta) / 4) * k; i += kFastThreads) md[i] = ms[i];
@@ -90,11 +179,14 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
     const uint32_t first = d.level_off[level - 1];
     const uint32_t nmask = d.level_off[level] - first;
     const uint32_t full = (1u << k) - 1u;
-    const int last_lane = (L - 1) >> 3, last_reg = ((L - 1) & 7) >> 1, last_half = (L - 1) & 1;
+    const int last_lane = (L - 1) >> 3, last_reg = ((L - 1) & 7) >> 1, last_sh = ((L - 1) & 1) * 16;
+    const uint32_t stride = gridDim.x * (kFastThreads / 32);
 
-    for (uint32_t mi = blockIdx.x * (kFastThreads / 32) + warp; mi < nmask;
-         mi += gridDim.x * (kFastThreads / 32)) {
-        const uint32_t S = d.masks[first + mi];
+    uint32_t mi = blockIdx.x * (kFastThreads / 32) + warp;
+    uint32_t S = mi < nmask ? d.masks[first + mi] : 0u;
+    while (mi < nmask) {
+        const uint32_t mi_next = mi + stride;
+        const uint32_t S_next = mi_next < nmask ? d.masks[first + mi_next] : 0u;
         int voff[NV];
         uint4 dp[NV];
         {
@@ -111,91 +203,61 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
                 dp[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(src + voff[vi]))
                                 : make_uint4(kInf2, kInf2, kInf2, kInf2);
         }
-        for (uint32_t wrem = full & ~S; wrem; wrem &= wrem - 1) {
-            const int w = __ffs(wrem) - 1;
+        // best final key seen so far: read once per mask, not once per row (a stale value only
+        // costs a redundant atomic)
+        unsigned long long best_seen = *reinterpret_cast<volatile unsigned long long *>(d.best);
+        uint32_t wrem = full & ~S;
+        while (wrem) {
+            int w[NT];
+            const WMeta *mp[NT];
+            const uint16_t *rw[NT];
+#pragma unroll
+            for (int t = 0; t < NT; ++t) {
+                w[t] = __ffs(wrem) - 1;
+                if (wrem & (wrem - 1)) wrem &= wrem - 1;  // an odd tail repeats its last node
+                else if (t == NT - 1) wrem = 0;
+                mp[t] = wm + w[t];
+                rw[t] = rank_s + w[t] * k * Lpad + 8 * lane;
+            }
             // ---- 1. relax over the source nodes ----
-            const uint16_t *rw = rank_s + w * k * Lpad + 8 * lane;
-            uint32_t r0 = kInf2, r1 = kInf2, r2 = kInf2, r3 = kInf2;
+            uint32_t r[NT][4], o[NT][4];
+#pragma unroll
+            for (int t = 0; t < NT; ++t) r[t][0] = r[t][1] = r[t][2] = r[t][3] = kInf2;
 #pragma unroll
             for (int vi = 0; vi < NV; ++vi) {
-                const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[vi]);
-                r0 = vmin2(r0, vmax2(dp[vi].x, g.x));
-                r1 = vmin2(r1, vmax2(dp[vi].y, g.y));
-                r2 = vmin2(r2, vmax2(dp[vi].z, g.z));
-                r3 = vmin2(r3, vmax2(dp[vi].w, g.w));
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    const uint4 g = *reinterpret_cast<const uint4 *>(rw[t] + voff[vi]);
+                    r[t][0] = vmin2(r[t][0], vmax2(dp[vi].x, g.x));
+                    r[t][1] = vmin2(r[t][1], vmax2(dp[vi].y, g.y));
+                    r[t][2] = vmin2(r[t][2], vmax2(dp[vi].z, g.z));
+                    r[t][3] = vmin2(r[t][3], vmax2(dp[vi].w, g.w));
+                }
             }
             // ---- 2. window minimum ----
-            const WMeta m = wm[w];
-            // pair minima replicated in both halves, their prefix (q*) and suffix (t*) minima
-            const uint32_t m0 = vmin2(r0, __byte_perm(r0, 0, 0x1032));
-            const uint32_t m1 = vmin2(r1, __byte_perm(r1, 0, 0x1032));
-            const uint32_t m2 = vmin2(r2, __byte_perm(r2, 0, 0x1032));
-            const uint32_t m3 = vmin2(r3, __byte_perm(r3, 0, 0x1032));
-            const uint32_t q1 = vmin2(m0, m1), q2 = vmin2(q1, m2), B = vmin2(q2, m3);
-            const uint32_t t2 = vmin2(m2, m3), t1 = vmin2(m1, t2);
-            // exclusive in-lane prefix minima: (min g[0..2j-1], min g[0..2j])
-            uint32_t o0 = (r0 << 16) | 0xFFFFu;
-            uint32_t o1 = vmin2(m0, (r1 << 16) | 0xFFFFu);
-            uint32_t o2 = vmin2(q1, (r2 << 16) | 0xFFFFu);
-            uint32_t o3 = vmin2(q2, (r3 << 16) | 0xFFFFu);
-            // inclusive in-lane suffix minima: (min g[2j..7], min g[2j+1..7])
-            uint32_t z0 = vmin2(__byte_perm(m0, r0, 0x7610), t1);
-            uint32_t z1 = vmin2(__byte_perm(m1, r1, 0x7610), t2);
-            uint32_t z2 = vmin2(__byte_perm(m2, r2, 0x7610), m3);
-            uint32_t z3 = __byte_perm(m3, r3, 0x7610);
-            // rotate the 8 suffix minima right by r positions inside the lane
-            {
-                const uint32_t a0 = __funnelshift_l(z3, z0, m.sh16), a1 = __funnelshift_l(z0, z1, m.sh16);
-                const uint32_t a2 = __funnelshift_l(z1, z2, m.sh16), a3 = __funnelshift_l(z2, z3, m.sh16);
-                z0 = a0; z1 = a1; z2 = a2; z3 = a3;
-                if (m.rr & 1) { const uint32_t t = z3; z3 = z2; z2 = z1; z1 = z0; z0 = t; }
-                if (m.rr & 2) { uint32_t t = z0; z0 = z2; z2 = t; t = z1; z1 = z3; z3 = t; }
-            }
-            // fetch: positions >= r come from lane l-q, positions < r from lane l-q-1
-            {
-                const int dq = m.q, r = m.r;
-                uint32_t e0 = shfl_up_inf(z0, dq + (1 < r), lane);
-                uint32_t e1 = shfl_up_inf(z1, dq + (3 < r), lane);
-                uint32_t e2 = shfl_up_inf(z2, dq + (5 < r), lane);
-                uint32_t e3 = shfl_up_inf(z3, dq + (7 < r), lane);
-                if (m.jm >= 0) {  // r odd: register jm takes its low half from one lane further down
-                    const uint32_t zz = m.jm == 0 ? z0 : (m.jm == 1 ? z1 : (m.jm == 2 ? z2 : z3));
-                    const uint32_t x = shfl_up_inf(zz, dq + 1, lane);
-                    if (m.jm == 0) e0 = __byte_perm(x, e0, 0x7610);
-                    else if (m.jm == 1) e1 = __byte_perm(x, e1, 0x7610);
-                    else if (m.jm == 2) e2 = __byte_perm(x, e2, 0x7610);
-                    else e3 = __byte_perm(x, e3, 0x7610);
-                }
-                o0 = vmin2(o0, e0); o1 = vmin2(o1, e1); o2 = vmin2(o2, e2); o3 = vmin2(o3, e3);
-            }
-            // whole blocks in between: T1 = min B[l-n1 .. l-1], T2 = min B[l-q .. l-1]
-            {
-                uint32_t T1 = kInf2;
-                if (m.n1 >= 1) {
-                    uint32_t D = B;  // D = min B[l-2^s+1 .. l] after s doubling steps
-                    for (int st = 0; st < m.s; ++st) D = vmin2(D, shfl_up_inf(D, 1 << st, lane));
-                    T1 = vmin2(shfl_up_inf(D, 1, lane), shfl_up_inf(D, m.d2, lane));
-                }
-                const uint32_t T2 = vmin2(T1, shfl_up_inf(B, m.q, lane));
-                o0 = vmin2(o0, __byte_perm(T2, T1, m.sel[0]));
-                o1 = vmin2(o1, __byte_perm(T2, T1, m.sel[1]));
-                o2 = vmin2(o2, __byte_perm(T2, T1, m.sel[2]));
-                o3 = vmin2(o3, __byte_perm(T2, T1, m.sel[3]));
-            }
-            // ---- 3. write the row, offer its last element as a final state ----
-            const uint32_t S2 = S | (1u << w);
-            if (active)
-                *reinterpret_cast<uint4 *>(table_w + ((size_t)S2 * k + w) * Lpad + 8 * lane) =
-                    make_uint4(o0, o1, o2, o3);
-            if (lane == last_lane) {
-                const uint32_t reg = last_reg == 0 ? o0 : (last_reg == 1 ? o1 : (last_reg == 2 ? o2 : o3));
-                const uint32_t val = last_half ? (reg >> 16) : (reg & 0xFFFFu);
-                if (val != 0xFFFFu) {
-                    const unsigned long long key = pack_best(val, level, S2, w);
-                    if (key < *reinterpret_cast<volatile unsigned long long *>(d.best)) atomicMin(d.best, key);
+            window_min(r, mp, o);
+            // ---- 3. write the rows, offer their last elements as final states ----
+#pragma unroll
+            for (int t = 0; t < NT; ++t) {
+                const uint32_t S2 = S | (1u << w[t]);
+                if (active)
+                    *reinterpret_cast<uint4 *>(table_w + ((size_t)S2 * k + w[t]) * Lpad + 8 * lane) =
+                        make_uint4(o[t][0], o[t][1], o[t][2], o[t][3]);
+                if (lane == last_lane) {
+                    const uint32_t reg = last_reg == 0 ? o[t][0] : (last_reg == 1 ? o[t][1] : (last_reg == 2 ? o[t][2] : o[t][3]));
+                    const uint32_t val = (reg >> last_sh) & 0xFFFFu;
+                    if (val != 0xFFFFu) {
+                        const unsigned long long key = pack_best(val, level, S2, w[t]);
+                        if (key < best_seen) {
+                            atomicMin(d.best, key);
+                            best_seen = key;
+                        }
+                    }
                 }
             }
         }
+        mi = mi_next;
+        S = S_next;
     }
 }
 
@@ -231,24 +293,30 @@ bool fast_meta_build(int L, int k, const int16_t *lo, void *out)
         if (L > 1 && W < 8) return false;
         if (W >= L - 1) W = Lpad;  // the window always reaches layer 0: treat as "everything before"
         WMeta &m = fm->w[w];
-        m.q = W >> 3;
-        m.r = W & 7;
-        m.sh16 = (m.r & 1) ? 16 : 0;
-        m.rr = m.r >> 1;
-        m.jm = (m.r & 1) ? (m.r >> 1) : -1;
-        m.n1 = m.q - 1;
-        m.s = 0;
-        while (m.n1 >= 1 && (2 << m.s) <= m.n1) ++m.s;
-        m.d2 = 1 + m.n1 - (1 << m.s);
+        const int q = W >> 3, r = W & 7, e = r >> 1;
+        auto clamp = [](int x) { return x > 31 ? 31 : x; };
+        for (int j = 0; j < 4; ++j) m.de[j] = clamp(q + (j < e ? 1 : 0));
+        m.dx = (r & 1) ? clamp(q + 1) : 31;
+        m.sh16 = (r & 1) ? 16 : 0;
+        m.rot1 = e & 1;
+        m.rot2 = e & 2;
+        const int n1 = q - 1 > 31 ? 31 : q - 1;
+        int s = 0;
+        while (n1 >= 1 && (2 << s) <= n1) ++s;
+        for (int st = 0; st < 4; ++st) m.dd[st] = (n1 >= 1 && st < s) ? (1 << st) : 31;
+        m.d1 = n1 >= 1 ? 1 : 31;
+        m.d2 = n1 >= 1 ? 1 + n1 - (1 << s) : 31;
+        m.dq = clamp(q);
+        m.pad = 0;
         for (int j = 0; j < 4; ++j)
-            m.sel[j] = ((2 * j < m.r) ? 0x0010u : 0x0054u) | ((2 * j + 1 < m.r) ? 0x3200u : 0x7600u);
+            m.sel[j] = ((2 * j < r) ? 0x0010u : 0x0054u) | ((2 * j + 1 < r) ? 0x3200u : 0x7600u);
     }
     return true;
 }
 
 bool fast_sweep_supported(const Dev &d)
 {
-    if (d.elem != 2 || d.Lpad > 256 || d.k < 2 || d.k > 19 + 1 || !d.fast_meta) return false;
+    if (d.elem != 2 || d.Lpad > 240 || d.k < 2 || d.k > PP_MAX_K || !d.fast_meta) return false;
     int dev = 0, max_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&max_sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;

@@ -1,0 +1,47 @@
+"""Small driver for profilers: solves the Large instance restricted to its first --k nodes.
+
+    python -m paper_2210_12219_b200.profile_case --k 16 --solves 2
+
+With k = 16 the state table is 0.44 GB (still far above the 126 MB L2), small enough for a
+multi-pass counter capture of single sweep launches.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+
+import numpy as np
+
+
+def main():
+    import torch
+
+    import paper_2210_12219_b200 as pp
+    from paper_2210_12219_b200 import build
+    from paper_2210_12219_b200 import workloads as W
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--k", type=int, default=16)
+    ap.add_argument("--solves", type=int, default=2)
+    ap.add_argument("--generic", action="store_true")
+    args = ap.parse_args()
+    build.build()
+    large = W.config_large()
+    k = args.k
+    inst = W.Instance(large.L, k, large.layer_out_bits, large.layer_mem_bytes,
+                      large.node_mem_bytes[:k].copy(), np.ascontiguousarray(large.bw_kbps[:k, :k]))
+    sol = torch.zeros(ctypes.sizeof(pp.pp_solution) // 8, dtype=torch.float64, device="cuda")
+    with pp.Problem.from_instance(inst) as p:
+        if args.generic:
+            p.force_generic(1)
+        for _ in range(args.solves):
+            p.solve_exact_dev(sol.data_ptr())
+        torch.cuda.synchronize()
+        prof = p.last_solve_profile()
+        rec = pp.pp_solution.from_buffer_copy(sol.cpu().numpy().tobytes())
+        print("k=%d L=%d beta=%.6f m=%d sweep=%.3f ms total=%.3f ms fast=%d" %
+              (k, inst.L, rec.beta_ms, rec.m, prof.ms_sweep, prof.ms_total, prof.fast_path))
+
+
+if __name__ == "__main__":
+    main()

@@ -124,8 +124,8 @@ def test_register_tiled_sweep_on_uniform_memory_chains():
     seed = 0
     for L, k, wmin, wmax, n in ((9, 3, 8, 9, 6), (12, 5, 8, 10, 10), (17, 6, 8, 13, 10), (31, 4, 8, 16, 12),
                                 (40, 6, 8, 30, 10), (64, 5, 9, 40, 8), (100, 7, 8, 60, 6),
-                                (129, 4, 8, 70, 6), (200, 6, 21, 85, 4), (255, 3, 8, 140, 6),
-                                (256, 4, 15, 300, 4), (23, 2, 8, 14, 6), (50, 5, 8, 60, 6)):
+                                (129, 4, 8, 70, 6), (200, 6, 21, 85, 4), (239, 3, 8, 140, 6),
+                                (240, 4, 15, 300, 4), (23, 2, 8, 14, 6), (50, 5, 8, 60, 6)):
         for i in range(n):
             inst = W.uniform_memory_small(80000 + seed, L, k, wmin, wmax, ties=(i % 3 == 1),
                                           dead_links=0.25 if i % 3 == 2 else 0.0)
