@@ -7,10 +7,11 @@
 
 namespace pp {
 
-constexpr int kBatchThreads = 256;
+constexpr int kBatchThreads = 1024;
+constexpr int kBatchWarps = kBatchThreads / 32;
 
 struct BatchLayout {
-    size_t dp, gam, M, cap, lo, rowoff, mlist, loff, total;
+    size_t dp, gam, gs, M, cap, lo, rowoff, mlist, loff, total;
 };
 
 __host__ __device__ inline BatchLayout batch_layout(int L, int k)
@@ -20,6 +21,7 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     size_t o = 0;
     b.dp = o;      o += rows * L * sizeof(double);
     b.gam = o;     o += (size_t)L * k * k * sizeof(double);
+    b.gs = o;      o += (size_t)kBatchWarps * L * sizeof(double);
     b.M = o;       o += (size_t)(L + 1) * sizeof(uint64_t);
     b.cap = o;     o += (size_t)k * sizeof(uint64_t);
     b.rowoff = o;  o += ((size_t)1 << k) * sizeof(uint32_t);
@@ -48,7 +50,11 @@ __device__ inline uint32_t bits_below(uint32_t S, int k)
     return t;
 }
 
-__global__ void __launch_bounds__(kBatchThreads)
+// Work split inside a block: one warp per target row (S', w), lanes over the cut position.  The
+// warp first forms g[c] = min_v max(dp[S'\{w}][v][c], gamma[c][v][w]) into its own shared-memory
+// strip, then every lane scans its window [lo_w(c'), c'-1] of that strip.  Rows, gamma[v][w][.]
+// and the strip are all read with consecutive lanes on consecutive addresses.
+__global__ void __launch_bounds__(kBatchThreads, 1)
 k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
         const uint32_t *__restrict__ g_bw, double *__restrict__ o_beta, int32_t *__restrict__ o_m,
@@ -57,20 +63,21 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     extern __shared__ __align__(16) unsigned char smem[];
     const BatchLayout lay = batch_layout(L, k);
     double *dp = reinterpret_cast<double *>(smem + lay.dp);
-    double *gam = reinterpret_cast<double *>(smem + lay.gam);
+    double *gam = reinterpret_cast<double *>(smem + lay.gam);  // [v][w][c]
     uint64_t *M = reinterpret_cast<uint64_t *>(smem + lay.M);
     uint64_t *cap = reinterpret_cast<uint64_t *>(smem + lay.cap);
     uint32_t *rowoff = reinterpret_cast<uint32_t *>(smem + lay.rowoff);
     uint32_t *loff = reinterpret_cast<uint32_t *>(smem + lay.loff);
     uint16_t *mlist = reinterpret_cast<uint16_t *>(smem + lay.mlist);
     int16_t *lo = reinterpret_cast<int16_t *>(smem + lay.lo);
-    __shared__ unsigned long long s_val[kBatchThreads / 32];
-    __shared__ unsigned int s_tie[kBatchThreads / 32];
+    __shared__ unsigned long long s_val[kBatchWarps];
+    __shared__ unsigned int s_tie[kBatchWarps];
     __shared__ unsigned long long s_bestval;
     __shared__ unsigned int s_besttie;
     __shared__ int s_bad;
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    double *gs = reinterpret_cast<double *>(smem + lay.gs) + (size_t)wid * L;
     const uint32_t nm = 1u << k;
     const double kInf = __longlong_as_double(0x7FF0000000000000ll);
     const unsigned long long kInfBits = 0x7FF0000000000000ull;
@@ -104,7 +111,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         if (tid < k) cap[tid] = g_cap[inst * k + tid];
         __syncthreads();
         for (int e = tid; e < L * k * k; e += kBatchThreads) {
-            int c = e / (k * k), r = e - c * k * k, v = r / k, w = r - v * k;
+            int r = e / L, c = e - r * L, v = r / k, w = r - v * k;
             uint64_t b = bits[c];
             uint32_t link = bw[r];
             if (b >= PP_MAX_BITS || link >= PP_MAX_KBPS) s_bad = 1;
@@ -126,27 +133,37 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const int bad = s_bad;
         const int jmax = k < L ? k : L;
         for (int j = 2; j <= k; ++j) {
-            const uint32_t nmask = loff[j + 1] - loff[j];
-            const uint32_t items = nmask * j * L;
-            for (uint32_t it = tid; it < items; it += kBatchThreads) {
-                uint32_t mi = it / (j * L), r = it - mi * j * L;
-                int wi = r / L, c2 = r - wi * L;
-                uint32_t S2 = mlist[loff[j] + mi];
-                int w = __fns(S2, 0, wi + 1);
-                uint32_t P = S2 & ~(1u << w);
-                double best = kInf;
-                if (j <= jmax) {
-                    int l0 = lo[w * L + c2];
-                    for (uint32_t rem = P; rem; rem &= rem - 1) {
-                        int v = __ffs(rem) - 1;
-                        const double *src = dp + (size_t)(rowoff[P] + __popc(P & ((1u << v) - 1u))) * L;
-                        for (int c = l0; c < c2; ++c) {
-                            double cand = fmax(src[c], gam[(c * k + v) * k + w]);
-                            best = fmin(best, cand);
-                        }
-                    }
+            const uint32_t nrows = (loff[j + 1] - loff[j]) * j;
+            for (uint32_t rr = wid; rr < nrows; rr += kBatchWarps) {
+                const uint32_t mi = rr / j;
+                const int wi = rr - mi * j;
+                const uint32_t S2 = mlist[loff[j] + mi];
+                uint32_t t = S2;
+                for (int i = 0; i < wi; ++i) t &= t - 1;
+                const int w = __ffs(t) - 1;
+                const uint32_t P = S2 & ~(1u << w);
+                double *out = dp + (size_t)(rowoff[S2] + wi) * L;
+                if (j > jmax) {
+                    for (int c = lane; c < L; c += 32) out[c] = kInf;
+                    continue;
                 }
-                dp[(size_t)(rowoff[S2] + wi) * L + c2] = best;
+                const double *src0 = dp + (size_t)rowoff[P] * L;
+                for (int c = lane; c < L; c += 32) {
+                    double g = kInf;
+                    int vi = 0;
+                    for (uint32_t rem = P; rem; rem &= rem - 1, ++vi) {
+                        const int v = __ffs(rem) - 1;
+                        g = fmin(g, fmax(src0[vi * L + c], gam[(v * k + w) * L + c]));
+                    }
+                    gs[c] = g;
+                }
+                __syncwarp();
+                for (int c2 = lane; c2 < L; c2 += 32) {
+                    double best = kInf;
+                    for (int c = lo[w * L + c2]; c < c2; ++c) best = fmin(best, gs[c]);
+                    out[c2] = best;
+                }
+                __syncwarp();
             }
             __syncthreads();
         }
@@ -214,7 +231,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                     int c = l0 + it / k, v = it - (it / k) * k;
                     if (!((P >> v) & 1u)) continue;
                     double a = dp[(size_t)(rowoff[P] + __popc(P & ((1u << v) - 1u))) * L + c];
-                    double cand = fmax(a, gam[(c * k + v) * k + w]);
+                    double cand = fmax(a, gam[(v * k + w) * L + c]);
                     if (cand <= bstar) {
                         unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
                         pick = kk < pick ? kk : pick;

@@ -77,9 +77,23 @@ __device__ __forceinline__ void min_shfl_up(uint32_t &acc, uint32_t x, int delta
 constexpr int NT = 2;  // target nodes processed together
 
 // Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].
-__device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mp,
+__device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mptr,
                                            uint32_t (&o)[NT][4])
 {
+    // the constants of each node arrive as five 16-byte shared-memory loads
+    union MetaRegs {
+        WMeta m;
+        uint4 q[sizeof(WMeta) / 16];
+    };
+    MetaRegs mr[NT];
+#pragma unroll
+    for (int t = 0; t < NT; ++t)
+#pragma unroll
+        for (int i = 0; i < (int)(sizeof(WMeta) / 16); ++i)
+            mr[t].q[i] = reinterpret_cast<const uint4 *>(mptr[t])[i];
+    const WMeta *mp[NT];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) mp[t] = &mr[t].m;
     uint32_t z[NT][4], B[NT];
 #pragma unroll
     for (int t = 0; t < NT; ++t) {
@@ -152,6 +166,10 @@ template <int NV>
 __global__ void __launch_bounds__(kFastThreads, 1)
 k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
 {
+    // Programmatic dependent launch: let the next level's blocks be scheduled as soon as this
+    // level's blocks retire, so that their prologue (rank table -> shared memory) overlaps our
+    // tail.  Nothing the previous level wrote is touched before griddepcontrol.wait below.
+    asm volatile("griddepcontrol.launch_dependents;");
     extern __shared__ uint4 smem4[];
     uint16_t *rank_s = reinterpret_cast<uint16_t *>(smem4);
     const int k = d.k, L = d.L, Lpad = d.Lpad;
@@ -169,6 +187,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
         for (int i = threadIdx.x; i < (int)(sizeof(WMeta) / 4) * k; i += kFastThreads) md[i] = ms[i];
     }
     __syncthreads();
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -202,6 +221,17 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
             for (int vi = 0; vi < NV; ++vi)
                 dp[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(src + voff[vi]))
                                 : make_uint4(kInf2, kInf2, kInf2, kInf2);
+        }
+        // pull the next mask's source rows into L2 while this mask is being processed
+        if (mi_next < nmask && active && (lane & 7) == 0) {
+            uint32_t rem = S_next;
+            const uint16_t *src = table + (size_t)S_next * k * Lpad + 8 * lane;
+#pragma unroll
+            for (int vi = 0; vi < NV; ++vi) {
+                int v = __ffs(rem) - 1;
+                rem &= rem - 1;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(src + v * Lpad));
+            }
         }
         // best final key seen so far: read once per mask, not once per row (a stale value only
         // costs a redundant atomic)
@@ -271,8 +301,17 @@ cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned gr
 {
     cudaError_t e = cudaFuncSetAttribute(k_sweep_fast<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    k_sweep_fast<NV><<<grid, kFastThreads, sm, s>>>(d, level, meta);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kFastThreads);
+    cfg.dynamicSmemBytes = sm;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_sweep_fast<NV>, d, level, meta);
 }
 
 }  // namespace
