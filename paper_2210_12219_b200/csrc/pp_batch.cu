@@ -1,60 +1,83 @@
 // Many-instance exact search: one thread block per instance, the whole state table in shared
-// memory.  Same recurrence, final choice and backtrack rule as the single-instance path (see
-// pp_sweep.cu), but small enough that values are kept as the gamma doubles themselves:
-// fmin/fmax on non-negative doubles only select, so results are bit-identical to the ranked
-// path.  Global memory sees the inputs once and the result record once.
+// memory as 16-bit ranks.  Same recurrence, final choice and backtrack rule as the
+// single-instance path (see pp_sweep.cu); global memory sees the inputs once and the result
+// record once.
+//
+// Per instance the block
+//   1. stages the inputs, builds the memory prefix sums and the window table lo[w][c'];
+//   2. rank-compresses gamma (Eq. 3): layers sorted by bits, distinct bandwidths listed, one fp64
+//      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, counted by
+//      merging every pair of the sorted lists (IEEE division is monotone in the numerator);
+//   3. sweeps the popcount levels with a flat thread <-> (target row, position) mapping:
+//      phase A forms g[c] = min_v max(dp[S'\{w}][v][c], rank[v][w][c]) for every row of the level,
+//      two neighbouring positions per thread as one packed u16x2 word,
+//      phase B takes the window minimum over [lo_w(c'), c'-1];
+//   4. reduces the final states to the smallest (value, popcount, mask, node), walks back with
+//      the threshold rule, and maps the winning rank back to its quotient.
 #include "pp_internal.cuh"
 
 namespace pp {
 
-constexpr int kBatchThreads = 1024;
+constexpr int kBatchThreads = 512;
 constexpr int kBatchWarps = kBatchThreads / 32;
+constexpr uint16_t kInf16 = 0xFFFFu;
 
 struct BatchLayout {
-    size_t dp, gam, gs, M, cap, lo, rowoff, mlist, loff, total;
+    size_t dp, g, rank, gu, rk, cnt, M, cap, bits, sbits, bw, ubw, pair_u, pos, lo, rowoff, loff, rowinfo, total;
 };
 
 __host__ __device__ inline BatchLayout batch_layout(int L, int k)
 {
     BatchLayout b;
-    size_t rows = (size_t)k << (k - 1);
+    const size_t rows = (size_t)k << (k - 1);
+    // widest level: max_j C(k, j) * j
+    size_t best = 0, binom = 1;
+    for (int j = 1; j <= k; ++j) {
+        binom = binom * (size_t)(k - j + 1) / (size_t)j;
+        if (binom * j > best) best = binom * j;
+    }
+    const size_t U = (size_t)k * (k - 1) > 0 ? (size_t)k * (k - 1) : 1;
+    const size_t Ls = ((size_t)L + 1) & ~(size_t)1;  // row stride of the 16-bit tables: even, so that
+                                                     // two neighbouring cut positions form one word
     size_t o = 0;
-    b.dp = o;      o += rows * L * sizeof(double);
-    b.gam = o;     o += (size_t)L * k * k * sizeof(double);
-    b.gs = o;      o += (size_t)kBatchWarps * L * sizeof(double);
-    b.M = o;       o += (size_t)(L + 1) * sizeof(uint64_t);
-    b.cap = o;     o += (size_t)k * sizeof(uint64_t);
-    b.rowoff = o;  o += ((size_t)1 << k) * sizeof(uint32_t);
-    b.loff = o;    o += (size_t)(k + 2) * sizeof(uint32_t);
-    b.mlist = o;   o += ((size_t)1 << k) * sizeof(uint16_t);
-    b.lo = o;      o += (size_t)k * L * sizeof(int16_t);
-    b.total = (o + 15) & ~(size_t)15;
+    auto take = [&o](size_t bytes) { size_t at = o; o = (o + bytes + 15) & ~(size_t)15; return at; };
+    b.gu = take(U * L * sizeof(double));
+    b.M = take((size_t)(L + 1) * sizeof(uint64_t));
+    b.cap = take((size_t)k * sizeof(uint64_t));
+    b.bits = take((size_t)L * sizeof(uint64_t));
+    b.sbits = take((size_t)L * sizeof(uint64_t));
+    b.bw = take((size_t)k * k * sizeof(uint32_t));
+    b.ubw = take(U * sizeof(uint32_t));
+    b.rowoff = take(((size_t)1 << k) * sizeof(uint32_t));
+    b.loff = take((size_t)(k + 2) * sizeof(uint32_t));
+    b.rowinfo = take(rows * sizeof(uint32_t));
+    b.dp = take(rows * Ls * sizeof(uint16_t));
+    b.g = take(best * Ls * sizeof(uint16_t));
+    b.rank = take((size_t)k * k * Ls * sizeof(uint16_t));
+    b.rk = take(U * L * sizeof(uint16_t));
+    b.cnt = take(U * L * sizeof(uint32_t));
+    b.pair_u = take((size_t)k * k * sizeof(int16_t));
+    b.pos = take((size_t)L * sizeof(int16_t));
+    b.lo = take((size_t)k * L * sizeof(int16_t));
+    b.total = o;
     return b;
 }
 
 size_t batch_smem_bytes(int L, int k)
 {
-    if (k > 15) return (size_t)1 << 40;
+    if (k > 12) return (size_t)1 << 40;  // row descriptors hold the mask in 12 bits
+    if ((size_t)k * (k - 1) * L + 1 > 65534) return (size_t)1 << 40;  // ranks must fit 16 bits
     return batch_layout(L, k).total;
 }
 
-// number of set bits in all integers below S
-__device__ inline uint32_t bits_below(uint32_t S, int k)
+// row descriptor: source mask (12 bits) | target node (4 bits) << 12 | compact row of the first
+// source row << 16 (the output row is the descriptor's own index)
+__device__ __forceinline__ uint32_t info_pack(uint32_t P, int w, uint32_t src0)
 {
-    uint32_t t = 0;
-    for (int b = 0; b < k; ++b) {
-        uint32_t cyc = (S >> (b + 1)) << b;
-        uint32_t rem = S & ((2u << b) - 1u);
-        t += cyc + (rem > (1u << b) ? rem - (1u << b) : 0u);
-    }
-    return t;
+    return P | ((uint32_t)w << 12) | (src0 << 16);
 }
 
-// Work split inside a block: one warp per target row (S', w), lanes over the cut position.  The
-// warp first forms g[c] = min_v max(dp[S'\{w}][v][c], gamma[c][v][w]) into its own shared-memory
-// strip, then every lane scans its window [lo_w(c'), c'-1] of that strip.  Rows, gamma[v][w][.]
-// and the strip are all read with consecutive lanes on consecutive addresses.
-__global__ void __launch_bounds__(kBatchThreads, 1)
+__global__ void __launch_bounds__(kBatchThreads)
 k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
         const uint32_t *__restrict__ g_bw, double *__restrict__ o_beta, int32_t *__restrict__ o_m,
@@ -62,145 +85,230 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const BatchLayout lay = batch_layout(L, k);
-    double *dp = reinterpret_cast<double *>(smem + lay.dp);
-    double *gam = reinterpret_cast<double *>(smem + lay.gam);  // [v][w][c]
+    double *gu = reinterpret_cast<double *>(smem + lay.gu);          // [U][L] ascending in i
     uint64_t *M = reinterpret_cast<uint64_t *>(smem + lay.M);
     uint64_t *cap = reinterpret_cast<uint64_t *>(smem + lay.cap);
+    uint64_t *s_bits = reinterpret_cast<uint64_t *>(smem + lay.bits);
+    uint64_t *s_sorted = reinterpret_cast<uint64_t *>(smem + lay.sbits);
+    uint32_t *s_bw = reinterpret_cast<uint32_t *>(smem + lay.bw);
+    uint32_t *ubw = reinterpret_cast<uint32_t *>(smem + lay.ubw);
     uint32_t *rowoff = reinterpret_cast<uint32_t *>(smem + lay.rowoff);
-    uint32_t *loff = reinterpret_cast<uint32_t *>(smem + lay.loff);
-    uint16_t *mlist = reinterpret_cast<uint16_t *>(smem + lay.mlist);
+    uint32_t *loff = reinterpret_cast<uint32_t *>(smem + lay.loff);    // first compact row of each level
+    uint32_t *rowinfo = reinterpret_cast<uint32_t *>(smem + lay.rowinfo);
+    uint16_t *dp = reinterpret_cast<uint16_t *>(smem + lay.dp);        // [compact row][L]
+    uint16_t *gbuf = reinterpret_cast<uint16_t *>(smem + lay.g);       // [row within level][L]
+    uint16_t *rank = reinterpret_cast<uint16_t *>(smem + lay.rank);    // [v][w][c]
+    uint16_t *rk = reinterpret_cast<uint16_t *>(smem + lay.rk);        // [U][L]
+    uint32_t *cnt = reinterpret_cast<uint32_t *>(smem + lay.cnt);      // [U][L]
+    int16_t *pair_u = reinterpret_cast<int16_t *>(smem + lay.pair_u);
+    int16_t *pos = reinterpret_cast<int16_t *>(smem + lay.pos);
     int16_t *lo = reinterpret_cast<int16_t *>(smem + lay.lo);
-    __shared__ unsigned long long s_val[kBatchWarps];
-    __shared__ unsigned int s_tie[kBatchWarps];
-    __shared__ unsigned long long s_bestval;
-    __shared__ unsigned int s_besttie;
-    __shared__ int s_bad;
+    __shared__ unsigned long long s_key[kBatchWarps];
+    __shared__ unsigned long long s_best;
+    __shared__ int s_bad, s_U;
 
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    double *gs = reinterpret_cast<double *>(smem + lay.gs) + (size_t)wid * L;
     const uint32_t nm = 1u << k;
+    const int Ls = (L + 1) & ~1, Lh = Ls >> 1;  // row stride (even) and words per row
+    // a thread's items advance by the block size: (row, column) moves by (dr, dc) with one carry
+    const int drA = kBatchThreads / Lh, dcA = kBatchThreads - drA * Lh;
+    const int drB = kBatchThreads / L, dcB = kBatchThreads - drB * L;
     const double kInf = __longlong_as_double(0x7FF0000000000000ll);
-    const unsigned long long kInfBits = 0x7FF0000000000000ull;
 
-    // instance-independent tables
-    for (uint32_t S = tid; S < nm; S += kBatchThreads) rowoff[S] = bits_below(S, k);
-    if (tid <= k) {  // thread j lists the masks of popcount j
-        uint32_t cnt = 0;
-        for (uint32_t S = 0; S < nm; ++S) cnt += (__popc(S) < tid);
+    // ---- instance-independent tables -------------------------------------------------------
+    // Compact rows are ordered by (popcount, mask, node), so the rows of a level are contiguous.
+    // rowoff[S] = compact row of (S, lowest node of S); loff[j] = first row of level j.
+    if (tid <= k + 1) {
+        uint32_t cnt = 0;  // rows of all masks with popcount below tid
+        for (uint32_t S = 0; S < nm; ++S) cnt += (__popc(S) < tid) ? __popc(S) : 0;
         loff[tid] = cnt;
-        if (tid == k) loff[k + 1] = nm;
     }
     __syncthreads();
-    if (tid <= k) {
-        uint32_t at = loff[tid];
-        for (uint32_t S = 0; S < nm; ++S)
-            if (__popc(S) == tid) mlist[at++] = (uint16_t)S;
+    for (uint32_t S = tid; S < nm; S += kBatchThreads) {
+        const int pc = __popc(S);
+        uint32_t before = 0;  // masks of the same popcount below S
+        for (uint32_t T = 0; T < S; ++T) before += (__popc(T) == pc);
+        rowoff[S] = loff[pc] + before * pc;
     }
+    __syncthreads();
+    for (uint32_t S = 1 + tid; S < nm; S += kBatchThreads) {
+        int wi = 0;
+        for (uint32_t rem = S; rem; rem &= rem - 1, ++wi) {
+            const int w = __ffs(rem) - 1;
+            const uint32_t P = S & ~(1u << w);
+            rowinfo[rowoff[S] + wi] = info_pack(P, w, P ? rowoff[P] : 0u);
+        }
+    }
+    const int jmax = k < L ? k : L;
 
     for (int64_t inst = blockIdx.x; inst < B; inst += gridDim.x) {
         const uint64_t *bits = g_bits + inst * L;
         const uint64_t *mem = g_mem + inst * L;
         const uint32_t *bw = g_bw + inst * k * k;
         __syncthreads();
+        // ---- 1. stage inputs, prefix sums, windows ----
+        for (int i = tid; i < L; i += kBatchThreads) {
+            s_bits[i] = bits[i];
+            M[i + 1] = mem[i];
+        }
+        for (int i = tid; i < k * k; i += kBatchThreads) s_bw[i] = bw[i];
+        if (tid < k) cap[tid] = g_cap[inst * k + tid];
+        if (tid == 0) s_bad = 0;
+        __syncthreads();
         if (tid == 0) {
-            s_bad = 0;
             uint64_t acc = 0;
             M[0] = 0;
-            for (int i = 0; i < L; ++i) { acc += mem[i]; M[i + 1] = acc; }
+            for (int i = 1; i <= L; ++i) { acc += M[i]; M[i] = acc; }
+        } else if (tid == 32 % kBatchThreads) {
+            // distinct usable bandwidths, in order of first appearance
+            int U = 0;
+            for (int p = 0; p < k * k; ++p) {
+                const int v = p / k, w = p - v * k;
+                const uint32_t b = s_bw[p];
+                int u = -1;
+                if (v != w && b != 0) {
+                    for (int i = 0; i < U && u < 0; ++i)
+                        if (ubw[i] == b) u = i;
+                    if (u < 0) { u = U; ubw[U++] = b; }
+                }
+                pair_u[p] = (int16_t)u;
+            }
+            s_U = U;
         }
-        if (tid < k) cap[tid] = g_cap[inst * k + tid];
+        // layers in ascending order of bits (ties by index)
+        for (int c = tid; c < L; c += kBatchThreads) {
+            const uint64_t b = s_bits[c];
+            int p = 0;
+            for (int o = 0; o < L; ++o) {
+                const uint64_t x = s_bits[o];
+                p += (x < b) || (x == b && o < c);
+            }
+            pos[c] = (int16_t)p;
+            s_sorted[p] = b;
+            if (b >= PP_MAX_BITS) s_bad = 1;
+        }
+        for (int i = tid; i < k * k; i += kBatchThreads)
+            if (s_bw[i] >= PP_MAX_KBPS) s_bad = 1;
         __syncthreads();
-        for (int e = tid; e < L * k * k; e += kBatchThreads) {
-            int r = e / L, c = e - r * L, v = r / k, w = r - v * k;
-            uint64_t b = bits[c];
-            uint32_t link = bw[r];
-            if (b >= PP_MAX_BITS || link >= PP_MAX_KBPS) s_bad = 1;
-            gam[e] = (v == w || link == 0) ? kInf : __ddiv_rn((double)b, (double)link);
-        }
-        // lo[w][c'] = first c >= 0 such that layers c+1..c' fit on w (c' if none)
+        const int U = s_U;
         for (int e = tid; e < k * L; e += kBatchThreads) {
-            int w = e / L, c2 = e - w * L;
+            const int w = e / L, c2 = e - w * L;
             int c = c2;  // step down while the segment starting at layer c (previous cut c-1) fits
             while (c > 0 && M[c2 + 1] - M[c] <= cap[w]) --c;
             lo[e] = (int16_t)c;
         }
-        // base frontier
-        for (int e = tid; e < k * L; e += kBatchThreads) {
-            int v = e / L, c = e - v * L;
-            dp[(size_t)rowoff[1u << v] * L + c] = (M[c + 1] <= cap[v]) ? 0.0 : kInf;
+        // ---- 2. quotients and their ranks ----
+        for (int e = tid; e < U * L; e += kBatchThreads) {
+            const int u = e / L, i = e - u * L;
+            gu[e] = __ddiv_rn((double)s_sorted[i], (double)ubw[u]);
+            cnt[e] = 0;
         }
         __syncthreads();
-        const int bad = s_bad;
-        const int jmax = k < L ? k : L;
+        // one task per ordered pair of lists: walk list u (queries, ascending) against list u2
+        for (int t = tid; t < U * U; t += kBatchThreads) {
+            const int u = t / U, u2 = t - u * U;
+            const double *q = gu + u * L, *other = gu + u2 * L;
+            int j = 0;  // entries of `other` below the current query
+            double oj = other[0];
+            for (int i = 0; i < L; ++i) {
+                const double x = q[i];
+                while (j < L && oj < x) {
+                    ++j;
+                    if (j < L) oj = other[j];
+                }
+                if (j) atomicAdd(&cnt[u * L + i], (unsigned)j);
+            }
+        }
+        __syncthreads();
+        for (int e = tid; e < U * L; e += kBatchThreads) rk[e] = (uint16_t)(1u + cnt[e]);
+        __syncthreads();
+        for (int e = tid; e < k * k * Ls; e += kBatchThreads) {
+            const int r = e / Ls, c = e - r * Ls;
+            const int u = pair_u[r];
+            rank[e] = (u < 0 || c >= L) ? kInf16 : rk[u * L + pos[c]];
+        }
+        // base frontier
+        for (int e = tid; e < k * Ls; e += kBatchThreads) {
+            const int v = e / Ls, c = e - v * Ls;
+            dp[(size_t)rowoff[1u << v] * Ls + c] = (c < L && M[c + 1] <= cap[v]) ? (uint16_t)0 : kInf16;
+        }
+        __syncthreads();
+        // ---- 3. levels ----
         for (int j = 2; j <= k; ++j) {
-            const uint32_t nrows = (loff[j + 1] - loff[j]) * j;
-            for (uint32_t rr = wid; rr < nrows; rr += kBatchWarps) {
-                const uint32_t mi = rr / j;
-                const int wi = rr - mi * j;
-                const uint32_t S2 = mlist[loff[j] + mi];
-                uint32_t t = S2;
-                for (int i = 0; i < wi; ++i) t &= t - 1;
-                const int w = __ffs(t) - 1;
-                const uint32_t P = S2 & ~(1u << w);
-                double *out = dp + (size_t)(rowoff[S2] + wi) * L;
-                if (j > jmax) {
-                    for (int c = lane; c < L; c += 32) out[c] = kInf;
-                    continue;
-                }
-                const double *src0 = dp + (size_t)rowoff[P] * L;
-                for (int c = lane; c < L; c += 32) {
-                    double g = kInf;
-                    int vi = 0;
-                    for (uint32_t rem = P; rem; rem &= rem - 1, ++vi) {
+            const uint32_t row0 = loff[j], nrows = loff[j + 1] - row0;
+            if (j > jmax) {
+                for (uint32_t it = tid; it < nrows * Ls; it += kBatchThreads) dp[(size_t)row0 * Ls + it] = kInf16;
+                __syncthreads();
+                continue;
+            }
+            {  // phase A: thread <-> (row, word of two positions)
+                int rr = tid / Lh, cw = tid - rr * Lh;
+                while (rr < (int)nrows) {
+                    const uint32_t info = rowinfo[row0 + rr];
+                    const int w = (info >> 12) & 15;
+                    const uint32_t *src = reinterpret_cast<const uint32_t *>(dp + (size_t)(info >> 16) * Ls) + cw;
+                    const uint32_t *rw = reinterpret_cast<const uint32_t *>(rank + w * Ls) + cw;
+                    uint32_t g = 0xFFFFFFFFu;
+                    for (uint32_t rem = info & 0xFFFu; rem; rem &= rem - 1) {
                         const int v = __ffs(rem) - 1;
-                        g = fmin(g, fmax(src0[vi * L + c], gam[(v * k + w) * L + c]));
+                        g = __vminu2(g, __vmaxu2(*src, rw[v * k * Lh]));
+                        src += Lh;
                     }
-                    gs[c] = g;
+                    reinterpret_cast<uint32_t *>(gbuf)[rr * Lh + cw] = g;
+                    rr += drA;
+                    cw += dcA;
+                    if (cw >= Lh) { cw -= Lh; ++rr; }
                 }
-                __syncwarp();
-                for (int c2 = lane; c2 < L; c2 += 32) {
-                    double best = kInf;
-                    for (int c = lo[w * L + c2]; c < c2; ++c) best = fmin(best, gs[c]);
-                    out[c2] = best;
+            }
+            __syncthreads();
+            {  // phase B: thread <-> (row, position)
+                int rr = tid / L, c2 = tid - rr * L;
+                while (rr < (int)nrows) {
+                    const int w = (rowinfo[row0 + rr] >> 12) & 15;
+                    const uint16_t *gr = gbuf + rr * Ls;
+                    uint32_t best = kInf16;
+                    for (int c = lo[w * L + c2]; c < c2; ++c) {
+                        const uint32_t x = gr[c];
+                        best = x < best ? x : best;
+                    }
+                    dp[(size_t)(row0 + rr) * Ls + c2] = (uint16_t)best;
+                    rr += drB;
+                    c2 += dcB;
+                    if (c2 >= L) { c2 -= L; ++rr; }
                 }
-                __syncwarp();
             }
             __syncthreads();
         }
-        // final state: lexicographic minimum of (value, popcount, mask, node) at c = L-1
-        unsigned long long bv = kInfBits;
-        unsigned int bt = 0xFFFFFFFFu;
-        for (uint32_t e = tid; e < nm * (uint32_t)k; e += kBatchThreads) {
-            uint32_t S = e / k;
-            int v = e - S * k;
-            if (!((S >> v) & 1u)) continue;
-            double x = dp[(size_t)(rowoff[S] + __popc(S & ((1u << v) - 1u))) * L + (L - 1)];
-            unsigned long long xb = (unsigned long long)__double_as_longlong(x);
-            unsigned int tie = ((unsigned)__popc(S) << 25) | (S << 5) | (unsigned)v;
-            if (xb < bv || (xb == bv && tie < bt)) { bv = xb; bt = tie; }
+        // ---- 4. final state: smallest (value, popcount, mask, node) at c = L-1 ----
+        unsigned long long key = kNoBest;
+        for (uint32_t row = tid; row < loff[k + 1]; row += kBatchThreads) {
+            const uint32_t x = dp[(size_t)row * Ls + (L - 1)];
+            if (x == kInf16) continue;
+            const uint32_t info = rowinfo[row];
+            const int w = (info >> 12) & 15;
+            const uint32_t S = (info & 0xFFFu) | (1u << w);
+            const unsigned long long cand = pack_best(x, __popc(S), S, w);
+            key = cand < key ? cand : key;
         }
         for (int o = 16; o; o >>= 1) {
-            unsigned long long ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
-            unsigned int ot = __shfl_xor_sync(0xFFFFFFFFu, bt, o);
-            if (ov < bv || (ov == bv && ot < bt)) { bv = ov; bt = ot; }
+            const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, key, o);
+            key = other < key ? other : key;
         }
-        if (lane == 0) { s_val[wid] = bv; s_tie[wid] = bt; }
+        if (lane == 0) s_key[wid] = key;
         __syncthreads();
         if (tid == 0) {
-            for (int i = 1; i < kBatchThreads / 32; ++i)
-                if (s_val[i] < bv || (s_val[i] == bv && s_tie[i] < bt)) { bv = s_val[i]; bt = s_tie[i]; }
-            s_bestval = bv;
-            s_besttie = bt;
+            for (int i = 1; i < kBatchWarps; ++i) key = s_key[i] < key ? s_key[i] : key;
+            s_best = key;
         }
         __syncthreads();
-        bv = s_bestval;
-        bt = s_besttie;
+        key = s_best;
+        const int bad = s_bad;
         int32_t *cuts = o_cuts ? o_cuts + inst * (k - 1) : nullptr;
         int32_t *place = o_place + inst * k;
         if (tid < k) place[tid] = -1;
         if (cuts && tid < k - 1) cuts[tid] = -1;
         __syncthreads();
-        if (bad || bv >= kInfBits) {
+        if (bad || key == kNoBest) {
             if (tid == 0) {
                 o_beta[inst] = kInf;
                 o_m[inst] = 0;
@@ -208,11 +316,22 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             }
             continue;
         }
-        if (wid == 0) {  // backtrack by one warp
-            const double bstar = __longlong_as_double((long long)bv);
-            const int m = (int)(bt >> 25);
-            uint32_t S = (bt >> 5) & 0xFFFFFu;
-            int w = (int)(bt & 31u), c2 = L - 1;
+        if (wid == 0) {  // value of the winning rank, then the backtrack, by one warp
+            const uint32_t rstar = (uint32_t)(key >> 30);
+            const int m = (int)((key >> 25) & 31);
+            uint32_t S = (uint32_t)((key >> 5) & 0xFFFFF);
+            int w = (int)(key & 31), c2 = L - 1;
+            double bstar = 0.0;
+            if (rstar != 0) {
+                int found = -1;
+                for (int e = lane; e < U * L; e += 32)
+                    if (rk[e] == rstar) found = e;
+                for (int o = 16; o; o >>= 1) {
+                    const int other = __shfl_xor_sync(0xFFFFFFFFu, found, o);
+                    found = other > found ? other : found;
+                }
+                bstar = gu[found];  // equal ranks hold equal doubles
+            }
             if (lane == 0) {
                 o_beta[inst] = bstar;
                 o_m[inst] = m;
@@ -224,21 +343,22 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                     if (j < m - 1) cuts[j] = c2;
                 }
                 if (j == 0) break;
-                uint32_t P = S & ~(1u << w);
-                int l0 = lo[w * L + c2];
+                const uint32_t P = S & ~(1u << w);
+                const int l0 = lo[w * L + c2];
                 unsigned int pick = 0xFFFFFFFFu;
                 for (int it = lane; it < (c2 - l0) * k; it += 32) {
-                    int c = l0 + it / k, v = it - (it / k) * k;
+                    const int c = l0 + it / k, v = it - (it / k) * k;
                     if (!((P >> v) & 1u)) continue;
-                    double a = dp[(size_t)(rowoff[P] + __popc(P & ((1u << v) - 1u))) * L + c];
-                    double cand = fmax(a, gam[(v * k + w) * L + c]);
-                    if (cand <= bstar) {
-                        unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
+                    const uint32_t a = dp[(size_t)(rowoff[P] + __popc(P & ((1u << v) - 1u))) * Ls + c];
+                    const uint32_t b = rank[(v * k + w) * Ls + c];
+                    const uint32_t mx = a > b ? a : b;
+                    if (mx <= rstar) {
+                        const unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
                         pick = kk < pick ? kk : pick;
                     }
                 }
                 for (int o = 16; o; o >>= 1) {
-                    unsigned int other = __shfl_xor_sync(0xFFFFFFFFu, pick, o);
+                    const unsigned int other = __shfl_xor_sync(0xFFFFFFFFu, pick, o);
                     pick = other < pick ? other : pick;
                 }
                 if (pick == 0xFFFFFFFFu) {  // inconsistent table: flag the instance, keep going

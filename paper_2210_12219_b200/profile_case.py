@@ -1,6 +1,7 @@
 """Small driver for profilers: solves the Large instance restricted to its first --k nodes.
 
     python -m paper_2210_12219_b200.profile_case --k 16 --solves 2
+    python -m paper_2210_12219_b200.profile_case --batch 4096 --solves 1
 
 With k = 16 the state table is 0.44 GB (still far above the 126 MB L2), small enough for a
 multi-pass counter capture of single sweep launches.
@@ -24,8 +25,17 @@ def main():
     ap.add_argument("--k", type=int, default=16)
     ap.add_argument("--solves", type=int, default=2)
     ap.add_argument("--generic", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="solve this many batched instances instead")
     args = ap.parse_args()
     build.build()
+    if args.batch:
+        insts = W.config_batched(args.batch)
+        stack = lambda f: np.stack([f(i) for i in insts])
+        for _ in range(args.solves):
+            got = pp.solve_exact_batch(24, 8, stack(lambda i: i.layer_out_bits), stack(lambda i: i.layer_mem_bytes),
+                                       stack(lambda i: i.node_mem_bytes), stack(lambda i: i.bw_kbps))
+        print("batch of %d: %d feasible" % (args.batch, int((got.status == 0).sum())))
+        return
     large = W.config_large()
     k = args.k
     inst = W.Instance(large.L, k, large.layer_out_bits, large.layer_mem_bytes,
