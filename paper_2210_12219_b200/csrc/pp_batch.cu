@@ -7,7 +7,7 @@
 //   1. stages the inputs, builds the memory prefix sums and the window table lo[w][c'];
 //   2. rank-compresses gamma (Eq. 3): layers sorted by bits, distinct bandwidths listed, one fp64
 //      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, counted by
-//      merging every pair of the sorted lists (IEEE division is monotone in the numerator);
+//      binary search in each of the sorted lists (IEEE division is monotone in the numerator);
 //   3. sweeps the popcount levels with a flat thread <-> (target row, position) mapping:
 //      phase A forms g[c] = min_v max(dp[S'\{w}][v][c], rank[v][w][c]) for every row of the level,
 //      two neighbouring positions per thread as one packed u16x2 word,
@@ -77,7 +77,7 @@ __device__ __forceinline__ uint32_t info_pack(uint32_t P, int w, uint32_t src0)
     return P | ((uint32_t)w << 12) | (src0 << 16);
 }
 
-__global__ void __launch_bounds__(kBatchThreads)
+__global__ void __launch_bounds__(kBatchThreads, 2)
 k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
         const uint32_t *__restrict__ g_bw, double *__restrict__ o_beta, int32_t *__restrict__ o_m,
@@ -159,21 +159,21 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             uint64_t acc = 0;
             M[0] = 0;
             for (int i = 1; i <= L; ++i) { acc += M[i]; M[i] = acc; }
-        } else if (tid == 32 % kBatchThreads) {
-            // distinct usable bandwidths, in order of first appearance
-            int U = 0;
-            for (int p = 0; p < k * k; ++p) {
-                const int v = p / k, w = p - v * k;
-                const uint32_t b = s_bw[p];
-                int u = -1;
-                if (v != w && b != 0) {
-                    for (int i = 0; i < U && u < 0; ++i)
-                        if (ubw[i] == b) u = i;
-                    if (u < 0) { u = U; ubw[U++] = b; }
+        }
+        // distinct usable bandwidths in order of first appearance, one thread per node pair:
+        // first_p[p] = earliest pair with the same bandwidth, then its index among the firsts
+        for (int p = tid; p < k * k; p += kBatchThreads) {
+            const int v = p / k, w = p - v * k;
+            const uint32_t b = s_bw[p];
+            int first = -1;
+            if (v != w && b != 0) {
+                first = p;
+                for (int p2 = p - 1; p2 >= 0; --p2) {
+                    const int v2 = p2 / k;
+                    if (v2 != p2 - v2 * k && s_bw[p2] == b) first = p2;
                 }
-                pair_u[p] = (int16_t)u;
             }
-            s_U = U;
+            pair_u[p] = (int16_t)first;  // provisional: pair index of the first occurrence
         }
         // layers in ascending order of bits (ties by index)
         for (int c = tid; c < L; c += kBatchThreads) {
@@ -190,6 +190,23 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         for (int i = tid; i < k * k; i += kBatchThreads)
             if (s_bw[i] >= PP_MAX_KBPS) s_bad = 1;
         __syncthreads();
+        for (int p = tid; p < k * k; p += kBatchThreads) {
+            const int first = pair_u[p];
+            int u = -1;
+            if (first >= 0) {
+                u = 0;
+                for (int p2 = 0; p2 < first; ++p2) u += (pair_u[p2] == p2);
+                if (first == p) ubw[u] = s_bw[p];
+            }
+            reinterpret_cast<int16_t *>(cnt)[p] = (int16_t)u;  // staged: pair_u is still being read
+        }
+        if (tid == kBatchThreads - 1) {
+            int U = 0;
+            for (int p2 = 0; p2 < k * k; ++p2) U += (pair_u[p2] == p2);
+            s_U = U;
+        }
+        __syncthreads();
+        for (int p = tid; p < k * k; p += kBatchThreads) pair_u[p] = reinterpret_cast<int16_t *>(cnt)[p];
         const int U = s_U;
         for (int e = tid; e < k * L; e += kBatchThreads) {
             const int w = e / L, c2 = e - w * L;
@@ -204,19 +221,26 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             cnt[e] = 0;
         }
         __syncthreads();
-        // one task per ordered pair of lists: walk list u (queries, ascending) against list u2
-        for (int t = tid; t < U * U; t += kBatchThreads) {
-            const int u = t / U, u2 = t - u * U;
-            const double *q = gu + u * L, *other = gu + u2 * L;
-            int j = 0;  // entries of `other` below the current query
-            double oj = other[0];
-            for (int i = 0; i < L; ++i) {
-                const double x = q[i];
-                while (j < L && oj < x) {
-                    ++j;
-                    if (j < L) oj = other[j];
+        // one task per (quotient, group of 4 lists): binary search in each list of the group
+        {
+            const int ngrp = (U + 3) >> 2;
+            for (int t = tid; t < U * L * ngrp; t += kBatchThreads) {
+                // consecutive threads search the same lists with consecutive queries, so that a
+                // warp's probes fall into one 8L-byte list instead of one bank
+                const int grp = t / (U * L), e = t - grp * (U * L);
+                const double x = gu[e];
+                unsigned below = 0;
+                const int u_end = (grp * 4 + 4 < U) ? grp * 4 + 4 : U;
+                for (int u2 = grp * 4; u2 < u_end; ++u2) {
+                    const double *list = gu + u2 * L;
+                    int a = 0, b = L;  // first index with list[idx] >= x
+                    while (a < b) {
+                        const int mid = (a + b) >> 1;
+                        if (list[mid] < x) a = mid + 1; else b = mid;
+                    }
+                    below += (unsigned)a;
                 }
-                if (j) atomicAdd(&cnt[u * L + i], (unsigned)j);
+                if (below) atomicAdd(&cnt[e], below);
             }
         }
         __syncthreads();
@@ -267,10 +291,12 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                     const int w = (rowinfo[row0 + rr] >> 12) & 15;
                     const uint16_t *gr = gbuf + rr * Ls;
                     uint32_t best = kInf16;
-                    for (int c = lo[w * L + c2]; c < c2; ++c) {
-                        const uint32_t x = gr[c];
-                        best = x < best ? x : best;
+                    int c = lo[w * L + c2];
+                    for (; c + 4 <= c2; c += 4) {  // four independent loads per trip
+                        const uint32_t x0 = gr[c], x1 = gr[c + 1], x2 = gr[c + 2], x3 = gr[c + 3];
+                        best = min(min(best, min(x0, x1)), min(x2, x3));
                     }
+                    for (; c < c2; ++c) best = min(best, (uint32_t)gr[c]);
                     dp[(size_t)(row0 + rr) * Ls + c2] = (uint16_t)best;
                     rr += drB;
                     c2 += dcB;
