@@ -53,7 +53,7 @@ typedef enum {
     PP_INFEASIBLE = 1, /* not an error: no plan exists; beta = +inf, m = 0 */
     PP_ERR_ARG = -1,   /* null pointer, L < 1, k < 1, B < 0 */
     PP_ERR_LIMIT = -2, /* k > PP_MAX_K, L > PP_MAX_L, value above PP_MAX_BITS / PP_MAX_KBPS,
-                          or (batched solve) a state table that does not fit shared memory */
+                          or (batched solve) a shape whose tables do not fit shared memory */
     PP_ERR_NOMEM = -3, /* host or device allocation failed, or workspace too small */
     PP_ERR_CUDA = -4,  /* a CUDA runtime call failed (includes "no device") */
     PP_ERR_TIMEOUT = -5 /* reserved */
@@ -160,8 +160,9 @@ pp_status pp_eval_plans_dev(pp_problem *p, int64_t B, const uint8_t *nseg, const
  *   out_bits [B*L], mem [B*L], node_mem [B*k], bw [B*k*k]   inputs, instance-major
  *   beta_ms [B], m [B], cuts [B*(k-1)], placement [B*k], status [B] (PP_OK / PP_INFEASIBLE,
  *   or PP_ERR_LIMIT for an instance with a value above the limits)
- * Returns PP_ERR_LIMIT without touching outputs when k * 2^(k-1) * L doubles plus the gamma
- * table exceed the shared memory of one block.  Host variant is synchronous and uses the
+ * Returns PP_ERR_LIMIT without touching outputs when the instance shape does not fit one block:
+ * k > 12, k*(k-1)*L + 1 > 65534 (ranks are 16-bit), or k * 2^(k-1) * L 16-bit states plus the
+ * rank and quotient tables beyond the shared memory of a block (k = 8, L = 24 needs 90 KB).  Host variant is synchronous and uses the
  * legacy default stream; the _dev variant takes device pointers and a stream and is
  * asynchronous.  cuts may be NULL when k == 1.
  */

@@ -51,7 +51,7 @@ pp_status from_cuda(cudaError_t e)
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkLayout {
-    size_t pos, order, gu, rk, rank, table, total;
+    size_t pos, order, gu, rk, inv, rank, table, total;
 };
 
 WorkLayout work_layout(int L, int k, int Lpad, int U, int elem)
@@ -62,6 +62,7 @@ WorkLayout work_layout(int L, int k, int Lpad, int U, int elem)
     w.order = o; o = align_up(o + (size_t)L * 2, 256);
     w.gu = o;    o = align_up(o + (size_t)std::max(U, 1) * L * 8, 256);
     w.rk = o;    o = align_up(o + (size_t)std::max(U, 1) * L * 4, 256);
+    w.inv = o;   o = align_up(o + ((size_t)std::max(U, 1) * L + 2) * 4, 256);
     w.rank = o;  o = align_up(o + (size_t)k * k * Lpad * elem, 256);
     w.table = o; o = align_up(o + ((size_t)k << k) * Lpad * elem, 256);
     w.total = o;
@@ -94,6 +95,7 @@ void bind_work(pp_problem *p)
     p->d.order = reinterpret_cast<int16_t *>(b + w.order);
     p->d.gu = reinterpret_cast<double *>(b + w.gu);
     p->d.rk = reinterpret_cast<uint32_t *>(b + w.rk);
+    p->d.inv = reinterpret_cast<uint32_t *>(b + w.inv);
     p->d.rank = b + w.rank;
     p->d.table = b + w.table;
 }

@@ -29,6 +29,7 @@ struct Dev {
     int16_t *order;            // [L] layer at each position
     double *gu;                // [U*L] gu[u*L+i] = bits[order[i]] / ubw[u]  (ascending in i)
     uint32_t *rk;              // [U*L] rank of gu[u*L+i]
+    uint32_t *inv;             // [U*L+2] inv[r] = some entry e with rk[e] == r (equal ranks hold equal doubles)
     void *rank;                // [k*k*Lpad] rank[(w*k+v)*Lpad + c] of gamma[c][v][w], element type
     void *table;               // [2^k * k * Lpad] state rows, row (S, v) at (S*k+v)*Lpad
     unsigned long long *best;  // packed (rank, popcount, mask, v) of the best final state

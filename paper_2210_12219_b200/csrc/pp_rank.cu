@@ -9,9 +9,13 @@
 
 namespace pp {
 
-// One block: order[] = layers sorted by (bits, index), pos[] = inverse permutation.
-__global__ void k_order(Dev d)
+// One block: order[] = layers sorted by (bits, index), pos[] = inverse permutation, then
+// gu[u][i] = bits[order[i]] / ubw[u], one correctly rounded fp64 division per entry (never
+// contracted, no fast math).
+__global__ void __launch_bounds__(1024) k_order_quotients(Dev d)
 {
+    extern __shared__ unsigned char smem_raw[];
+    uint64_t *sorted = reinterpret_cast<uint64_t *>(smem_raw);  // [L]
     for (int c = threadIdx.x; c < d.L; c += blockDim.x) {
         uint64_t b = d.bits[c];
         int p = 0;
@@ -21,49 +25,57 @@ __global__ void k_order(Dev d)
         }
         d.pos[c] = (int16_t)p;
         d.order[p] = (int16_t)c;
+        sorted[p] = b;
     }
-}
-
-// gu[u][i]: one correctly rounded fp64 division per entry (never contracted, no fast math).
-__global__ void k_quotients(Dev d)
-{
-    int n = d.U * d.L;
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
+    __syncthreads();
+    const int n = d.U * d.L;
+    for (int e = threadIdx.x; e < n; e += blockDim.x) {
         int u = e / d.L, i = e - u * d.L;
-        d.gu[e] = __ddiv_rn((double)d.bits[d.order[i]], (double)d.ubw[u]);
+        d.gu[e] = __ddiv_rn((double)sorted[i], (double)d.ubw[u]);
     }
 }
 
-// rk[u][i] = 1 + #{(u', i') : gu[u'][i'] < gu[u][i]}.
-// Block = one list u (its queries are ascending in i); thread t owns list u' = t, t+blockDim, ...
-// and merges it against the block's list held in shared memory, adding its counts with
-// shared-memory atomics.  Every step advances one of two cursors, so a merge costs <= 2L steps.
-__global__ void k_rank_lists(Dev d)
+// rk[e] = 1 + #{e' : gu[e'] < gu[e]}.  A block owns kRankQueries quotients and streams all U
+// lists through shared memory in tiles; thread (q, g) binary-searches the lists g, g+4, ... of
+// each tile for query q, and the four partial counts meet in a shared-memory atomic.
+constexpr int kRankQueries = 256;
+constexpr int kRankGroups = 4;
+constexpr int kRankTileBytes = 48 * 1024;
+
+__global__ void __launch_bounds__(kRankQueries *kRankGroups) k_rank(Dev d, int tile_lists)
 {
     extern __shared__ unsigned char smem_raw[];
-    double *q = reinterpret_cast<double *>(smem_raw);            // [L] this block's list
-    unsigned int *cnt = reinterpret_cast<unsigned int *>(q + d.L); // [L]
-    const int L = d.L, u = blockIdx.x;
-    for (int i = threadIdx.x; i < L; i += blockDim.x) {
-        q[i] = d.gu[(size_t)u * L + i];
-        cnt[i] = 0;
-    }
-    __syncthreads();
-    for (int u2 = threadIdx.x; u2 < d.U; u2 += blockDim.x) {
-        const double *other = d.gu + (size_t)u2 * L;
-        int j = 0;  // entries of `other` below the current query
-        double oj = other[0];
-        for (int i = 0; i < L; ++i) {
-            double x = q[i];
-            while (j < L && oj < x) {
-                ++j;
-                if (j < L) oj = other[j];
+    double *tile = reinterpret_cast<double *>(smem_raw);  // [tile_lists][L]
+    __shared__ unsigned int s_cnt[kRankQueries];
+    const int L = d.L, U = d.U, n = U * L;
+    const int q = threadIdx.x % kRankQueries, grp = threadIdx.x / kRankQueries;
+    const int e = blockIdx.x * kRankQueries + q;
+    const double x = e < n ? d.gu[e] : 0.0;
+    if (grp == 0) s_cnt[q] = 0;
+    unsigned int below = 0;
+    for (int u0 = 0; u0 < U; u0 += tile_lists) {
+        const int nl = (U - u0 < tile_lists) ? U - u0 : tile_lists;
+        __syncthreads();
+        for (int i = threadIdx.x; i < nl * L; i += blockDim.x) tile[i] = d.gu[(size_t)u0 * L + i];
+        __syncthreads();
+        if (e < n)
+            for (int l = grp; l < nl; l += kRankGroups) {
+                const double *list = tile + l * L;
+                int a = 0, b = L;  // first index with list[idx] >= x
+                while (a < b) {
+                    const int mid = (a + b) >> 1;
+                    if (list[mid] < x) a = mid + 1; else b = mid;
+                }
+                below += (unsigned)a;
             }
-            if (j) atomicAdd(&cnt[i], (unsigned int)j);
-        }
     }
+    if (e < n && below) atomicAdd(&s_cnt[q], below);
     __syncthreads();
-    for (int i = threadIdx.x; i < L; i += blockDim.x) d.rk[(size_t)u * L + i] = 1u + cnt[i];
+    if (grp == 0 && e < n) {
+        const unsigned int r = 1u + s_cnt[q];
+        d.rk[e] = r;
+        d.inv[r] = (uint32_t)e;  // any entry of that rank will do
+    }
 }
 
 template <typename T>
@@ -86,15 +98,17 @@ __global__ void k_expand(Dev d)
 cudaError_t launch_rank_build(const Dev &d, cudaStream_t s, int *launches)
 {
     *launches = 0;
-    k_order<<<1, 256, 0, s>>>(d);
+    k_order_quotients<<<1, 1024, (size_t)d.L * sizeof(uint64_t), s>>>(d);
     ++*launches;
     if (d.U > 0) {
-        int n = d.U * d.L;
-        k_quotients<<<(n + 255) / 256, 256, 0, s>>>(d);
-        ++*launches;
-        size_t sm = (size_t)d.L * (sizeof(double) + sizeof(unsigned int));
-        int threads = d.U < 32 ? 32 : (d.U > 256 ? 256 : ((d.U + 31) / 32) * 32);
-        k_rank_lists<<<d.U, threads, sm, s>>>(d);
+        int tile_lists = kRankTileBytes / (int)(d.L * sizeof(double));
+        if (tile_lists < 1) tile_lists = 1;
+        if (tile_lists > d.U) tile_lists = d.U;
+        const size_t sm = (size_t)tile_lists * d.L * sizeof(double);
+        cudaError_t e = cudaFuncSetAttribute(k_rank, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        if (e != cudaSuccess) return e;
+        const int n = d.U * d.L;
+        k_rank<<<(n + kRankQueries - 1) / kRankQueries, kRankQueries * kRankGroups, sm, s>>>(d, tile_lists);
         ++*launches;
     }
     if (d.elem == 2)

@@ -100,6 +100,7 @@ extern "C" pp_status pp_solve_exact_static(int32_t L, const uint64_t *layer_out_
     const size_t o_order = o; o = up256(o + (size_t)L * 2);
     const size_t o_gu = o;    o = up256(o + (size_t)(U > 0 ? U : 1) * L * 8);
     const size_t o_rk = o;    o = up256(o + (size_t)(U > 0 ? U : 1) * L * 4);
+    const size_t o_inv = o;   o = up256(o + ((size_t)(U > 0 ? U : 1) * L + 2) * 4);
     const size_t o_rank = o;  o = up256(o + (size_t)k * k * Lpad * elem);
     const size_t o_table = o; o = up256(o + ((size_t)k << k) * Lpad * elem);
     if (o > (size_t)PP_STATIC_SCRATCH_BYTES) return PP_ERR_LIMIT;
@@ -161,6 +162,7 @@ extern "C" pp_status pp_solve_exact_static(int32_t L, const uint64_t *layer_out_
     d.order = reinterpret_cast<int16_t *>(b + o_order);
     d.gu = reinterpret_cast<double *>(b + o_gu);
     d.rk = reinterpret_cast<uint32_t *>(b + o_rk);
+    d.inv = reinterpret_cast<uint32_t *>(b + o_inv);
     d.rank = b + o_rank;
     d.table = b + o_table;
 

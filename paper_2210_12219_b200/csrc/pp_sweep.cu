@@ -130,7 +130,6 @@ template <typename T>
 __global__ void k_finalize(Dev d, pp_solution *out)
 {
     __shared__ unsigned int s_key[32];
-    __shared__ double s_beta;
     __shared__ unsigned int s_pick;
     const T *table = reinterpret_cast<const T *>(d.table);
     const T *rank = reinterpret_cast<const T *>(d.rank);
@@ -155,21 +154,14 @@ __global__ void k_finalize(Dev d, pp_solution *out)
     uint32_t S = (uint32_t)((key >> 5) & 0xFFFFF);
     int w = (int)(key & 31);
 
-    // beta* as a double: any list entry that carries the winning rank
-    if (tid == 0) s_beta = 0.0;
-    __syncthreads();
-    if (rstar != 0) {
-        int n = d.U * L;
-        for (int e = tid; e < n; e += blockDim.x)
-            if (d.rk[e] == rstar) s_beta = d.gu[e];  // equal ranks hold equal doubles
-    }
-    __syncthreads();
+    // beta* as a double: an entry that carries the winning rank (equal ranks hold equal doubles)
     if (tid == 0) {
-        out->beta_ms = s_beta;
+        out->beta_ms = rstar != 0 ? d.gu[d.inv[rstar]] : 0.0;
         out->status = PP_OK;
         out->m = m;
     }
 
+    __syncthreads();  // the -1 fill above is complete before plan entries are written
     int c2 = L - 1;
     for (int j = m - 1; j >= 0; --j) {
         if (tid == 0) {
@@ -181,9 +173,10 @@ __global__ void k_finalize(Dev d, pp_solution *out)
         const int lo = d.lo[w * L + c2];
         const int span = c2 - lo;  // candidates c = lo .. c2-1
         unsigned int bestk = 0xFFFFFFFFu;
-        for (int item = tid; item < span * k; item += blockDim.x) {
-            int c = lo + item / k, v = item - (item / k) * k;
-            if (!((P >> v) & 1u)) continue;
+        const int np = __popc(P);
+        for (int item = tid; item < span * np; item += blockDim.x) {
+            const int vi = item / span, c = lo + (item - vi * span);
+            const int v = __fns(P, 0, vi + 1);
             T a = table[((size_t)P * k + v) * Lpad + c];
             T b = rank[((size_t)w * k + v) * Lpad + c];
             T mx = a > b ? a : b;
@@ -222,9 +215,9 @@ __global__ void k_finalize(Dev d, pp_solution *out)
 cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s)
 {
     if (d.elem == 2)
-        k_finalize<uint16_t><<<1, 256, 0, s>>>(d, out);
+        k_finalize<uint16_t><<<1, 1024, 0, s>>>(d, out);
     else
-        k_finalize<uint32_t><<<1, 256, 0, s>>>(d, out);
+        k_finalize<uint32_t><<<1, 1024, 0, s>>>(d, out);
     return cudaGetLastError();
 }
 
