@@ -25,7 +25,13 @@ namespace pp {
 
 namespace {
 
-constexpr int kFastThreads = 512;
+#ifndef PP_FAST_THREADS
+#define PP_FAST_THREADS 512
+#endif
+#ifndef PP_FAST_NT
+#define PP_FAST_NT 1
+#endif
+constexpr int kFastThreads = PP_FAST_THREADS;
 constexpr uint32_t kInf2 = 0xFFFFFFFFu;
 
 // Per-target-node constants of the window step (W = 8q + r, e = r >> 1), built on the host.
@@ -59,6 +65,8 @@ __device__ __forceinline__ uint32_t vmax2(uint32_t a, uint32_t b)
     asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
     return r;
 }
+// three-input packed minimum: one issue slot where two two-input minima would take two
+__device__ __forceinline__ uint32_t vmin3(uint32_t a, uint32_t b, uint32_t c) { return __vimin3_u16x2(a, b, c); }
 // shuffle up by delta (<= 31) lanes, +inf shifted in from below lane 0
 __device__ __forceinline__ uint32_t shfl_up_inf(uint32_t x, int delta)
 {
@@ -74,7 +82,7 @@ __device__ __forceinline__ void min_shfl_up(uint32_t &acc, uint32_t x, int delta
                  : "+r"(acc) : "r"(x), "r"(delta));
 }
 
-constexpr int NT = 2;  // target nodes processed together
+constexpr int NT = PP_FAST_NT;  // target nodes processed together
 
 // Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].
 __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mptr,
@@ -157,7 +165,7 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
         for (int j = 0; j < 4; ++j) {
             const uint32_t e = __funnelshift_l(f[t][j], f[t][j + 1], sh);
             const uint32_t mid = __byte_perm(T2[t], T1[t], mp[t]->sel[j]);
-            o[t][j] = vmin2(vmin2(o[t][j], e), mid);
+            o[t][j] = vmin3(o[t][j], e, mid);
         }
     }
 }
@@ -200,92 +208,127 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
     const uint32_t full = (1u << k) - 1u;
     const int last_lane = (L - 1) >> 3, last_reg = ((L - 1) & 7) >> 1, last_sh = ((L - 1) & 1) * 16;
     const uint32_t stride = gridDim.x * (kFastThreads / 32);
+    const int npairs = (k - NV + NT - 1) / NT;  // target nodes per mask, NT at a time
 
     uint32_t mi = blockIdx.x * (kFastThreads / 32) + warp;
     uint32_t S = mi < nmask ? d.masks[first + mi] : 0u;
+    int voff[NV];
+    uint4 dp[NV];
+    unsigned long long best_seen = kNoBest;
+    // source rows of mask Sx -> registers (and the best final key seen so far: read once per mask,
+    // not once per row; a stale value only costs a redundant atomic)
+    auto load_rows = [&](uint32_t Sx) {
+        uint32_t rem = Sx;
+#pragma unroll
+        for (int vi = 0; vi < NV; ++vi) {
+            int v = __ffs(rem) - 1;
+            rem &= rem - 1;
+            voff[vi] = v * Lpad;
+        }
+        const uint16_t *src = table + (size_t)Sx * k * Lpad + 8 * lane;
+#pragma unroll
+        for (int vi = 0; vi < NV; ++vi)
+            dp[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(src + voff[vi]))
+                            : make_uint4(kInf2, kInf2, kInf2, kInf2);
+        best_seen = *reinterpret_cast<volatile unsigned long long *>(d.best);
+    };
+    if (mi < nmask) load_rows(S);
     while (mi < nmask) {
         const uint32_t mi_next = mi + stride;
         const uint32_t S_next = mi_next < nmask ? d.masks[first + mi_next] : 0u;
-        int voff[NV];
-        uint4 dp[NV];
-        {
-            uint32_t rem = S;
+        const uint32_t S_cur = S;
+        uint32_t wrem = full & ~S_cur;
+
+        // next two target nodes (an odd tail repeats its last node), branch-free
+        auto pick = [&](int (&w)[NT]) {
+            w[0] = __ffs(wrem) - 1;
+            wrem &= wrem - 1;
 #pragma unroll
-            for (int vi = 0; vi < NV; ++vi) {
-                int v = __ffs(rem) - 1;
-                rem &= rem - 1;
-                voff[vi] = v * Lpad;
+            for (int t = 1; t < NT; ++t) {
+                w[t] = wrem ? __ffs(wrem) - 1 : w[t - 1];
+                wrem &= wrem - 1;
             }
-            const uint16_t *src = table + (size_t)S * k * Lpad + 8 * lane;
-#pragma unroll
-            for (int vi = 0; vi < NV; ++vi)
-                dp[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(src + voff[vi]))
-                                : make_uint4(kInf2, kInf2, kInf2, kInf2);
-        }
-        // pull the next mask's source rows into L2 while this mask is being processed
-        if (mi_next < nmask && active && (lane & 7) == 0) {
-            uint32_t rem = S_next;
-            const uint16_t *src = table + (size_t)S_next * k * Lpad + 8 * lane;
-#pragma unroll
-            for (int vi = 0; vi < NV; ++vi) {
-                int v = __ffs(rem) - 1;
-                rem &= rem - 1;
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(src + v * Lpad));
-            }
-        }
-        // best final key seen so far: read once per mask, not once per row (a stale value only
-        // costs a redundant atomic)
-        unsigned long long best_seen = *reinterpret_cast<volatile unsigned long long *>(d.best);
-        uint32_t wrem = full & ~S;
-        while (wrem) {
-            int w[NT];
-            const WMeta *mp[NT];
+        };
+        // 1. relax over the source nodes, two of them per three-input minimum
+        auto relax = [&](const int (&w)[NT], uint32_t (&r)[NT][4]) {
             const uint16_t *rw[NT];
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
-                w[t] = __ffs(wrem) - 1;
-                if (wrem & (wrem - 1)) wrem &= wrem - 1;  // an odd tail repeats its last node
-                else if (t == NT - 1) wrem = 0;
-                mp[t] = wm + w[t];
                 rw[t] = rank_s + w[t] * k * Lpad + 8 * lane;
+                r[t][0] = r[t][1] = r[t][2] = r[t][3] = kInf2;
             }
-            // ---- 1. relax over the source nodes ----
-            uint32_t r[NT][4], o[NT][4];
 #pragma unroll
-            for (int t = 0; t < NT; ++t) r[t][0] = r[t][1] = r[t][2] = r[t][3] = kInf2;
-#pragma unroll
-            for (int vi = 0; vi < NV; ++vi) {
+            for (int vi = 0; vi + 1 < NV; vi += 2) {
 #pragma unroll
                 for (int t = 0; t < NT; ++t) {
                     const uint4 g = *reinterpret_cast<const uint4 *>(rw[t] + voff[vi]);
-                    r[t][0] = vmin2(r[t][0], vmax2(dp[vi].x, g.x));
-                    r[t][1] = vmin2(r[t][1], vmax2(dp[vi].y, g.y));
-                    r[t][2] = vmin2(r[t][2], vmax2(dp[vi].z, g.z));
-                    r[t][3] = vmin2(r[t][3], vmax2(dp[vi].w, g.w));
+                    const uint4 h = *reinterpret_cast<const uint4 *>(rw[t] + voff[vi + 1]);
+                    r[t][0] = vmin3(r[t][0], vmax2(dp[vi].x, g.x), vmax2(dp[vi + 1].x, h.x));
+                    r[t][1] = vmin3(r[t][1], vmax2(dp[vi].y, g.y), vmax2(dp[vi + 1].y, h.y));
+                    r[t][2] = vmin3(r[t][2], vmax2(dp[vi].z, g.z), vmax2(dp[vi + 1].z, h.z));
+                    r[t][3] = vmin3(r[t][3], vmax2(dp[vi].w, g.w), vmax2(dp[vi + 1].w, h.w));
                 }
             }
-            // ---- 2. window minimum ----
+            if (NV & 1) {
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                    const uint4 g = *reinterpret_cast<const uint4 *>(rw[t] + voff[NV - 1]);
+                    r[t][0] = vmin2(r[t][0], vmax2(dp[NV - 1].x, g.x));
+                    r[t][1] = vmin2(r[t][1], vmax2(dp[NV - 1].y, g.y));
+                    r[t][2] = vmin2(r[t][2], vmax2(dp[NV - 1].z, g.z));
+                    r[t][3] = vmin2(r[t][3], vmax2(dp[NV - 1].w, g.w));
+                }
+            }
+        };
+        // 2. + 3. window minimum, write the rows, offer their last elements as final states
+        auto finish = [&](const int (&w)[NT], const uint32_t (&r)[NT][4]) {
+            const WMeta *mp[NT];
+#pragma unroll
+            for (int t = 0; t < NT; ++t) mp[t] = wm + w[t];
+            uint32_t o[NT][4];
             window_min(r, mp, o);
-            // ---- 3. write the rows, offer their last elements as final states ----
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
-                const uint32_t S2 = S | (1u << w[t]);
+                const uint32_t S2 = S_cur | (1u << w[t]);
                 if (active)
                     *reinterpret_cast<uint4 *>(table_w + ((size_t)S2 * k + w[t]) * Lpad + 8 * lane) =
                         make_uint4(o[t][0], o[t][1], o[t][2], o[t][3]);
-                if (lane == last_lane) {
-                    const uint32_t reg = last_reg == 0 ? o[t][0] : (last_reg == 1 ? o[t][1] : (last_reg == 2 ? o[t][2] : o[t][3]));
-                    const uint32_t val = (reg >> last_sh) & 0xFFFFu;
-                    if (val != 0xFFFFu) {
-                        const unsigned long long key = pack_best(val, level, S2, w[t]);
-                        if (key < best_seen) {
-                            atomicMin(d.best, key);
-                            best_seen = key;
-                        }
+                const uint32_t reg = last_reg == 0 ? o[t][0] : (last_reg == 1 ? o[t][1] : (last_reg == 2 ? o[t][2] : o[t][3]));
+                const uint32_t val = (reg >> last_sh) & 0xFFFFu;
+                if (lane == last_lane && val != 0xFFFFu) {
+                    const unsigned long long key = pack_best(val, level, S2, w[t]);
+                    if (key < best_seen) {
+                        atomicMin(d.best, key);
+                        best_seen = key;
                     }
                 }
             }
+        };
+        // software pipeline over the pairs of target nodes: the relaxation of the next pair
+        // (independent loads and min/max) sits in the same straight-line block as the window
+        // step of the current pair (dependent shuffle chains), so the scheduler can fill the
+        // latencies of one with the other
+        int w[NT];
+        uint32_t r[NT][4];
+        pick(w);
+        relax(w, r);
+        for (int it = 1; it < npairs; ++it) {
+            int wn[NT];
+            uint32_t rn[NT][4];
+            pick(wn);
+            relax(wn, rn);
+            finish(w, r);
+#pragma unroll
+            for (int t = 0; t < NT; ++t) {
+                w[t] = wn[t];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) r[t][j] = rn[t][j];
+            }
         }
+        // the source rows are dead once the last pair is relaxed: fetch the next mask's rows now,
+        // so that their latency hides behind the last window step
+        if (mi_next < nmask) load_rows(S_next);
+        finish(w, r);
         mi = mi_next;
         S = S_next;
     }
