@@ -172,7 +172,7 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
 
 template <int NV>
 __global__ void __launch_bounds__(kFastThreads, 1)
-k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
+k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
 {
     // Programmatic dependent launch: let the next level's blocks be scheduled as soon as this
     // level's blocks retire, so that their prologue (rank table -> shared memory) overlaps our
@@ -204,14 +204,16 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
     const uint16_t *table = reinterpret_cast<const uint16_t *>(d.table);
     uint16_t *table_w = reinterpret_cast<uint16_t *>(d.table);
     const uint32_t first = d.level_off[level - 1];
-    const uint32_t nmask = d.level_off[level] - first;
+    // Work items: (mask, part).  Levels with few masks split each mask's target nodes over
+    // `split` warps (part p takes the targets whose ordinal is p mod split), so that small
+    // levels are not serialised on a handful of warps.
+    const uint32_t nmask = (d.level_off[level] - first) * (uint32_t)split;
     const uint32_t full = (1u << k) - 1u;
     const int last_lane = (L - 1) >> 3, last_reg = ((L - 1) & 7) >> 1, last_sh = ((L - 1) & 1) * 16;
     const uint32_t stride = gridDim.x * (kFastThreads / 32);
-    const int npairs = (k - NV + NT - 1) / NT;  // target nodes per mask, NT at a time
 
     uint32_t mi = blockIdx.x * (kFastThreads / 32) + warp;
-    uint32_t S = mi < nmask ? d.masks[first + mi] : 0u;
+    uint32_t S = mi < nmask ? d.masks[first + mi / split] : 0u;
     int voff[NV];
     uint4 dp[NV];
     unsigned long long best_seen = kNoBest;
@@ -235,9 +237,18 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g)
     if (mi < nmask) load_rows(S);
     while (mi < nmask) {
         const uint32_t mi_next = mi + stride;
-        const uint32_t S_next = mi_next < nmask ? d.masks[first + mi_next] : 0u;
+        const uint32_t S_next = mi_next < nmask ? d.masks[first + mi_next / split] : 0u;
         const uint32_t S_cur = S;
         uint32_t wrem = full & ~S_cur;
+        if (split > 1) {  // keep this part's share of the target nodes
+            const int part = (int)(mi % (uint32_t)split);
+            uint32_t keep = 0;
+            int idx = 0;
+            for (uint32_t rem = wrem; rem; rem &= rem - 1, ++idx)
+                if (idx % split == part) keep |= rem & (0u - rem);
+            wrem = keep;
+        }
+        const int npairs = (__popc(wrem) + NT - 1) / NT;  // target nodes of this item, NT at a time
 
         // next two target nodes (an odd tail repeats its last node), branch-free
         auto pick = [&](int (&w)[NT]) {
@@ -340,7 +351,7 @@ size_t fast_smem_bytes(const Dev &d)
 }
 
 template <int NV>
-cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned grid, size_t sm, cudaStream_t s)
+cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned grid, int split, size_t sm, cudaStream_t s)
 {
     cudaError_t e = cudaFuncSetAttribute(k_sweep_fast<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
@@ -354,7 +365,7 @@ cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned gr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_sweep_fast<NV>, d, level, meta);
+    return cudaLaunchKernelEx(&cfg, k_sweep_fast<NV>, d, level, meta, split);
 }
 
 }  // namespace
@@ -413,12 +424,18 @@ cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s)
     unsigned long long n = 1;  // source masks of popcount level-1
     for (int i = 0; i < level - 1; ++i) n = n * (unsigned)(d.k - i) / (unsigned)(i + 1);
     const unsigned wpb = kFastThreads / 32;
-    unsigned grid = (unsigned)((n + wpb - 1) / wpb);
+    const int nw = d.k - (level - 1);  // target nodes per mask
+    int split = 1;
+    if (n < (unsigned long long)sms * wpb) {
+        split = (int)(((unsigned long long)sms * wpb + n - 1) / n);
+        if (split > nw) split = nw;
+    }
+    unsigned grid = (unsigned)((n * split + wpb - 1) / wpb);
     if (grid > (unsigned)sms) grid = (unsigned)sms;
     const size_t sm = fast_smem_bytes(d);
     const FastMeta *meta = static_cast<const FastMeta *>(d.fast_meta);
     switch (level - 1) {
-#define PP_CASE(N) case N: return launch_nv<N>(d, level, meta, grid, sm, s);
+#define PP_CASE(N) case N: return launch_nv<N>(d, level, meta, grid, split, sm, s);
         PP_CASE(1) PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6) PP_CASE(7) PP_CASE(8)
         PP_CASE(9) PP_CASE(10) PP_CASE(11) PP_CASE(12) PP_CASE(13) PP_CASE(14) PP_CASE(15)
         PP_CASE(16) PP_CASE(17) PP_CASE(18) PP_CASE(19)
