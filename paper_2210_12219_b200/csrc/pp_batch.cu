@@ -112,7 +112,6 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     const int Ls = (L + 1) & ~1, Lh = Ls >> 1;  // row stride (even) and words per row
     // a thread's items advance by the block size: (row, column) moves by (dr, dc) with one carry
     const int drA = kBatchThreads / Lh, dcA = kBatchThreads - drA * Lh;
-    const int drB = kBatchThreads / L, dcB = kBatchThreads - drB * L;
     const double kInf = __longlong_as_double(0x7FF0000000000000ll);
 
     // ---- instance-independent tables -------------------------------------------------------
@@ -285,22 +284,26 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                 }
             }
             __syncthreads();
-            {  // phase B: thread <-> (row, position)
-                int rr = tid / L, c2 = tid - rr * L;
+            {  // phase B: thread <-> (row, word): the windows of two neighbouring positions
+               // [l0, c2-1] and [l1, c2] share the run [l1, c2-1], scanned once
+                int rr = tid / Lh, cw = tid - rr * Lh;
                 while (rr < (int)nrows) {
                     const int w = (rowinfo[row0 + rr] >> 12) & 15;
                     const uint16_t *gr = gbuf + rr * Ls;
-                    uint32_t best = kInf16;
-                    int c = lo[w * L + c2];
-                    for (; c + 4 <= c2; c += 4) {  // four independent loads per trip
-                        const uint32_t x0 = gr[c], x1 = gr[c + 1], x2 = gr[c + 2], x3 = gr[c + 3];
-                        best = min(min(best, min(x0, x1)), min(x2, x3));
-                    }
-                    for (; c < c2; ++c) best = min(best, (uint32_t)gr[c]);
-                    dp[(size_t)(row0 + rr) * Ls + c2] = (uint16_t)best;
-                    rr += drB;
-                    c2 += dcB;
-                    if (c2 >= L) { c2 -= L; ++rr; }
+                    const int c2 = 2 * cw;
+                    const int l0 = lo[w * L + c2];
+                    const bool has1 = c2 + 1 < L;
+                    const int l1 = has1 ? lo[w * L + c2 + 1] : c2 + 1;
+                    uint32_t head = kInf16, common = kInf16;
+                    const int split = l1 < c2 ? l1 : c2;
+                    for (int c = l0; c < split; ++c) head = min(head, (uint32_t)gr[c]);
+                    for (int c = l1; c < c2; ++c) common = min(common, (uint32_t)gr[c]);
+                    const uint32_t out0 = min(head, common);
+                    const uint32_t out1 = (has1 && l1 <= c2) ? min(common, (uint32_t)gr[c2]) : (uint32_t)kInf16;
+                    reinterpret_cast<uint32_t *>(dp + (size_t)(row0 + rr) * Ls)[cw] = out0 | (out1 << 16);
+                    rr += drA;
+                    cw += dcA;
+                    if (cw >= Lh) { cw -= Lh; ++rr; }
                 }
             }
             __syncthreads();
