@@ -117,6 +117,20 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
+def aggregate_over_ranks(units_this_rank: float, seconds_this_rank: float, dist=None, device=None):
+    """Whole-job throughput of independent replicas: units summed over ranks divided by the
+    slowest rank's time.  Works with any initialised torch.distributed backend (NCCL on GPUs,
+    gloo on CPU); without one it is the single-rank ratio."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return units_this_rank / seconds_this_rank, seconds_this_rank
+    import torch
+    t = torch.tensor([seconds_this_rank], dtype=torch.float64, device=device)
+    u = torch.tensor([units_this_rank], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(u.item()) / float(t.item()), float(t.item())
+
+
 def stack(insts):
     return (np.stack([i.layer_out_bits for i in insts]), np.stack([i.layer_mem_bytes for i in insts]),
             np.stack([i.node_mem_bytes for i in insts]), np.stack([i.bw_kbps for i in insts]))
@@ -209,7 +223,8 @@ def run_ours(args):
                 step_device()
             ev1.record(stream)
             barrier()
-        ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+        ms_local = ev0.elapsed_time(ev1)
+        ms_total = max_over_ranks(ms_local)
         clk = clocks.summary()
         prof = prob.last_solve_profile()
         launches_per_step = prof.total_launches + 2
@@ -237,7 +252,7 @@ def run_ours(args):
 
     sol_rec = pp.pp_solution.from_buffer_copy(d_sol.cpu().numpy().tobytes())
     ms_per_step = ms_total / args.steps
-    value = world * relax_step / (ms_per_step * 1e-3)
+    value, _ = aggregate_over_ranks(relax_step * args.steps, ms_local * 1e-3, dist, dev)
 
     # ---- end to end through the host-pointer entry points ----
     h2d = (large.layer_out_bits.nbytes + large.layer_mem_bytes.nbytes + large.node_mem_bytes.nbytes
@@ -262,8 +277,8 @@ def run_ours(args):
     for _ in range(e2e_steps):
         host_out = step_host()
     barrier()
-    e2e_s = max_over_ranks((time.perf_counter() - t0) / e2e_steps)
-    e2e_value = world * relax_step / e2e_s
+    e2e_local = (time.perf_counter() - t0) / e2e_steps
+    e2e_value, e2e_s = aggregate_over_ranks(relax_step, e2e_local, dist, dev)
     assert host_out[0].beta_ms == sol_rec.beta_ms and host_out[0].m == sol_rec.m
 
     # ---- roofline of the dominant kernel (the popcount sweep of the Large instance) ----

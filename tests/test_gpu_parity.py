@@ -174,6 +174,9 @@ def test_large_config_full_size():
     # those nodes, which the oracle can afford for up to 8 nodes.
     inst = W.config_large()
     want = oracle.dp_fact(inst, oracle.max_threads())
+    from tests.test_workloads_golden import read_golden
+    checksum, g_beta, g_m, g_cuts, g_nodes = read_golden()["large"]
+    assert inst.checksum() == checksum and want.beta_ms == g_beta and want.plan() == (g_m, g_cuts, g_nodes)
     with pp.Problem.from_instance(inst) as p:
         got = p.solve_exact()
         assert_same(inst, got, want)
