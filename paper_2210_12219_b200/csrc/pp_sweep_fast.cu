@@ -170,6 +170,19 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
     }
 }
 
+// Slow path of the final-state bookkeeping, kept out of line so that the common case is a
+// compare and a branch.
+__device__ __noinline__ unsigned long long offer_final(unsigned long long *best, unsigned long long best_seen,
+                                                       uint32_t val, int level, uint32_t S2, int w)
+{
+    const unsigned long long key = pack_best(val, level, S2, w);
+    if (key < best_seen) {
+        atomicMin(best, key);
+        return key;
+    }
+    return best_seen;
+}
+
 template <int NV>
 __global__ void __launch_bounds__(kFastThreads, 1)
 k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
@@ -240,6 +253,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
         const uint32_t S_next = mi_next < nmask ? d.masks[first + mi_next / split] : 0u;
         const uint32_t S_cur = S;
         uint32_t wrem = full & ~S_cur;
+        uint16_t *const row_base = table_w + (size_t)S_cur * k * Lpad + 8 * lane;
         if (split > 1) {  // keep this part's share of the target nodes
             const int part = (int)(mi % (uint32_t)split);
             uint32_t keep = 0;
@@ -301,18 +315,14 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
                 const uint32_t S2 = S_cur | (1u << w[t]);
-                if (active)
-                    *reinterpret_cast<uint4 *>(table_w + ((size_t)S2 * k + w[t]) * Lpad + 8 * lane) =
+                if (active)  // row (S2, w) lies ((k << w) + w) rows after row (S_cur, 0)
+                    *reinterpret_cast<uint4 *>(row_base + (uint32_t)(((k << w[t]) + w[t]) * Lpad)) =
                         make_uint4(o[t][0], o[t][1], o[t][2], o[t][3]);
                 const uint32_t reg = last_reg == 0 ? o[t][0] : (last_reg == 1 ? o[t][1] : (last_reg == 2 ? o[t][2] : o[t][3]));
                 const uint32_t val = (reg >> last_sh) & 0xFFFFu;
-                if (lane == last_lane && val != 0xFFFFu) {
-                    const unsigned long long key = pack_best(val, level, S2, w[t]);
-                    if (key < best_seen) {
-                        atomicMin(d.best, key);
-                        best_seen = key;
-                    }
-                }
+                // ranks at or below the best rank seen so far are rare: everything else ends here
+                if (lane == last_lane && val <= (uint32_t)(best_seen >> 30) && val != 0xFFFFu)
+                    best_seen = offer_final(d.best, best_seen, val, level, S2, w[t]);
             }
         };
         // software pipeline over the pairs of target nodes: the relaxation of the next pair
