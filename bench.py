@@ -36,6 +36,13 @@ from paper_2210_12219_b200 import workloads as W  # noqa: E402
 
 METRIC = "exact-plan DP relaxations/s"
 UNIT = "relaxations/s"
+# DRAM bytes per sweep launch (18 launches per Large solve, base frontier included) from the ncu
+# capture summarised in profiles/sweep_dram_traffic_large.md; set to None whenever the sweep
+# kernels change after that capture.
+SWEEP_DRAM_BYTES_PER_LAUNCH = 94.87e6
+# Issue rate of packed 16-bit min/max measured on this part: 64 lanes per clock per SM, two
+# elements per lane (a three-input min/max issues at the same rate).
+PACKED_MINMAX_LANES_PER_CLK_SM = 64
 N_PLANS = 262144
 N_BATCH = 4096
 BATCH_L, BATCH_K = 24, 8
@@ -261,12 +268,19 @@ def run_ours(args):
     d2h = (ctypes.sizeof(pp.pp_solution) + N_PLANS * 9
            + N_BATCH * (8 + 4 + 4 * (BATCH_K - 1) + 4 * BATCH_K + 1))
 
+    # the step's inputs live in pinned host memory; the C entry points copy them to the device
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
+    h_bits, h_mem, h_cap, h_bw = (pin(a) for a in (large.layer_out_bits, large.layer_mem_bytes,
+                                                    large.node_mem_bytes, large.bw_kbps))
+    h_nseg, h_ends, h_nodes = pin(nseg), pin(ends), pin(nodes)
+    hb_bits, hb_mem, hb_cap, hb_bw = pin(b_bits), pin(b_mem), pin(b_cap), pin(b_bw)
+
     def step_host():
-        with pp.Problem.from_instance(large) as p2:
+        with pp.Problem(L, h_bits, h_mem, k, h_cap, h_bw) as p2:
             p2.set_workspace(ws)
             s = p2.solve_exact()
-            bsol = pp.solve_exact_batch(BATCH_L, BATCH_K, b_bits, b_mem, b_cap, b_bw)
-            beta, pstat = p2.eval_plans(nseg, ends, nodes)
+            bsol = pp.solve_exact_batch(BATCH_L, BATCH_K, hb_bits, hb_mem, hb_cap, hb_bw)
+            beta, pstat = p2.eval_plans(h_nseg, h_ends, h_nodes)
         return s, bsol, beta, pstat
 
     for _ in range(2):
@@ -287,10 +301,21 @@ def run_ours(args):
     sweep_t = statistics.median(sweep_ms) * 1e-3
     alg_bytes = 2 * n_states(k, L) * elem  # every state written once and read once
     achieved = alg_bytes / sweep_t / 1e9
+    n_launch = prof.sweep_launches
+    # the same sweep against the plain-ALU bound: 2 element-ops per relaxation + 3 per state, at
+    # the measured packed min/max rate and the maximum SM clock
+    alu_ops = 2 * relax_large + 3 * n_states(k, L)
+    alu_peak = PACKED_MINMAX_LANES_PER_CLK_SM * 2 * 148 * peaks.get("sm_max_mhz", 1965.0) * 1e6
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": which,
-                "kernel": "sweep (%d launches per solve, base frontier included)" % prof.sweep_launches,
-                "algorithmic_bytes_per_solve": alg_bytes, "sweep_ms": sweep_t * 1e3}
+                "frac": achieved / peaks["hbm_gbs"],
+                "traffic": SWEEP_DRAM_BYTES_PER_LAUNCH if prof.fast_path else None,
+                "peak_source": which + " (burst copy figure; the sweep is timed alone)",
+                "kernel": "k_sweep_fast + k_base (%d launches per solve)" % n_launch,
+                "algorithmic_bytes_per_launch": alg_bytes / n_launch,
+                "ms_per_launch": sweep_t * 1e3 / n_launch,
+                "algorithmic_bytes_per_solve": alg_bytes, "sweep_ms": sweep_t * 1e3,
+                "alu": {"ops_per_solve": alu_ops, "achieved_ops_per_s": alu_ops / sweep_t,
+                        "peak_ops_per_s": alu_peak, "frac": alu_ops / sweep_t / alu_peak}}
 
     med = statistics.median
     out = {

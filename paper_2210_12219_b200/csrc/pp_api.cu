@@ -249,11 +249,18 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         {fmeta.data(), fmeta.size(), 0}};
     size_t total = 0;
     for (auto &q : parts) { q.off = total; total = align_up(total + q.bytes, 256); }
-    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&p->d_inputs), total);
-    if (e == cudaSuccess) e = cudaMemset(p->d_inputs, 0, total);
+    // one staging buffer, one copy: the parts are small and a copy per part costs more than the bytes
+    std::vector<unsigned char> staging;
+    try {
+        staging.assign(total, 0);
+    } catch (const std::bad_alloc &) {
+        delete p;
+        return PP_ERR_NOMEM;
+    }
     for (auto &q : parts)
-        if (e == cudaSuccess && q.src && q.bytes)
-            e = cudaMemcpy(p->d_inputs + q.off, q.src, q.bytes, cudaMemcpyHostToDevice);
+        if (q.src && q.bytes) std::memcpy(staging.data() + q.off, q.src, q.bytes);
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&p->d_inputs), total);
+    if (e == cudaSuccess) e = cudaMemcpy(p->d_inputs, staging.data(), total, cudaMemcpyHostToDevice);
     for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreate(&p->ev[i]);
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->h_sol), sizeof(pp_solution));
     if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->h_err), sizeof(int32_t));
