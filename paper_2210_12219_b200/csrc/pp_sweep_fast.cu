@@ -229,9 +229,11 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
     uint32_t S = mi < nmask ? d.masks[first + mi / split] : 0u;
     int voff[NV];
     uint4 dp[NV];
-    unsigned long long best_seen = kNoBest;
-    // source rows of mask Sx -> registers (and the best final key seen so far: read once per mask,
-    // not once per row; a stale value only costs a redundant atomic)
+    // best final key seen so far: read once per mask, not once per row (a stale value only costs a
+    // redundant atomic); the read for the next mask is issued early and consumed after the last
+    // row of the current one
+    unsigned long long best_seen = kNoBest, best_next = kNoBest;
+    // source rows of mask Sx -> registers
     auto load_rows = [&](uint32_t Sx) {
         uint32_t rem = Sx;
 #pragma unroll
@@ -245,9 +247,10 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
         for (int vi = 0; vi < NV; ++vi)
             dp[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(src + voff[vi]))
                             : make_uint4(kInf2, kInf2, kInf2, kInf2);
-        best_seen = *reinterpret_cast<volatile unsigned long long *>(d.best);
+        best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
     };
     if (mi < nmask) load_rows(S);
+    best_seen = best_next;
     while (mi < nmask) {
         const uint32_t mi_next = mi + stride;
         const uint32_t S_next = mi_next < nmask ? d.masks[first + mi_next / split] : 0u;
@@ -350,6 +353,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
         // so that their latency hides behind the last window step
         if (mi_next < nmask) load_rows(S_next);
         finish(w, r);
+        best_seen = best_next < best_seen ? best_next : best_seen;
         mi = mi_next;
         S = S_next;
     }
