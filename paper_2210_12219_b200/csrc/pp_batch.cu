@@ -6,8 +6,8 @@
 // Per instance the block
 //   1. stages the inputs, builds the memory prefix sums and the window table lo[w][c'];
 //   2. rank-compresses gamma (Eq. 3): layers sorted by bits, distinct bandwidths listed, one fp64
-//      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, counted by
-//      binary search in each of the sorted lists (IEEE division is monotone in the numerator);
+//      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, obtained by
+//      a bitonic sort of all quotients in shared memory;
 //   3. sweeps the popcount levels with a flat thread <-> (target row, position) mapping:
 //      phase A forms g[c] = min_v max(dp[S'\{w}][v][c], rank[v][w][c]) for every row of the level,
 //      two neighbouring positions per thread as one packed u16x2 word,
@@ -23,7 +23,7 @@ constexpr int kBatchWarps = kBatchThreads / 32;
 constexpr uint16_t kInf16 = 0xFFFFu;
 
 struct BatchLayout {
-    size_t dp, g, rank, gu, rk, cnt, M, cap, bits, sbits, bw, ubw, pair_u, pos, lo, rowoff, loff, rowinfo, total;
+    size_t dp, g, rank, gu, rk, cnt, skey, sval, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, total;
 };
 
 __host__ __device__ inline BatchLayout batch_layout(int L, int k)
@@ -42,12 +42,17 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     size_t o = 0;
     auto take = [&o](size_t bytes) { size_t at = o; o = (o + bytes + 15) & ~(size_t)15; return at; };
     b.gu = take(U * L * sizeof(double));
+    size_t npad = 1;
+    while (npad < U * L) npad <<= 1;
+    b.skey = take(npad * sizeof(unsigned long long));
+    b.sval = take(npad * sizeof(uint16_t));
     b.M = take((size_t)(L + 1) * sizeof(uint64_t));
     b.cap = take((size_t)k * sizeof(uint64_t));
     b.bits = take((size_t)L * sizeof(uint64_t));
     b.sbits = take((size_t)L * sizeof(uint64_t));
     b.bw = take((size_t)k * k * sizeof(uint32_t));
     b.ubw = take(U * sizeof(uint32_t));
+    b.uord = take(U * sizeof(int16_t));
     b.rowoff = take(((size_t)1 << k) * sizeof(uint32_t));
     b.loff = take((size_t)(k + 2) * sizeof(uint32_t));
     b.rowinfo = take(rows * sizeof(uint32_t));
@@ -92,6 +97,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     uint64_t *s_sorted = reinterpret_cast<uint64_t *>(smem + lay.sbits);
     uint32_t *s_bw = reinterpret_cast<uint32_t *>(smem + lay.bw);
     uint32_t *ubw = reinterpret_cast<uint32_t *>(smem + lay.ubw);
+    int16_t *uord = reinterpret_cast<int16_t *>(smem + lay.uord);  // lists by ascending bandwidth
     uint32_t *rowoff = reinterpret_cast<uint32_t *>(smem + lay.rowoff);
     uint32_t *loff = reinterpret_cast<uint32_t *>(smem + lay.loff);    // first compact row of each level
     uint32_t *rowinfo = reinterpret_cast<uint32_t *>(smem + lay.rowinfo);
@@ -100,6 +106,8 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     uint16_t *rank = reinterpret_cast<uint16_t *>(smem + lay.rank);    // [v][w][c]
     uint16_t *rk = reinterpret_cast<uint16_t *>(smem + lay.rk);        // [U][L]
     uint32_t *cnt = reinterpret_cast<uint32_t *>(smem + lay.cnt);      // [U][L]
+    unsigned long long *skey = reinterpret_cast<unsigned long long *>(smem + lay.skey);  // sort keys
+    uint16_t *sval = reinterpret_cast<uint16_t *>(smem + lay.sval);    // sort payload: entry index
     int16_t *pair_u = reinterpret_cast<int16_t *>(smem + lay.pair_u);
     int16_t *pos = reinterpret_cast<int16_t *>(smem + lay.pos);
     int16_t *lo = reinterpret_cast<int16_t *>(smem + lay.lo);
@@ -207,6 +215,11 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         __syncthreads();
         for (int p = tid; p < k * k; p += kBatchThreads) pair_u[p] = reinterpret_cast<int16_t *>(cnt)[p];
         const int U = s_U;
+        for (int u = tid; u < U; u += kBatchThreads) {  // distinct values: positions are unique
+            int at = 0;
+            for (int u2 = 0; u2 < U; ++u2) at += (ubw[u2] < ubw[u]);
+            uord[at] = (int16_t)u;
+        }
         for (int e = tid; e < k * L; e += kBatchThreads) {
             const int w = e / L, c2 = e - w * L;
             int c = c2;  // step down while the segment starting at layer c (previous cut c-1) fits
@@ -217,33 +230,44 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         for (int e = tid; e < U * L; e += kBatchThreads) {
             const int u = e / L, i = e - u * L;
             gu[e] = __ddiv_rn((double)s_sorted[i], (double)ubw[u]);
-            cnt[e] = 0;
         }
         __syncthreads();
-        // one task per (quotient, group of 4 lists): binary search in each list of the group
+        // Rank = 1 + number of quotients strictly below: bitonic sort of the bit patterns (positive
+        // doubles order like unsigned integers) with the entry index as payload, then every run of
+        // equal keys takes the position of its first element.
         {
-            const int ngrp = (U + 3) >> 2;
-            for (int t = tid; t < U * L * ngrp; t += kBatchThreads) {
-                // consecutive threads search the same lists with consecutive queries, so that a
-                // warp's probes fall into one 8L-byte list instead of one bank
-                const int grp = t / (U * L), e = t - grp * (U * L);
-                const double x = gu[e];
-                unsigned below = 0;
-                const int u_end = (grp * 4 + 4 < U) ? grp * 4 + 4 : U;
-                for (int u2 = grp * 4; u2 < u_end; ++u2) {
-                    const double *list = gu + u2 * L;
-                    int a = 0, b = L;  // first index with list[idx] >= x
-                    while (a < b) {
-                        const int mid = (a + b) >> 1;
-                        if (list[mid] < x) a = mid + 1; else b = mid;
+            const int n = U * L;
+            int npad = 1;
+            while (npad < n) npad <<= 1;
+            for (int i = tid; i < npad; i += kBatchThreads) {
+                skey[i] = i < n ? (unsigned long long)__double_as_longlong(gu[i]) : ~0ull;
+                sval[i] = (uint16_t)i;
+            }
+            __syncthreads();
+            for (int size = 2; size <= npad; size <<= 1)
+                for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                    for (int t = tid; t < (npad >> 1); t += kBatchThreads) {
+                        const int lo_i = 2 * t - (t & (stride - 1));  // index with the stride bit clear
+                        const int hi_i = lo_i + stride;
+                        const bool up = (lo_i & size) == 0;
+                        const unsigned long long a = skey[lo_i], b = skey[hi_i];
+                        if ((a > b) == up) {
+                            skey[lo_i] = b;
+                            skey[hi_i] = a;
+                            const uint16_t va = sval[lo_i];
+                            sval[lo_i] = sval[hi_i];
+                            sval[hi_i] = va;
+                        }
                     }
-                    below += (unsigned)a;
+                    __syncthreads();
                 }
-                if (below) atomicAdd(&cnt[e], below);
+            for (int i = tid; i < n; i += kBatchThreads) {
+                int first = i;  // runs of equal quotients are short except in degenerate inputs
+                const unsigned long long key = skey[i];
+                while (first > 0 && skey[first - 1] == key) --first;
+                rk[sval[i]] = (uint16_t)(1 + first);
             }
         }
-        __syncthreads();
-        for (int e = tid; e < U * L; e += kBatchThreads) rk[e] = (uint16_t)(1u + cnt[e]);
         __syncthreads();
         for (int e = tid; e < k * k * Ls; e += kBatchThreads) {
             const int r = e / Ls, c = e - r * Ls;
