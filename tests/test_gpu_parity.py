@@ -195,6 +195,28 @@ def test_large_config_full_size():
         assert_same(inst, p.solve_exact(), want)
 
 
+def test_maximum_sizes():
+    # k at the library limit (20 nodes, every sweep instantiation up to 19 source nodes) on a
+    # short uniform-memory chain, and L at the limit (1024 layers) on few nodes
+    inst = W.uniform_memory_small(90000, 16, pp.PP_MAX_K, 8, 12)
+    want = oracle.dp_fact(inst, oracle.max_threads())
+    with pp.Problem.from_instance(inst) as p:
+        got = p.solve_exact()
+        assert p.last_solve_profile().fast_path == 1
+        assert_same(inst, got, want)
+        p.force_generic(1)
+        assert_same(inst, p.solve_exact(), want)
+    base = W.random_small(90001, pp.PP_MAX_L, 3)
+    cap = np.full(3, int(base.layer_mem_bytes.sum()) // 2, dtype=np.uint64)
+    inst = make_instance(base.layer_out_bits, base.layer_mem_bytes, cap, base.bw_kbps)
+    assert_same(inst, gpu_solve(inst), oracle.dp_fact(inst, oracle.max_threads()))
+    # one over either limit is refused
+    with pytest.raises(pp.PPError) as ei:
+        pp.Problem(pp.PP_MAX_L + 1, np.ones(pp.PP_MAX_L + 1, np.uint64), np.ones(pp.PP_MAX_L + 1, np.uint64),
+                   2, np.ones(2, np.uint64), np.ones(4, np.uint32))
+    assert ei.value.status == pp.PP_ERR_LIMIT
+
+
 def test_32bit_rank_path():
     # enough distinct gamma values that 16-bit ranks do not fit: L * U + 1 > 65534
     L, k = 700, 11
