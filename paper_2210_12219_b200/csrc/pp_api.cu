@@ -6,6 +6,7 @@
 #include <cstring>
 #include <limits>
 #include <map>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -24,9 +25,11 @@ struct pp_problem {
     bool own_work = false;
     cudaStream_t stream = nullptr;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
-    pp_solution *h_sol = nullptr;  // pinned
+    pp_solution h_sol_buf{};       // host copy of the result record
+    int32_t h_err_buf = 0;
+    pp_solution *h_sol = &h_sol_buf;
     pp_solution *d_sol = nullptr;
-    int32_t *h_err = nullptr;      // pinned
+    int32_t *h_err = &h_err_buf;
     Dev d{};
     bool solved = false;
     int sweep_launches = 0, total_launches = 0, fast_used = 0;
@@ -34,6 +37,56 @@ struct pp_problem {
 };
 
 namespace {
+
+// Masks sorted by (popcount, value) depend on k only: built once per k and process, then copied.
+struct MaskList {
+    std::vector<uint32_t> masks, level_off;
+};
+const MaskList &mask_list(int k)
+{
+    static std::mutex mu;
+    static std::map<int, MaskList> cache;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find(k);
+    if (it != cache.end()) return it->second;
+    MaskList ml;
+    const uint32_t nm = 1u << k;
+    ml.level_off.assign(k + 2, 0);
+    for (uint32_t S = 1; S < nm; ++S) ml.level_off[__builtin_popcount(S) + 1]++;
+    for (int j = 1; j <= k + 1; ++j) ml.level_off[j] += ml.level_off[j - 1];
+    ml.masks.assign(nm - 1, 0);
+    std::vector<uint32_t> at(ml.level_off.begin(), ml.level_off.end());
+    for (uint32_t S = 1; S < nm; ++S) ml.masks[at[__builtin_popcount(S)]++] = S;
+    return cache.emplace(k, std::move(ml)).first->second;
+}
+
+// Staging buffers of the host-pointer entry points come from a pool of the library's own that
+// keeps its memory between calls (the default pool would hand it back at every synchronisation).
+cudaError_t staging_alloc(void **ptr, size_t bytes, cudaStream_t s)
+{
+    static std::mutex mu;
+    static cudaMemPool_t pools[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaMalloc(ptr, bytes);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!pools[dev]) {
+            cudaMemPoolProps props = {};
+            props.allocType = cudaMemAllocationTypePinned;
+            props.handleTypes = cudaMemHandleTypeNone;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = dev;
+            e = cudaMemPoolCreate(&pools[dev], &props);
+            if (e != cudaSuccess) return e;
+            unsigned long long keep = ~0ull;
+            e = cudaMemPoolSetAttribute(pools[dev], cudaMemPoolAttrReleaseThreshold, &keep);
+            if (e != cudaSuccess) return e;
+        }
+    }
+    return cudaMallocFromPoolAsync(ptr, bytes, pools[dev], s);
+}
 
 pp_status from_cuda(cudaError_t e)
 {
@@ -211,15 +264,9 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         const int per32 = 32 / p->elem;
         p->Lpad = (L + per32 - 1) / per32 * per32;
         // masks by (popcount, value)
-        const uint32_t nm = 1u << k;
-        p->level_off.assign(k + 2, 0);
-        for (uint32_t S = 1; S < nm; ++S) p->level_off[__builtin_popcount(S) + 1]++;
-        for (int j = 1; j <= k + 1; ++j) p->level_off[j] += p->level_off[j - 1];
-        p->masks.assign(nm - 1, 0);
-        {
-            std::vector<uint32_t> at(p->level_off.begin(), p->level_off.end());
-            for (uint32_t S = 1; S < nm; ++S) p->masks[at[__builtin_popcount(S)]++] = S;
-        }
+        const MaskList &ml = mask_list(k);
+        p->masks = ml.masks;
+        p->level_off = ml.level_off;
     } catch (const std::bad_alloc &) {
         delete p;
         return PP_ERR_NOMEM;
@@ -259,11 +306,9 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     }
     for (auto &q : parts)
         if (q.src && q.bytes) std::memcpy(staging.data() + q.off, q.src, q.bytes);
-    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&p->d_inputs), total);
+    cudaError_t e = staging_alloc(reinterpret_cast<void **>(&p->d_inputs), total, nullptr);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_inputs, staging.data(), total, cudaMemcpyHostToDevice);
     for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreate(&p->ev[i]);
-    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->h_sol), sizeof(pp_solution));
-    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void **>(&p->h_err), sizeof(int32_t));
     if (e != cudaSuccess) {
         pp_status rc = from_cuda(e);
         pp_problem_destroy(p);
@@ -293,11 +338,9 @@ void pp_problem_destroy(pp_problem *p)
 {
     if (!p) return;
     if (p->own_work && p->d_work) cudaFree(p->d_work);
-    if (p->d_inputs) cudaFree(p->d_inputs);
+    if (p->d_inputs) cudaFreeAsync(p->d_inputs, p->stream);  // ordered after the problem's queued work
     for (auto &e : p->ev)
         if (e) cudaEventDestroy(e);
-    if (p->h_sol) cudaFreeHost(p->h_sol);
-    if (p->h_err) cudaFreeHost(p->h_err);
     delete p;
 }
 
@@ -400,8 +443,8 @@ pp_status pp_eval_plans(pp_problem *p, int64_t B, const uint8_t *nseg, const int
     size_t o_beta = align_up(o_nodes + b_rows, 256), o_st = align_up(o_beta + b_beta, 256);
     size_t total = o_st + (size_t)B;
     unsigned char *buf = nullptr;
-    PP_CUDA(cudaMalloc(reinterpret_cast<void **>(&buf), total));
     cudaStream_t s = p->stream;
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), total, s));
     cudaError_t e = cudaMemcpyAsync(buf, nseg, b_nseg, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_ends, ends, b_rows, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_nodes, nodes, b_rows, cudaMemcpyHostToDevice, s);
@@ -411,8 +454,8 @@ pp_status pp_eval_plans(pp_problem *p, int64_t B, const uint8_t *nseg, const int
                         reinterpret_cast<double *>(buf + o_beta), buf + o_st, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(beta_ms, buf + o_beta, b_beta, cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(plan_status, buf + o_st, (size_t)B, cudaMemcpyDeviceToHost, s);
+    cudaFreeAsync(buf, s);
     cudaError_t e2 = cudaStreamSynchronize(s);
-    cudaFree(buf);
     if (e != cudaSuccess) return from_cuda(e);
     return from_cuda(e2);
 }
@@ -455,8 +498,8 @@ pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *
     off[0] = 0;
     for (int i = 0; i < 9; ++i) off[i + 1] = align_up(off[i] + sz[i], 256);
     unsigned char *buf = nullptr;
-    PP_CUDA(cudaMalloc(reinterpret_cast<void **>(&buf), off[9]));
     cudaStream_t s = nullptr;
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), off[9], s));
     const void *src[4] = {out_bits, mem, node_mem, bw};
     cudaError_t e = cudaSuccess;
     for (int i = 0; i < 4 && e == cudaSuccess; ++i)
@@ -480,8 +523,8 @@ pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *
             if (n) e = cudaMemcpyAsync(dst[i], buf + off[4 + i], n, cudaMemcpyDeviceToHost, s);
         }
     }
+    cudaFreeAsync(buf, s);
     cudaError_t e2 = cudaStreamSynchronize(s);
-    cudaFree(buf);
     if (st != PP_OK) return st;
     if (e != cudaSuccess) return from_cuda(e);
     return from_cuda(e2);
