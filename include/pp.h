@@ -84,7 +84,8 @@ typedef struct {
     int32_t sweep_launches;  /* kernels launched for the sweep, base frontier included */
     int32_t total_launches;  /* all kernels of the solve */
     int32_t state_bytes;     /* bytes of one state element: 2 (16-bit ranks) or 4 */
-    int32_t fast_path;       /* 1 if the register-tiled sweep kernel ran, 0 if the generic one */
+    int32_t fast_path;       /* register-tiled sweep: 1 = constant-width windows, 2 = general
+                                windows; 0 = the generic kernel ran */
 } pp_profile;
 
 /*

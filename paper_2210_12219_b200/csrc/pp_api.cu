@@ -190,7 +190,7 @@ pp_status queue_solve(pp_problem *p, pp_solution *sol_dev)
     PP_CUDA(cudaEventRecord(p->ev[3], s));
     p->sweep_launches = sweep;
     p->total_launches = launches + sweep + 1;
-    p->fast_used = fast ? 1 : 0;
+    p->fast_used = fast ? (p->d.fast_meta ? 1 : 2) : 0;
     p->solved = true;
     return PP_OK;
 }

@@ -1,9 +1,10 @@
 // Register-tiled sweep of one popcount level for 16-bit ranks.
 //
-// Envelope: 16-bit state elements, Lpad <= 240 (rows occupy at most 30 lanes), the whole rank
-// table in shared memory, and for every node w a sliding window of constant width:
-// lo_w(c') = max(0, c' - W_w), W_w >= 8 (chains whose layers all need the same memory, e.g.
-// stacks of identical blocks).  Anything else runs on the generic kernel.
+// Envelope: 16-bit state elements, Lpad <= 240 (rows occupy at most 30 lanes) and the whole rank
+// table in shared memory.  Two window steps: a shuffle-only one when every node w has a sliding
+// window of constant width, lo_w(c') = max(0, c' - W_w), W_w >= 8 (chains whose layers all need
+// the same memory, e.g. stacks of identical blocks), and one for arbitrary window tables that
+// goes through per-warp shared-memory strips.  Anything else runs on the generic kernel.
 //
 // Mapping: one warp per source mask S.  Lane l owns the 8 consecutive cut positions 8l..8l+7 of
 // every row, as four packed u16x2 registers (one 16-byte vector).  The |S| source rows
@@ -83,6 +84,7 @@ __device__ __forceinline__ void min_shfl_up(uint32_t &acc, uint32_t x, int delta
 }
 
 constexpr int NT = PP_FAST_NT;  // target nodes processed together
+constexpr int kStripElems = 256 + 256 + 160;  // per-warp strips of the general window step (u16)
 
 // Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].
 __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mptr,
@@ -170,6 +172,84 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
     }
 }
 
+// Window minimum for arbitrary (non-decreasing) window starts lo_w(c'), read from the window table
+// staged in shared memory.  Same block decomposition as above, but the tail of the block that
+// holds lo, and the whole blocks in between, are fetched from per-warp shared-memory strips:
+//   sfx[c]     in-lane inclusive suffix minima of every lane,
+//   T[s][l]    minimum of the 2^s block minima ending at lane l (sparse table, s = 0..4),
+//   g[c]       the relaxed row itself, for the rare window that lies inside one block.
+__device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const uint16_t *lo_row,
+                                                   uint16_t *sfx, uint16_t *gs, uint16_t *T, int lane,
+                                                   bool active, uint32_t (&o)[4])
+{
+    const uint32_t m0 = vmin2(r[0], __byte_perm(r[0], 0, 0x1032));
+    const uint32_t m1 = vmin2(r[1], __byte_perm(r[1], 0, 0x1032));
+    const uint32_t m2 = vmin2(r[2], __byte_perm(r[2], 0, 0x1032));
+    const uint32_t m3 = vmin2(r[3], __byte_perm(r[3], 0, 0x1032));
+    const uint32_t q1 = vmin2(m0, m1), q2 = vmin2(q1, m2);
+    const uint32_t t2 = vmin2(m2, m3), t1 = vmin2(m1, t2);
+    const uint32_t B = vmin2(q2, m3);
+    // exclusive in-lane prefix minima, one per position
+    uint32_t xp[4];
+    xp[0] = __byte_perm(r[0], kInf2, 0x1044);
+    xp[1] = vmin2(m0, __byte_perm(r[1], kInf2, 0x1044));
+    xp[2] = vmin2(q1, __byte_perm(r[2], kInf2, 0x1044));
+    xp[3] = vmin2(q2, __byte_perm(r[3], kInf2, 0x1044));
+    const uint32_t s0 = vmin2(__byte_perm(m0, r[0], 0x7610), t1);
+    const uint32_t s1 = vmin2(__byte_perm(m1, r[1], 0x7610), t2);
+    const uint32_t s2 = vmin2(__byte_perm(m2, r[2], 0x7610), m3);
+    const uint32_t s3 = __byte_perm(m3, r[3], 0x7610);
+    __syncwarp();  // the previous row's readers are done with the strips
+    *reinterpret_cast<uint4 *>(sfx + 8 * lane) = make_uint4(s0, s1, s2, s3);
+    *reinterpret_cast<uint4 *>(gs + 8 * lane) = make_uint4(r[0], r[1], r[2], r[3]);
+    uint32_t D = B;
+    T[lane] = (uint16_t)D;
+    min_shfl_up(D, D, 1); T[32 + lane] = (uint16_t)D;
+    min_shfl_up(D, D, 2); T[64 + lane] = (uint16_t)D;
+    min_shfl_up(D, D, 4); T[96 + lane] = (uint16_t)D;
+    min_shfl_up(D, D, 8); T[128 + lane] = (uint16_t)D;
+    __syncwarp();
+    const int base = 8 * lane;
+    // lanes beyond the row have no window table entries: give them empty windows (start = own
+    // position), which also keeps every index below inside the 256-element strips
+    const uint32_t own = (uint32_t)base * 0x00010001u + 0x00010000u;  // (base, base + 1)
+    uint4 lov = make_uint4(own, own + 0x00020002u, own + 0x00040004u, own + 0x00060006u);
+    if (active) lov = *reinterpret_cast<const uint4 *>(lo_row + 8 * lane);
+    const uint32_t lw[4] = {lov.x, lov.y, lov.z, lov.w};
+    uint32_t val[8];
+    bool inblock = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int a = (int)((lw[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);  // window start
+        const int c2 = base + i;
+        const uint32_t x = (xp[i >> 1] >> (16 * (i & 1))) & 0xFFFFu;
+        const int la = a >> 3;
+        const int n = lane - 1 - la;  // whole blocks strictly between
+        uint32_t v = min(x, (uint32_t)sfx[a]);
+        if (n >= 1) {
+            const int s = 31 - __clz(n);
+            v = min(v, min((uint32_t)T[s * 32 + lane - 1], (uint32_t)T[s * 32 + la + (1 << s)]));
+        }
+        if (a >= c2) v = 0xFFFFu;               // empty window
+        else if (a >= base) inblock = true;      // window inside this lane's block: fixed below
+        val[i] = v;
+    }
+    if (__any_sync(0xFFFFFFFFu, inblock)) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int a = (int)((lw[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+            const int c2 = base + i;
+            if (a >= base && a < c2) {
+                uint32_t v = 0xFFFFu;
+                for (int c = a; c < c2; ++c) v = min(v, (uint32_t)gs[c]);
+                val[i] = v;
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = val[2 * j] | (val[2 * j + 1] << 16);
+}
+
 // Slow path of the final-state bookkeeping, kept out of line so that the common case is a
 // compare and a branch.
 __device__ __noinline__ unsigned long long offer_final(unsigned long long *best, unsigned long long best_seen,
@@ -183,7 +263,7 @@ __device__ __noinline__ unsigned long long offer_final(unsigned long long *best,
     return best_seen;
 }
 
-template <int NV>
+template <int NV, bool GEN>
 __global__ void __launch_bounds__(kFastThreads, 1)
 k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
 {
@@ -203,10 +283,21 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
         for (int i = threadIdx.x; i < rank_elems / 8; i += kFastThreads) smem4[i] = src[i];
         for (int i = threadIdx.x; i < 32; i += kFastThreads)
             smem4[rank_elems / 8 + i] = make_uint4(kInf2, kInf2, kInf2, kInf2);
-        const int *ms = reinterpret_cast<const int *>(meta_g);
-        int *md = reinterpret_cast<int *>(wm);
-        for (int i = threadIdx.x; i < (int)(sizeof(WMeta) / 4) * k; i += kFastThreads) md[i] = ms[i];
+        if (!GEN) {
+            const int *ms = reinterpret_cast<const int *>(meta_g);
+            int *md = reinterpret_cast<int *>(wm);
+            for (int i = threadIdx.x; i < (int)(sizeof(WMeta) / 4) * k; i += kFastThreads) md[i] = ms[i];
+        }
     }
+    // general windows: the window table lo[w][c'] (row stride Lpad, pads empty) and three strips
+    // per warp live behind the per-node constants
+    uint16_t *lo_s = reinterpret_cast<uint16_t *>(wm + PP_MAX_K);
+    uint16_t *strips = lo_s + k * Lpad + (threadIdx.x >> 5) * kStripElems;
+    if (GEN)
+        for (int i = threadIdx.x; i < k * Lpad; i += kFastThreads) {
+            const int w = i / Lpad, c = i - w * Lpad;
+            lo_s[i] = (uint16_t)(c < L ? d.lo[w * L + c] : c);
+        }
     __syncthreads();
     asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
 
@@ -314,7 +405,10 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
 #pragma unroll
             for (int t = 0; t < NT; ++t) mp[t] = wm + w[t];
             uint32_t o[NT][4];
-            window_min(r, mp, o);
+            if (GEN)
+                window_min_general(r[0], lo_s + w[0] * Lpad, strips, strips + 256, strips + 512, lane, active, o[0]);
+            else
+                window_min(r, mp, o);
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
                 const uint32_t S2 = S_cur | (1u << w[t]);
@@ -361,13 +455,16 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
 
 size_t fast_smem_bytes(const Dev &d)
 {
-    return (((size_t)d.k * d.k * d.Lpad * 2 + 512 + 15) & ~(size_t)15) + sizeof(WMeta) * PP_MAX_K;
+    size_t b = (((size_t)d.k * d.k * d.Lpad * 2 + 512 + 15) & ~(size_t)15) + sizeof(WMeta) * PP_MAX_K;
+    if (!d.fast_meta)  // general windows: window table + strips
+        b += ((size_t)d.k * d.Lpad + (size_t)(kFastThreads / 32) * kStripElems) * 2;
+    return b;
 }
 
-template <int NV>
+template <int NV, bool GEN>
 cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned grid, int split, size_t sm, cudaStream_t s)
 {
-    cudaError_t e = cudaFuncSetAttribute(k_sweep_fast<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    cudaError_t e = cudaFuncSetAttribute(k_sweep_fast<NV, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -379,7 +476,7 @@ cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned gr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_sweep_fast<NV>, d, level, meta, split);
+    return cudaLaunchKernelEx(&cfg, k_sweep_fast<NV, GEN>, d, level, meta, split);
 }
 
 }  // namespace
@@ -423,7 +520,7 @@ bool fast_meta_build(int L, int k, const int16_t *lo, void *out)
 
 bool fast_sweep_supported(const Dev &d)
 {
-    if (d.elem != 2 || d.Lpad > 240 || d.k < 2 || d.k > PP_MAX_K || !d.fast_meta) return false;
+    if (d.elem != 2 || d.Lpad > 240 || d.k < 2 || d.k > PP_MAX_K) return false;
     int dev = 0, max_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&max_sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
@@ -449,7 +546,9 @@ cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s)
     const size_t sm = fast_smem_bytes(d);
     const FastMeta *meta = static_cast<const FastMeta *>(d.fast_meta);
     switch (level - 1) {
-#define PP_CASE(N) case N: return launch_nv<N>(d, level, meta, grid, split, sm, s);
+#define PP_CASE(N) \
+    case N: return meta ? launch_nv<N, false>(d, level, meta, grid, split, sm, s) \
+                        : launch_nv<N, true>(d, level, meta, grid, split, sm, s);
         PP_CASE(1) PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6) PP_CASE(7) PP_CASE(8)
         PP_CASE(9) PP_CASE(10) PP_CASE(11) PP_CASE(12) PP_CASE(13) PP_CASE(14) PP_CASE(15)
         PP_CASE(16) PP_CASE(17) PP_CASE(18) PP_CASE(19)

@@ -146,11 +146,44 @@ def test_register_tiled_sweep_on_uniform_memory_chains():
                 assert_same(inst, p.solve_exact(), want)
                 assert p.last_solve_profile().fast_path == 0
     assert n_fast >= 80
-    # a node whose window is narrower than 8 layers sends the instance to the generic kernel
+    # a node whose window is narrower than 8 layers takes the general-window variant
     inst = W.uniform_memory_small(81000, 30, 4, 3, 7)
     with pp.Problem.from_instance(inst) as p:
         assert_same(inst, p.solve_exact(), oracle.dp_fact(inst))
-        assert p.last_solve_profile().fast_path == 0
+        assert p.last_solve_profile().fast_path == 2
+
+
+def test_register_tiled_sweep_with_general_windows():
+    # arbitrary layer memories: window starts come from the staged window table; includes
+    # windows inside one 8-position block, empty windows, windows reaching layer 0, L from one
+    # lane to 30 lanes, and every state compared on the small ones
+    seed = 0
+    for L, k, n in ((5, 3, 8), (9, 4, 10), (17, 5, 10), (33, 6, 10), (64, 6, 6), (100, 7, 5), (150, 5, 5),
+                    (199, 4, 5), (240, 4, 4), (12, 8, 6), (50, 10, 2)):
+        for i in range(n):
+            kind = i % 4
+            inst = W.random_small(85000 + seed, L, k, tight=(kind == 1), ties=(kind == 2),
+                                  dead_links=0.3 if kind == 3 else 0.0)
+            if kind == 0 and L >= 30:  # long windows: a few nodes hold most of the chain
+                cap = inst.node_mem_bytes.copy()
+                cap[: max(1, k // 2)] = np.uint64(int(inst.layer_mem_bytes.sum()) // 2)
+                inst = make_instance(inst.layer_out_bits, inst.layer_mem_bytes, cap, inst.bw_kbps, inst.name)
+            seed += 1
+            want = oracle.dp_fact(inst, 4, want_table=(L * (1 << k) <= 16384))
+            with pp.Problem.from_instance(inst) as p:
+                got = p.solve_exact()
+                assert p.last_solve_profile().fast_path == 2, inst.name
+                assert_same(inst, got, want)
+                if want.table is not None:
+                    for S in range(1, 1 << k):
+                        for v in range(k):
+                            if S >> v & 1 and bin(S).count("1") <= L:
+                                assert np.array_equal(p.debug_read_state_row(S, v), want.table[S, v]), \
+                                    (inst.name, S, v)
+    for inst in (W.config_resnet50_shaped(), W.config_deeper_cnn()):
+        with pp.Problem.from_instance(inst) as p:
+            assert_same(inst, p.solve_exact(), oracle.dp_fact(inst, 8))
+            assert p.last_solve_profile().fast_path == 2
 
 
 def test_named_configs_2_and_3():
