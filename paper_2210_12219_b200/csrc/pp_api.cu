@@ -283,6 +283,16 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         delete p;
         return PP_ERR_NOMEM;
     }
+    std::vector<uint32_t> gmeta;
+    try {
+        if (!has_fast && p->elem == 2 && p->Lpad <= 240 && k >= 2) {
+            gmeta.resize((size_t)k * p->Lpad);
+            gen_meta_build(L, k, p->Lpad, p->lo.data(), gmeta.data());
+        }
+    } catch (const std::bad_alloc &) {
+        delete p;
+        return PP_ERR_NOMEM;
+    }
     // upload the small arrays in one allocation
     struct Part { const void *src; size_t bytes; size_t off; };
     std::vector<Part> parts = {
@@ -293,7 +303,8 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         {p->masks.data(), p->masks.size() * 4, 0},     {p->level_off.data(), p->level_off.size() * 4, 0},
         {nullptr, 8, 0} /* best */,                    {nullptr, 4, 0} /* err */,
         {nullptr, sizeof(pp_solution), 0} /* solution */,
-        {fmeta.data(), fmeta.size(), 0}};
+        {fmeta.data(), fmeta.size(), 0},
+        {gmeta.data(), gmeta.size() * 4, 0}};
     size_t total = 0;
     for (auto &q : parts) { q.off = total; total = align_up(total + q.bytes, 256); }
     // one staging buffer, one copy: the parts are small and a copy per part costs more than the bytes
@@ -330,6 +341,7 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     d.err = reinterpret_cast<int32_t *>(b + parts[10].off);
     p->d_sol = reinterpret_cast<pp_solution *>(b + parts[11].off);
     d.fast_meta = has_fast ? b + parts[12].off : nullptr;
+    d.gen_meta = gmeta.empty() ? nullptr : reinterpret_cast<uint32_t *>(b + parts[13].off);
     *out = p;
     return PP_OK;
 }

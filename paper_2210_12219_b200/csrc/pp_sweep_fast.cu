@@ -84,7 +84,7 @@ __device__ __forceinline__ void min_shfl_up(uint32_t &acc, uint32_t x, int delta
 }
 
 constexpr int NT = PP_FAST_NT;  // target nodes processed together
-constexpr int kStripElems = 256 + 256 + 160;  // per-warp strips of the general window step (u16)
+constexpr int kStripElems = 256 + 256 + 168;  // per-warp strips of the general window step (u16)
 
 // Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].
 __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mptr,
@@ -172,13 +172,16 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
     }
 }
 
-// Window minimum for arbitrary (non-decreasing) window starts lo_w(c'), read from the window table
-// staged in shared memory.  Same block decomposition as above, but the tail of the block that
-// holds lo, and the whole blocks in between, are fetched from per-warp shared-memory strips:
-//   sfx[c]     in-lane inclusive suffix minima of every lane,
-//   T[s][l]    minimum of the 2^s block minima ending at lane l (sparse table, s = 0..4),
+// Window minimum for arbitrary (non-decreasing) window starts lo_w(c').  Same block decomposition
+// as above, but the tail of the block that holds lo, and the whole blocks in between, are fetched
+// from per-warp shared-memory strips through lookup words prepared on the host (gen_meta_build):
+//   sfx[i][l]  in-lane inclusive suffix minima of every lane (position-major); entry (0, 30) is
+//              +inf because rows occupy at most 30 lanes,
+//   T[s][l]    minimum of the 2^s block minima ending at lane l (sparse table, s = 0..4);
+//              T[160] is a constant +inf,
 //   g[c]       the relaxed row itself, for the rare window that lies inside one block.
-__device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const uint16_t *lo_row,
+// Lookup word of (w, c'): sfx index | T index 1 << 8 | T index 2 << 16 | lo << 24.
+__device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const uint32_t *meta_row,
                                                    uint16_t *sfx, uint16_t *gs, uint16_t *T, int lane,
                                                    bool active, uint32_t (&o)[4])
 {
@@ -195,12 +198,11 @@ __device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const
     xp[1] = vmin2(m0, __byte_perm(r[1], kInf2, 0x1044));
     xp[2] = vmin2(q1, __byte_perm(r[2], kInf2, 0x1044));
     xp[3] = vmin2(q2, __byte_perm(r[3], kInf2, 0x1044));
-    const uint32_t s0 = vmin2(__byte_perm(m0, r[0], 0x7610), t1);
-    const uint32_t s1 = vmin2(__byte_perm(m1, r[1], 0x7610), t2);
-    const uint32_t s2 = vmin2(__byte_perm(m2, r[2], 0x7610), m3);
-    const uint32_t s3 = __byte_perm(m3, r[3], 0x7610);
+    const uint32_t sv[4] = {vmin2(__byte_perm(m0, r[0], 0x7610), t1), vmin2(__byte_perm(m1, r[1], 0x7610), t2),
+                            vmin2(__byte_perm(m2, r[2], 0x7610), m3), __byte_perm(m3, r[3], 0x7610)};
     __syncwarp();  // the previous row's readers are done with the strips
-    *reinterpret_cast<uint4 *>(sfx + 8 * lane) = make_uint4(s0, s1, s2, s3);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sfx[i * 32 + lane] = (uint16_t)(sv[i >> 1] >> (16 * (i & 1)));
     *reinterpret_cast<uint4 *>(gs + 8 * lane) = make_uint4(r[0], r[1], r[2], r[3]);
     uint32_t D = B;
     T[lane] = (uint16_t)D;
@@ -209,36 +211,29 @@ __device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const
     min_shfl_up(D, D, 4); T[96 + lane] = (uint16_t)D;
     min_shfl_up(D, D, 8); T[128 + lane] = (uint16_t)D;
     __syncwarp();
+    // lanes beyond the row take empty windows whose lookups all hit the +inf entries
+    const uint4 none = make_uint4(0xFFA0A01Eu, 0xFFA0A01Eu, 0xFFA0A01Eu, 0xFFA0A01Eu);
+    const uint4 ma = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane) : none;
+    const uint4 mb = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane + 4) : none;
+    const uint32_t mw[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
     const int base = 8 * lane;
-    // lanes beyond the row have no window table entries: give them empty windows (start = own
-    // position), which also keeps every index below inside the 256-element strips
-    const uint32_t own = (uint32_t)base * 0x00010001u + 0x00010000u;  // (base, base + 1)
-    uint4 lov = make_uint4(own, own + 0x00020002u, own + 0x00040004u, own + 0x00060006u);
-    if (active) lov = *reinterpret_cast<const uint4 *>(lo_row + 8 * lane);
-    const uint32_t lw[4] = {lov.x, lov.y, lov.z, lov.w};
     uint32_t val[8];
     bool inblock = false;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const int a = (int)((lw[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);  // window start
-        const int c2 = base + i;
+        const uint32_t w = mw[i];
+        const int a = (int)(w >> 24), c2 = base + i;
         const uint32_t x = (xp[i >> 1] >> (16 * (i & 1))) & 0xFFFFu;
-        const int la = a >> 3;
-        const int n = lane - 1 - la;  // whole blocks strictly between
-        uint32_t v = min(x, (uint32_t)sfx[a]);
-        if (n >= 1) {
-            const int s = 31 - __clz(n);
-            v = min(v, min((uint32_t)T[s * 32 + lane - 1], (uint32_t)T[s * 32 + la + (1 << s)]));
-        }
-        if (a >= c2) v = 0xFFFFu;               // empty window
-        else if (a >= base) inblock = true;      // window inside this lane's block: fixed below
+        uint32_t v = min(min((uint32_t)sfx[w & 255u], (uint32_t)T[(w >> 8) & 255u]),
+                         min((uint32_t)T[(w >> 16) & 255u], x));
+        if (a >= c2) v = 0xFFFFu;           // empty window
+        else if (a >= base) inblock = true;  // window inside this lane's block: fixed below
         val[i] = v;
     }
     if (__any_sync(0xFFFFFFFFu, inblock)) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int a = (int)((lw[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
-            const int c2 = base + i;
+            const int a = (int)(mw[i] >> 24), c2 = base + i;
             if (a >= base && a < c2) {
                 uint32_t v = 0xFFFFu;
                 for (int c = a; c < c2; ++c) v = min(v, (uint32_t)gs[c]);
@@ -289,15 +284,14 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
             for (int i = threadIdx.x; i < (int)(sizeof(WMeta) / 4) * k; i += kFastThreads) md[i] = ms[i];
         }
     }
-    // general windows: the window table lo[w][c'] (row stride Lpad, pads empty) and three strips
-    // per warp live behind the per-node constants
-    uint16_t *lo_s = reinterpret_cast<uint16_t *>(wm + PP_MAX_K);
-    uint16_t *strips = lo_s + k * Lpad + (threadIdx.x >> 5) * kStripElems;
-    if (GEN)
-        for (int i = threadIdx.x; i < k * Lpad; i += kFastThreads) {
-            const int w = i / Lpad, c = i - w * Lpad;
-            lo_s[i] = (uint16_t)(c < L ? d.lo[w * L + c] : c);
-        }
+    // general windows: the lookup words of every (node, position) and three strips per warp live
+    // behind the per-node constants
+    uint32_t *gm_s = reinterpret_cast<uint32_t *>(wm + PP_MAX_K);
+    uint16_t *strips = reinterpret_cast<uint16_t *>(gm_s + k * Lpad) + (threadIdx.x >> 5) * kStripElems;
+    if (GEN) {
+        for (int i = threadIdx.x; i < k * Lpad; i += kFastThreads) gm_s[i] = d.gen_meta[i];
+        if ((threadIdx.x & 31) == 0) strips[512 + 160] = 0xFFFFu;  // the constant +inf of the T strip
+    }
     __syncthreads();
     asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
 
@@ -406,7 +400,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
             for (int t = 0; t < NT; ++t) mp[t] = wm + w[t];
             uint32_t o[NT][4];
             if (GEN)
-                window_min_general(r[0], lo_s + w[0] * Lpad, strips, strips + 256, strips + 512, lane, active, o[0]);
+                window_min_general(r[0], gm_s + w[0] * Lpad, strips, strips + 256, strips + 512, lane, active, o[0]);
             else
                 window_min(r, mp, o);
 #pragma unroll
@@ -456,8 +450,8 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
 size_t fast_smem_bytes(const Dev &d)
 {
     size_t b = (((size_t)d.k * d.k * d.Lpad * 2 + 512 + 15) & ~(size_t)15) + sizeof(WMeta) * PP_MAX_K;
-    if (!d.fast_meta)  // general windows: window table + strips
-        b += ((size_t)d.k * d.Lpad + (size_t)(kFastThreads / 32) * kStripElems) * 2;
+    if (!d.fast_meta)  // general windows: lookup words + strips
+        b += (size_t)d.k * d.Lpad * 4 + (size_t)(kFastThreads / 32) * kStripElems * 2;
     return b;
 }
 
@@ -518,9 +512,32 @@ bool fast_meta_build(int L, int k, const int16_t *lo, void *out)
     return true;
 }
 
+// Lookup words of the general window step (see window_min_general), row stride Lpad <= 240.
+void gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out)
+{
+    for (int w = 0; w < k; ++w)
+        for (int c2 = 0; c2 < Lpad; ++c2) {
+            const int a = c2 < L ? lo[w * L + c2] : c2;  // pads: empty window
+            const int lane = c2 >> 3, base = lane * 8;
+            uint32_t sfx = 30, t1 = 160, t2 = 160;      // the +inf entries
+            if (a < c2 && a < base) {
+                const int la = a >> 3, oa = a & 7;
+                sfx = (uint32_t)(oa * 32 + la);
+                const int n = lane - 1 - la;
+                if (n >= 1) {
+                    int s = 0;
+                    while ((2 << s) <= n) ++s;
+                    t1 = (uint32_t)(s * 32 + lane - 1);
+                    t2 = (uint32_t)(s * 32 + la + (1 << s));
+                }
+            }
+            out[w * Lpad + c2] = sfx | (t1 << 8) | (t2 << 16) | ((uint32_t)a << 24);
+        }
+}
+
 bool fast_sweep_supported(const Dev &d)
 {
-    if (d.elem != 2 || d.Lpad > 240 || d.k < 2 || d.k > PP_MAX_K) return false;
+    if (d.elem != 2 || d.Lpad > 240 || d.k < 2 || d.k > PP_MAX_K || (!d.fast_meta && !d.gen_meta)) return false;
     int dev = 0, max_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&max_sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
