@@ -1,24 +1,27 @@
 // Register-tiled sweep of one popcount level for 16-bit ranks.
 //
 // Envelope: 16-bit state elements, Lpad <= 240 (rows occupy at most 30 lanes) and the whole rank
-// table in shared memory.  Two window steps: a shuffle-only one when every node w has a sliding
-// window of constant width, lo_w(c') = max(0, c' - W_w), W_w >= 8 (chains whose layers all need
-// the same memory, e.g. stacks of identical blocks), and one for arbitrary window tables that
-// goes through per-warp shared-memory strips.  Anything else runs on the generic kernel.
+// table in shared memory.  Two window steps: one for nodes whose sliding window has a constant
+// width, lo_w(c') = max(0, c' - W_w), W_w >= 8 (chains whose layers all need the same memory,
+// e.g. stacks of identical blocks), and one for arbitrary window tables that looks everything up
+// in per-warp shared-memory strips.  Anything else runs on the generic kernel.
 //
 // Mapping: one warp per source mask S.  Lane l owns the 8 consecutive cut positions 8l..8l+7 of
 // every row, as four packed u16x2 registers (one 16-byte vector).  The |S| source rows
-// dp[S][v][.] are loaded once into registers; then, two target nodes w not in S at a time (their
-// instruction streams interleaved so that one's shuffle latency hides behind the other), the warp
+// dp[S][v][.] are loaded once into registers; then, for every target node w not in S, the warp
 //   1. relaxes   g[c] = min_v max(dp[S][v][c], rank[w][v][c])    (one 128-bit shared-memory load
-//      and eight packed min/max per (v, w) and lane),
+//      and eight packed min/max per (v, w) and lane; two source nodes share a three-input min),
 //   2. takes the window minimum  out[c'] = min g[c'-W .. c'-1]   with blocks of 8 = lanes:
-//      window = tail of the block that holds c'-W  (in-lane suffix minima, fetched by shuffles)
-//             + whole blocks in between            (sliding minimum over the block minima)
+//      window = tail of the block that holds c'-W  (in-lane suffix minima, published to a
+//               per-warp strip and read back at offset -W)
+//             + whole blocks in between            (sliding minimum over the block minima,
+//               by doubling shuffles)
 //             + head of the own block              (in-lane exclusive prefix minima),
 //      all of it branch-free: what a node does not need is a shuffle from distance 31, which
-//      finds no source lane and leaves the accumulator alone,
+//      finds no source lane and leaves the accumulator alone, or a read of the +inf pad,
 //   3. writes row dp[S + w][w][.] with one 16-byte store per lane.
+// The relaxation of the next target node is issued in the same straight-line block as the window
+// step of the current one, so that independent loads fill the latencies of the dependent chain.
 // Row (S + w, w) has the single source mask S, so no two warps ever write the same row.
 #include "pp_internal.cuh"
 
@@ -26,27 +29,31 @@ namespace pp {
 
 namespace {
 
-#ifndef PP_FAST_THREADS
-#define PP_FAST_THREADS 512
+#ifndef PP_NV768
+#define PP_NV768 6
+#endif
+#ifndef PP_NV640
+#define PP_NV640 9
 #endif
 #ifndef PP_FAST_NT
 #define PP_FAST_NT 1
 #endif
-constexpr int kFastThreads = PP_FAST_THREADS;
+// Threads per block by the number of source rows a warp keeps in registers: fewer rows leave room
+// for more resident warps (the register file holds 64K registers per SM).
+constexpr int kMaxFastThreads = 768;
+__host__ __device__ constexpr int fast_threads(int nv, bool gen) { return gen ? 512 : (nv <= PP_NV768 ? 768 : (nv <= PP_NV640 ? 640 : 512)); }
 constexpr uint32_t kInf2 = 0xFFFFFFFFu;
 
-// Per-target-node constants of the window step (W = 8q + r, e = r >> 1), built on the host.
+// Per-target-node constants of the window step (W = 8q + r), built on the host.
 // A shuffle distance of 31 means "nothing": rows occupy at most 30 lanes, so no lane that holds
 // data finds a source and +inf (or the untouched accumulator) results.
 struct alignas(16) WMeta {
-    int de[4];       // source distance of suffix register j: q, or q + 1 when j < e
-    int dx;          // q + 1: the extra register that an odd r needs
-    int sh16;        // 16 if r is odd else 0
-    int rot1, rot2;  // e & 1, e & 2: rotate the suffix registers by e before they travel
-    int dd[4];       // doubling distances 1, 2, 4, 8 for the first s steps, then 31
+    int toff;        // -ceil(W / 2): 32-bit word offset of position c' - W in the suffix strip
+    int sh16;        // 16 if W is odd else 0
     int d1, d2;      // T1 = min(D << d1, D << d2): 1 and 1 + n1 - 2^s, or 31 when n1 = q - 1 = 0
+    int dd[4];       // doubling distances 1, 2, 4, 8 for the first s steps, then 31
     int dq;          // q: the one more block that positions below r need
-    int pad;
+    int pad[3];
     uint32_t sel[4]; // byte selectors that pick T(q) or T(q-1) per half of each register
 };
 
@@ -85,12 +92,15 @@ __device__ __forceinline__ void min_shfl_up(uint32_t &acc, uint32_t x, int delta
 
 constexpr int NT = PP_FAST_NT;  // target nodes processed together
 constexpr int kStripElems = 256 + 256 + 168;  // per-warp strips of the general window step (u16)
+constexpr int kTailWords = 128 + 128;           // per-warp suffix strip of the constant-window step: +inf pad, data
 
-// Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].
-__device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mptr,
+// Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].  tl points at this lane's four
+// words of the warp's suffix strip; the 128 words below the strip hold +inf.
+__device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMeta *const *mptr, uint32_t *tl,
                                            uint32_t (&o)[NT][4])
 {
-    // the constants of each node arrive as five 16-byte shared-memory loads
+    static_assert(NT == 1, "the suffix strip holds one row at a time");
+    // the constants of each node arrive as four 16-byte shared-memory loads
     union MetaRegs {
         WMeta m;
         uint4 q[sizeof(WMeta) / 16];
@@ -104,7 +114,8 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
     const WMeta *mp[NT];
 #pragma unroll
     for (int t = 0; t < NT; ++t) mp[t] = &mr[t].m;
-    uint32_t z[NT][4], B[NT];
+    uint32_t B[NT];
+    uint32_t f[NT][5];
 #pragma unroll
     for (int t = 0; t < NT; ++t) {
         // pair minima replicated in both halves, their prefix (q*) and suffix (t*) minima
@@ -120,29 +131,20 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
         o[t][1] = vmin2(m0, __byte_perm(r[t][1], kInf2, 0x1044));
         o[t][2] = vmin2(q1, __byte_perm(r[t][2], kInf2, 0x1044));
         o[t][3] = vmin2(q2, __byte_perm(r[t][3], kInf2, 0x1044));
-        // inclusive in-lane suffix minima: (min g[2j..7], min g[2j+1..7])
+        // inclusive in-lane suffix minima: (min g[2j..7], min g[2j+1..7]), published to the strip
         const uint32_t s0 = vmin2(__byte_perm(m0, r[t][0], 0x7610), t1);
         const uint32_t s1 = vmin2(__byte_perm(m1, r[t][1], 0x7610), t2);
         const uint32_t s2 = vmin2(__byte_perm(m2, r[t][2], 0x7610), m3);
         const uint32_t s3 = __byte_perm(m3, r[t][3], 0x7610);
-        // rotate the four suffix registers right by e = r >> 1 so that register j is the one
-        // output register j needs, whichever lane it comes from
-        const bool p1 = mp[t]->rot1 != 0, p2 = mp[t]->rot2 != 0;
-        const uint32_t a0 = p1 ? s3 : s0, a1 = p1 ? s0 : s1, a2 = p1 ? s1 : s2, a3 = p1 ? s2 : s3;
-        z[t][0] = p2 ? a2 : a0;
-        z[t][1] = p2 ? a3 : a1;
-        z[t][2] = p2 ? a0 : a2;
-        z[t][3] = p2 ? a1 : a3;
+        __syncwarp();  // the previous row's readers are done
+        *reinterpret_cast<uint4 *>(tl) = make_uint4(s0, s1, s2, s3);
+        __syncwarp();
+        // tail of the block that holds c' - W: the five words that cover positions c' - W of this
+        // lane's eight outputs (negative positions read the +inf pad)
+        const uint32_t *tp = tl + mp[t]->toff;
+#pragma unroll
+        for (int j = 0; j < 5; ++j) f[t][j] = tp[j];
     }
-    // tail of the block that holds c' - W: registers from lane l-q (or l-q-1 for j < e); for an
-    // odd r every output register straddles two of them and is funnel-shifted by 16 bits
-    uint32_t f[NT][5];
-#pragma unroll
-    for (int t = 0; t < NT; ++t) f[t][0] = shfl_up_inf(z[t][3], mp[t]->dx);
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-#pragma unroll
-        for (int t = 0; t < NT; ++t) f[t][j + 1] = shfl_up_inf(z[t][j], mp[t]->de[j]);
     // whole blocks in between: D = min B[l-2^s+1 .. l], T1 = min B[l-n1 .. l-1], T2 = min B[l-q .. l-1]
     uint32_t D[NT], T1[NT], T2[NT];
 #pragma unroll
@@ -165,7 +167,8 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
         const int sh = mp[t]->sh16;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const uint32_t e = __funnelshift_l(f[t][j], f[t][j + 1], sh);
+            // an odd W straddles two words per output register
+            const uint32_t e = __funnelshift_r(f[t][j], f[t][j + 1], sh);
             const uint32_t mid = __byte_perm(T2[t], T1[t], mp[t]->sel[j]);
             o[t][j] = vmin3(o[t][j], e, mid);
         }
@@ -259,9 +262,10 @@ __device__ __noinline__ unsigned long long offer_final(unsigned long long *best,
 }
 
 template <int NV, bool GEN>
-__global__ void __launch_bounds__(kFastThreads, 1)
+__global__ void __launch_bounds__(fast_threads(NV, GEN), 1)
 k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
 {
+    constexpr int kFastThreads = fast_threads(NV, GEN);
     // Programmatic dependent launch: let the next level's blocks be scheduled as soon as this
     // level's blocks retire, so that their prologue (rank table -> shared memory) overlaps our
     // tail.  Nothing the previous level wrote is touched before griddepcontrol.wait below.
@@ -287,6 +291,12 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
     // general windows: the lookup words of every (node, position) and three strips per warp live
     // behind the per-node constants
     uint32_t *gm_s = reinterpret_cast<uint32_t *>(wm + PP_MAX_K);
+    // constant windows: per-warp suffix strip (128 words of +inf, then the row's 128 words)
+    uint32_t *tl = gm_s + (threadIdx.x >> 5) * kTailWords + 128 + 4 * (threadIdx.x & 31);
+    if (!GEN) {
+        uint32_t *pad = gm_s + (threadIdx.x >> 5) * kTailWords;
+        for (int i = threadIdx.x & 31; i < kTailWords; i += 32) pad[i] = kInf2;
+    }
     uint16_t *strips = reinterpret_cast<uint16_t *>(gm_s + k * Lpad) + (threadIdx.x >> 5) * kStripElems;
     if (GEN) {
         for (int i = threadIdx.x; i < k * Lpad; i += kFastThreads) gm_s[i] = d.gen_meta[i];
@@ -402,7 +412,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
             if (GEN)
                 window_min_general(r[0], gm_s + w[0] * Lpad, strips, strips + 256, strips + 512, lane, active, o[0]);
             else
-                window_min(r, mp, o);
+                window_min(r, mp, tl, o);
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
                 const uint32_t S2 = S_cur | (1u << w[t]);
@@ -451,7 +461,9 @@ size_t fast_smem_bytes(const Dev &d)
 {
     size_t b = (((size_t)d.k * d.k * d.Lpad * 2 + 512 + 15) & ~(size_t)15) + sizeof(WMeta) * PP_MAX_K;
     if (!d.fast_meta)  // general windows: lookup words + strips
-        b += (size_t)d.k * d.Lpad * 4 + (size_t)(kFastThreads / 32) * kStripElems * 2;
+        b += (size_t)d.k * d.Lpad * 4 + (size_t)(512 / 32) * kStripElems * 2;
+    else               // constant windows: suffix strips
+        b += (size_t)(kMaxFastThreads / 32) * kTailWords * 4;
     return b;
 }
 
@@ -462,7 +474,7 @@ cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned gr
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kFastThreads);
+    cfg.blockDim = dim3(fast_threads(NV, GEN));
     cfg.dynamicSmemBytes = sm;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
@@ -491,13 +503,10 @@ bool fast_meta_build(int L, int k, const int16_t *lo, void *out)
         if (L > 1 && W < 8) return false;
         if (W >= L - 1) W = Lpad;  // the window always reaches layer 0: treat as "everything before"
         WMeta &m = fm->w[w];
-        const int q = W >> 3, r = W & 7, e = r >> 1;
+        const int q = W >> 3, r = W & 7;
         auto clamp = [](int x) { return x > 31 ? 31 : x; };
-        for (int j = 0; j < 4; ++j) m.de[j] = clamp(q + (j < e ? 1 : 0));
-        m.dx = (r & 1) ? clamp(q + 1) : 31;
+        m.toff = -((W + 1) >> 1);
         m.sh16 = (r & 1) ? 16 : 0;
-        m.rot1 = e & 1;
-        m.rot2 = e & 2;
         const int n1 = q - 1 > 31 ? 31 : q - 1;
         int s = 0;
         while (n1 >= 1 && (2 << s) <= n1) ++s;
@@ -505,7 +514,7 @@ bool fast_meta_build(int L, int k, const int16_t *lo, void *out)
         m.d1 = n1 >= 1 ? 1 : 31;
         m.d2 = n1 >= 1 ? 1 + n1 - (1 << s) : 31;
         m.dq = clamp(q);
-        m.pad = 0;
+        m.pad[0] = m.pad[1] = m.pad[2] = 0;
         for (int j = 0; j < 4; ++j)
             m.sel[j] = ((2 * j < r) ? 0x0010u : 0x0054u) | ((2 * j + 1 < r) ? 0x3200u : 0x7600u);
     }
@@ -551,7 +560,7 @@ cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     unsigned long long n = 1;  // source masks of popcount level-1
     for (int i = 0; i < level - 1; ++i) n = n * (unsigned)(d.k - i) / (unsigned)(i + 1);
-    const unsigned wpb = kFastThreads / 32;
+    const unsigned wpb = fast_threads(level - 1, d.fast_meta == nullptr) / 32;
     const int nw = d.k - (level - 1);  // target nodes per mask
     int split = 1;
     if (n < (unsigned long long)sms * wpb) {
