@@ -86,6 +86,8 @@ typedef struct {
     int32_t state_bytes;     /* bytes of one state element: 2 (16-bit ranks) or 4 */
     int32_t fast_path;       /* register-tiled sweep: 1 = constant-width windows, 2 = general
                                 windows; 0 = the generic kernel ran */
+    int32_t pair_levels;     /* popcount levels swept by the kernel that takes two source masks
+                                per warp (constant-width windows only) */
 } pp_profile;
 
 /*
@@ -184,8 +186,9 @@ pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out);
  * `mask` must contain node v.  Synchronous. */
 pp_status pp_debug_read_state_row(pp_problem *p, uint32_t mask, int32_t v, double *row_out);
 
-/* Force (1) or forbid (0) the generic sweep kernel; -1 restores the automatic choice.
- * Meant for tests that want both kernels checked on the same instance. */
+/* Force (1) or forbid (0) the generic sweep kernel; 2 = automatic choice among the kernels that
+ * take one source mask per warp (the two-mask kernel is left out); 3 = the two-mask kernel on every
+ * level it can run, however small; -1 restores the automatic choice.  Meant for tests that want every kernel checked on the same instance. */
 pp_status pp_problem_force_generic(pp_problem *p, int32_t mode);
 
 /*

@@ -38,7 +38,8 @@ class pp_profile(ctypes.Structure):
     _fields_ = [("ms_rank", ctypes.c_float), ("ms_sweep", ctypes.c_float),
                 ("ms_finalize", ctypes.c_float), ("ms_total", ctypes.c_float),
                 ("sweep_launches", ctypes.c_int32), ("total_launches", ctypes.c_int32),
-                ("state_bytes", ctypes.c_int32), ("fast_path", ctypes.c_int32)]
+                ("state_bytes", ctypes.c_int32), ("fast_path", ctypes.c_int32),
+                ("pair_levels", ctypes.c_int32)]
 
 
 class PPError(RuntimeError):

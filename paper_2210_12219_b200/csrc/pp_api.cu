@@ -32,16 +32,34 @@ struct pp_problem {
     int32_t *h_err = &h_err_buf;
     Dev d{};
     bool solved = false;
-    int sweep_launches = 0, total_launches = 0, fast_used = 0;
+    int sweep_launches = 0, total_launches = 0, fast_used = 0, pair_levels = 0;
     int force_generic = -1;
+    bool mask_swaps = false;            // the mask list pairs up (see mask_list)
+    std::vector<signed char> pair_lvl;  // per level: 1 = two-mask kernel, 0 = one-mask, -1 = not decided yet
 };
 
 namespace {
 
-// Masks sorted by (popcount, value) depend on k only: built once per k and process, then copied.
+// Mask lists depend on k only: built once per k and process, then copied.  Level j (popcount j)
+// lists its masks in revolving-door order: A(n, j) = A(n-1, j), then the masks of A(n-1, j-1) in
+// reverse, each with node n-1 added.  Neighbours in that list differ by one node swapped for
+// another, which is what the two-mask sweep kernel pairs up.
 struct MaskList {
     std::vector<uint32_t> masks, level_off;
+    bool swaps = true;  // every two neighbours of a level differ by exactly one swap (checked)
 };
+void revolving_door(int n, int j, uint32_t add, bool reversed, std::vector<uint32_t> &out)
+{
+    if (j == 0) { out.push_back(add); return; }
+    if (j == n) { out.push_back(add | ((1u << n) - 1u)); return; }
+    if (!reversed) {
+        revolving_door(n - 1, j, add, false, out);
+        revolving_door(n - 1, j - 1, add | (1u << (n - 1)), true, out);
+    } else {
+        revolving_door(n - 1, j - 1, add | (1u << (n - 1)), false, out);
+        revolving_door(n - 1, j, add, true, out);
+    }
+}
 const MaskList &mask_list(int k)
 {
     static std::mutex mu;
@@ -52,11 +70,15 @@ const MaskList &mask_list(int k)
     MaskList ml;
     const uint32_t nm = 1u << k;
     ml.level_off.assign(k + 2, 0);
-    for (uint32_t S = 1; S < nm; ++S) ml.level_off[__builtin_popcount(S) + 1]++;
-    for (int j = 1; j <= k + 1; ++j) ml.level_off[j] += ml.level_off[j - 1];
-    ml.masks.assign(nm - 1, 0);
-    std::vector<uint32_t> at(ml.level_off.begin(), ml.level_off.end());
-    for (uint32_t S = 1; S < nm; ++S) ml.masks[at[__builtin_popcount(S)]++] = S;
+    ml.masks.reserve(nm - 1);
+    for (int j = 1; j <= k; ++j) {
+        ml.level_off[j] = (uint32_t)ml.masks.size();
+        revolving_door(k, j, 0u, false, ml.masks);
+        for (size_t i = ml.level_off[j] + 1; i < ml.masks.size(); ++i)
+            if (__builtin_popcount(ml.masks[i] ^ ml.masks[i - 1]) != 2) ml.swaps = false;
+    }
+    ml.level_off[k + 1] = (uint32_t)ml.masks.size();
+    ml.level_off[0] = 0;
     return cache.emplace(k, std::move(ml)).first->second;
 }
 
@@ -177,18 +199,25 @@ pp_status queue_solve(pp_problem *p, pp_solution *sol_dev)
     PP_CUDA(launch_rank_build(d, s, &launches));
     PP_CUDA(cudaEventRecord(p->ev[1], s));
     PP_CUDA(launch_base(d, s));
-    int sweep = 1;
+    int sweep = 1, pairs = 0;
     const int top = std::min(p->k, p->L);
     bool fast = fast_sweep_supported(d);
     if (p->force_generic == 1) fast = false;
     for (int level = 2; level <= top; ++level) {
-        PP_CUDA(fast ? launch_sweep_fast(d, level, s) : launch_sweep_generic(d, level, s));
+        if (fast && p->force_generic != 2) {
+            if (p->pair_lvl[level] < 0) p->pair_lvl[level] = pair_sweep_takes(d, level, p->force_generic == 3) ? 1 : 0;
+            PP_CUDA(p->pair_lvl[level] ? launch_sweep_pair(d, level, s) : launch_sweep_fast(d, level, s));
+            pairs += p->pair_lvl[level];
+        } else {
+            PP_CUDA(fast ? launch_sweep_fast(d, level, s) : launch_sweep_generic(d, level, s));
+        }
         ++sweep;
     }
     PP_CUDA(cudaEventRecord(p->ev[2], s));
     PP_CUDA(launch_finalize(d, sol_dev, s));
     PP_CUDA(cudaEventRecord(p->ev[3], s));
     p->sweep_launches = sweep;
+    p->pair_levels = pairs;
     p->total_launches = launches + sweep + 1;
     p->fast_used = fast ? (p->d.fast_meta ? 1 : 2) : 0;
     p->solved = true;
@@ -267,6 +296,8 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         const MaskList &ml = mask_list(k);
         p->masks = ml.masks;
         p->level_off = ml.level_off;
+        p->mask_swaps = ml.swaps;
+        p->pair_lvl.assign(k + 2, -1);
     } catch (const std::bad_alloc &) {
         delete p;
         return PP_ERR_NOMEM;
@@ -279,6 +310,16 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         fmeta.resize(fast_meta_bytes());
         has_fast = p->elem == 2 && p->Lpad <= 240 && k >= 2 &&
                    fast_meta_build(L, k, p->lo.data(), fmeta.data());
+    } catch (const std::bad_alloc &) {
+        delete p;
+        return PP_ERR_NOMEM;
+    }
+    std::vector<unsigned char> pmeta;
+    try {
+        if (has_fast && p->mask_swaps) {
+            pmeta.resize(pair_meta_bytes());
+            if (!pair_meta_build(L, k, p->lo.data(), pmeta.data())) pmeta.clear();
+        }
     } catch (const std::bad_alloc &) {
         delete p;
         return PP_ERR_NOMEM;
@@ -304,7 +345,8 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         {nullptr, 8, 0} /* best */,                    {nullptr, 4, 0} /* err */,
         {nullptr, sizeof(pp_solution), 0} /* solution */,
         {fmeta.data(), fmeta.size(), 0},
-        {gmeta.data(), gmeta.size() * 4, 0}};
+        {gmeta.data(), gmeta.size() * 4, 0},
+        {pmeta.data(), pmeta.size(), 0}};
     size_t total = 0;
     for (auto &q : parts) { q.off = total; total = align_up(total + q.bytes, 256); }
     // one staging buffer, one copy: the parts are small and a copy per part costs more than the bytes
@@ -342,6 +384,7 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     p->d_sol = reinterpret_cast<pp_solution *>(b + parts[11].off);
     d.fast_meta = has_fast ? b + parts[12].off : nullptr;
     d.gen_meta = gmeta.empty() ? nullptr : reinterpret_cast<uint32_t *>(b + parts[13].off);
+    d.pair_meta = pmeta.empty() ? nullptr : b + parts[14].off;
     *out = p;
     return PP_OK;
 }
@@ -389,8 +432,9 @@ pp_status pp_problem_set_workspace(pp_problem *p, void *device_buffer, uint64_t 
 
 pp_status pp_problem_force_generic(pp_problem *p, int32_t mode)
 {
-    if (!p || mode < -1 || mode > 1) return PP_ERR_ARG;
+    if (!p || mode < -1 || mode > 3) return PP_ERR_ARG;
     p->force_generic = mode;
+    p->pair_lvl.assign(p->k + 2, -1);
     return PP_OK;
 }
 
@@ -430,6 +474,7 @@ pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out)
     out->total_launches = p->total_launches;
     out->state_bytes = p->elem;
     out->fast_path = p->fast_used;
+    out->pair_levels = p->pair_levels;
     return PP_OK;
 }
 

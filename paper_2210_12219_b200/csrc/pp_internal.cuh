@@ -23,7 +23,8 @@ struct Dev {
                                //        (= c' when even the single layer c' does not fit)
     const int16_t *pair_u;     // [k*k] index into ubw of the pair's bandwidth, -1 if unusable
     const uint32_t *ubw;       // [U] distinct bandwidth values
-    const uint32_t *masks;     // [2^k - 1] all non-empty masks sorted by (popcount, value)
+    const uint32_t *masks;     // [2^k - 1] all non-empty masks by popcount, each level in revolving-door
+                               //        order (neighbours differ by one node swapped for another)
     const uint32_t *level_off; // [k+2] masks of popcount j are masks[level_off[j] .. level_off[j+1])
     int16_t *pos;              // [L] position of layer c in the ascending order of bits
     int16_t *order;            // [L] layer at each position
@@ -36,6 +37,7 @@ struct Dev {
     int32_t *err;              // device error word (0 = fine)
     const void *fast_meta;     // per-node window constants of the register-tiled sweep, or null
     const uint32_t *gen_meta;  // [k*Lpad] per-(node, position) lookup words of its general-window step, or null
+    const void *pair_meta;     // per-node window constants of the two-mask sweep, or null
 };
 
 static constexpr unsigned long long kNoBest = ~0ull;
@@ -55,6 +57,10 @@ bool fast_meta_build(int L, int k, const int16_t *lo, void *out);
 void gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out);
 bool fast_sweep_supported(const Dev &d);
 cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s);
+size_t pair_meta_bytes();
+bool pair_meta_build(int L, int k, const int16_t *lo, void *out);
+bool pair_sweep_takes(const Dev &d, int level, bool whenever_possible);
+cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s);
 cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s);
 cudaError_t launch_eval(const Dev &d, int64_t B, const uint8_t *nseg, const int32_t *ends,
                         const int32_t *nodes, double *beta, uint8_t *status, cudaStream_t s);

@@ -24,6 +24,7 @@
 // step of the current one, so that independent loads fill the latencies of the dependent chain.
 // Row (S + w, w) has the single source mask S, so no two warps ever write the same row.
 #include "pp_internal.cuh"
+#include "pp_sweep_ops.cuh"
 
 namespace pp {
 
@@ -42,8 +43,6 @@ namespace {
 // for more resident warps (the register file holds 64K registers per SM).
 constexpr int kMaxFastThreads = 768;
 __host__ __device__ constexpr int fast_threads(int nv, bool gen) { return gen ? 512 : (nv <= PP_NV768 ? 768 : (nv <= PP_NV640 ? 640 : 512)); }
-constexpr uint32_t kInf2 = 0xFFFFFFFFu;
-
 // Per-target-node constants of the window step (W = 8q + r), built on the host.
 // A shuffle distance of 31 means "nothing": rows occupy at most 30 lanes, so no lane that holds
 // data finds a source and +inf (or the untouched accumulator) results.
@@ -60,35 +59,6 @@ struct alignas(16) WMeta {
 struct FastMeta {
     WMeta w[PP_MAX_K];
 };
-
-__device__ __forceinline__ uint32_t vmin2(uint32_t a, uint32_t b)
-{
-    uint32_t r;
-    asm("min.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
-__device__ __forceinline__ uint32_t vmax2(uint32_t a, uint32_t b)
-{
-    uint32_t r;
-    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
-// three-input packed minimum: one issue slot where two two-input minima would take two
-__device__ __forceinline__ uint32_t vmin3(uint32_t a, uint32_t b, uint32_t c) { return __vimin3_u16x2(a, b, c); }
-// shuffle up by delta (<= 31) lanes, +inf shifted in from below lane 0
-__device__ __forceinline__ uint32_t shfl_up_inf(uint32_t x, int delta)
-{
-    uint32_t y;
-    asm volatile("{ .reg .pred p; shfl.sync.up.b32 %0|p, %1, %2, 0, 0xffffffff; @!p mov.b32 %0, 0xffffffff; }"
-                 : "=r"(y) : "r"(x), "r"(delta));
-    return y;
-}
-// acc = min(acc, x shifted up by delta lanes); lanes without a source keep acc
-__device__ __forceinline__ void min_shfl_up(uint32_t &acc, uint32_t x, int delta)
-{
-    asm volatile("{ .reg .pred p; .reg .b32 t; shfl.sync.up.b32 t|p, %1, %2, 0, 0xffffffff; @p min.u16x2 %0, %0, t; }"
-                 : "+r"(acc) : "r"(x), "r"(delta));
-}
 
 constexpr int NT = PP_FAST_NT;  // target nodes processed together
 constexpr int kStripElems = 256 + 256 + 168;  // per-warp strips of the general window step (u16)
@@ -246,19 +216,6 @@ __device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) o[j] = val[2 * j] | (val[2 * j + 1] << 16);
-}
-
-// Slow path of the final-state bookkeeping, kept out of line so that the common case is a
-// compare and a branch.
-__device__ __noinline__ unsigned long long offer_final(unsigned long long *best, unsigned long long best_seen,
-                                                       uint32_t val, int level, uint32_t S2, int w)
-{
-    const unsigned long long key = pack_best(val, level, S2, w);
-    if (key < best_seen) {
-        atomicMin(best, key);
-        return key;
-    }
-    return best_seen;
 }
 
 template <int NV, bool GEN>

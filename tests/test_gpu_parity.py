@@ -120,7 +120,7 @@ def test_register_tiled_sweep_on_uniform_memory_chains():
     # chains of identical layers take the register-tiled sweep kernel; rows of every raggedness
     # (L not a multiple of 8 or 16, one lane up to all 32 lanes), every window remainder r = W % 8
     # and block count q = W // 8, windows wider than the chain, ties and dead links
-    n_fast = 0
+    n_fast = n_pair = 0
     seed = 0
     for L, k, wmin, wmax, n in ((9, 3, 8, 9, 6), (12, 5, 8, 10, 10), (17, 6, 8, 13, 10), (31, 4, 8, 16, 12),
                                 (40, 6, 8, 30, 10), (64, 5, 9, 40, 8), (100, 7, 8, 60, 6),
@@ -142,10 +142,22 @@ def test_register_tiled_sweep_on_uniform_memory_chains():
                             if S >> v & 1 and bin(S).count("1") <= L:
                                 assert np.array_equal(p.debug_read_state_row(S, v), want.table[S, v]), \
                                     (inst.name, S, v)
+                # the kernel that takes two source masks per warp, forced onto every level it can run
+                p.force_generic(3)
+                assert_same(inst, p.solve_exact(), want)
+                prof = p.last_solve_profile()
+                assert prof.fast_path == 1 and prof.pair_levels == max(0, min(k, L, 13) - 2), inst.name
+                n_pair += prof.pair_levels > 0
+                if want.table is not None:
+                    for S in range(1, 1 << k):
+                        for v in range(k):
+                            if S >> v & 1 and bin(S).count("1") <= L:
+                                assert np.array_equal(p.debug_read_state_row(S, v), want.table[S, v]), \
+                                    (inst.name, S, v, "two-mask kernel")
                 p.force_generic(1)
                 assert_same(inst, p.solve_exact(), want)
                 assert p.last_solve_profile().fast_path == 0
-    assert n_fast >= 80
+    assert n_fast >= 80 and n_pair >= 70
     # a node whose window is narrower than 8 layers takes the general-window variant
     inst = W.uniform_memory_small(81000, 30, 4, 3, 7)
     with pp.Problem.from_instance(inst) as p:
@@ -215,7 +227,7 @@ def test_large_config_full_size():
         assert_same(inst, got, want)
         assert oracle.eval_plan(inst, *got.plan()) == (got.beta_ms, 0)
         prof = p.last_solve_profile()
-        assert prof.state_bytes == 2 and prof.fast_path == 1
+        assert prof.state_bytes == 2 and prof.fast_path == 1 and prof.pair_levels >= 6
         rng = np.random.default_rng(9)
         for size in (1, 2, 3, 5, 7, 8):
             nodes = sorted(int(x) for x in rng.choice(inst.k, size=size, replace=False))
