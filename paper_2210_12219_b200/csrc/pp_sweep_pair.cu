@@ -16,8 +16,14 @@
 // Window decomposition as in the one-mask kernel, blocks of 8 = lanes, W = 8q + r:
 //   out[8l + j] = min( suffix of block l - q (j >= r) or l - q - 1 (j < r) from offset (j - r) mod 8,
 //                      q - 1 (resp. q) whole blocks in between, prefix of the own block ).
-// The suffix minima travel through a per-warp strip of 8 planes (one per offset) x 64 words
-// (32 words of +inf, then one word per lane), so that all accesses are conflict-free.
+// The suffix minima travel through a per-warp strip of 16 slots x 64 words.  Slots 8..15 hold the
+// in-lane suffix minima sfx_i (i = slot - 8) of lane x at word 31 + x; slots 1..7 hold
+// E_i = min(sfx_i, block minimum of the next lane) (i = slot), i.e. the suffix run on through one
+// more block, at word 32 + x (word 31, the lane before lane 0, holds the minimum of block 0: its own
+// suffixes are empty).  Output j then reads slot j - r + 8 at word 31 + l - q whatever j is:
+// for j >= r that is sfx_{j-r} of lane l - q, for j < r it is E_{8+j-r} of lane l - q - 1, and in both
+// cases the q - 1 whole blocks l-q+1 .. l-1 remain.  The words below 31 stay +inf.  Addresses
+// differ by constants, nothing is selected, the code is branch-free, no access has a bank conflict.
 #include "pp_internal.cuh"
 #include "pp_sweep_ops.cuh"
 
@@ -32,46 +38,102 @@ namespace {
 #define PP_PAIR_MIN_NV 3
 #endif
 #ifndef PP_PAIR_MAX_NV
-#define PP_PAIR_MAX_NV 11
+#define PP_PAIR_MAX_NV 12
 #endif
 // threads per block by the number of source rows per mask (2 * NV rows of 4 registers per lane)
-__host__ __device__ constexpr int pair_threads(int nv) { return nv <= PP_PAIR_T512 ? 512 : 384; }
-constexpr int kMaxPairWarps = 16;
-constexpr int kPlane = 64;              // words per strip plane
-constexpr int kStripWords = 8 * kPlane;  // per warp
+#ifndef PP_PAIR_T384
+#define PP_PAIR_T384 11
+#endif
+#ifndef PP_PAIR_PIPE
+#define PP_PAIR_PIPE 1
+#endif
+#ifndef PP_PAIR_STAGED
+#define PP_PAIR_STAGED 1
+#endif
+#ifndef PP_PAIR_FILL
+#define PP_PAIR_FILL 2
+#endif
+__host__ __device__ constexpr int pair_threads(int nv) { return nv <= PP_PAIR_T512 ? 512 : (nv <= PP_PAIR_T384 ? 384 : 256); }
+constexpr int kPlane = 64;               // words per strip slot
+constexpr int kStripWords = 16 * kPlane;  // per warp
 
 // Per-target-node constants (W = 8q + r), built on the host.  A shuffle distance of 31 means
 // "nothing": rows occupy at most 30 lanes.
 struct alignas(16) PMeta {
     int dd[4];   // doubling distances 1, 2, 4, 8 for the first s steps (2^s <= q - 1 < 2^(s+1)), then 31
     int d1, d2;  // T1 = min(D << d1, D << d2): 1 and q - 2^s, or 31 when q = 1
-    int dq;      // q: the one more block that offsets below r need
-    int qr;      // q | r << 8
+    int soff;    // (8 - r) * 64 - q: word offset from a lane's word of slot 0 to what its output 0 reads
+    int rowoff;  // ((k << w) + w) * Lpad / 8: row (S + w, w) in 16-byte pieces after row (S, 0)
+    int rwoff;   // w * k * Lpad: element offset of the node's block of the rank table
+    int pad[3];
 };
 
 struct PairMeta {
     PMeta w[PP_MAX_K];
 };
 
-// Last combine for W mod 8 == R.  sp = this lane's word of plane 0, moved back by q lanes.
-template <int R>
-__device__ __forceinline__ void pair_combine(const uint32_t *sp, const uint32_t (&o)[8], uint32_t T1, uint32_t T2,
-                                             uint32_t (&out)[8])
+// 16-byte store under a predicate, no branch
+__device__ __forceinline__ void st_if(uint4 *ptr, const uint4 &v, bool on)
 {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint32_t f = sp[((j - R) & 7) * kPlane - (j < R ? 1 : 0)];
-        const uint32_t mid = j < R ? T2 : T1;
-        out[j] = j == 0 ? vmin2(f, mid) : vmin3(o[j], f, mid);
-    }
+    asm volatile("{ .reg .pred p; setp.ne.u32 p, %5, 0; @p st.global.v4.u32 [%0], {%1, %2, %3, %4}; }" ::"l"(ptr),
+                 "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"((uint32_t)on)
+                 : "memory");
 }
 
-template <int NV>
+__device__ __forceinline__ uint4 max4(const uint4 &a, const uint4 &b)
+{
+    return make_uint4(vmax2(a.x, b.x), vmax2(a.y, b.y), vmax2(a.z, b.z), vmax2(a.w, b.w));
+}
+__device__ __forceinline__ void set4(uint32_t (&r)[4], const uint4 &a)
+{
+    r[0] = a.x; r[1] = a.y; r[2] = a.z; r[3] = a.w;
+}
+__device__ __forceinline__ void min4(uint32_t (&r)[4], const uint4 &a)
+{
+    r[0] = vmin2(r[0], a.x); r[1] = vmin2(r[1], a.y); r[2] = vmin2(r[2], a.z); r[3] = vmin2(r[3], a.w);
+}
+__device__ __forceinline__ void min4(uint32_t (&r)[4], const uint4 &a, const uint4 &b)
+{
+    r[0] = vmin3(r[0], a.x, b.x); r[1] = vmin3(r[1], a.y, b.y);
+    r[2] = vmin3(r[2], a.z, b.z); r[3] = vmin3(r[3], a.w, b.w);
+}
+__device__ __forceinline__ void setmin4(uint32_t (&r)[4], const uint4 &a, const uint4 &b)
+{
+    r[0] = vmin2(a.x, b.x); r[1] = vmin2(a.y, b.y); r[2] = vmin2(a.z, b.z); r[3] = vmin2(a.w, b.w);
+}
+
+// (t + 1, t + 1) for the best final rank t seen so far: a packed value x holds a rank <= t in
+// one of its halves exactly when max(x, that) != x
+__device__ __forceinline__ uint32_t offer_threshold(unsigned long long best_seen)
+{
+    const unsigned long long r = best_seen >> 30;
+    const uint32_t t = (r > 0xFFFEull ? 0xFFFEu : (uint32_t)r) + 1u;
+    return t | (t << 16);
+}
+// Slow path of the final-state bookkeeping for the two rows of a pair (x = their last elements).
+__device__ __noinline__ unsigned long long offer_pair(unsigned long long *best, unsigned long long best_seen,
+                                                      uint32_t x, bool ok1, bool ok2, int level, uint32_t A,
+                                                      uint32_t B, int w)
+{
+    const uint32_t v1 = x & 0xFFFFu, v2 = x >> 16;
+    if (ok1 && v1 != 0xFFFFu) best_seen = offer_final(best, best_seen, v1, level, A | (1u << w), w);
+    if (ok2 && v2 != 0xFFFFu) best_seen = offer_final(best, best_seen, v2, level, B | (1u << w), w);
+    return best_seen;
+}
+
+template <int M>
+struct Mode {
+    static constexpr int value = M;
+};
+
+// L8: the chain length is a multiple of 8, so the last element of a row is a lane's last position.
+template <int NV, bool L8>
 __global__ void __launch_bounds__(pair_threads(NV), 1)
 k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
 {
     constexpr int kThreads = pair_threads(NV);
     constexpr int kWarps = kThreads / 32;
+    constexpr int NC = NV - 1;  // sources common to both masks
     // the next level's prologue (rank table -> shared memory) may overlap this level's tail
     asm volatile("griddepcontrol.launch_dependents;");
     extern __shared__ uint4 smem4[];
@@ -97,20 +159,27 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const bool active = lane < (Lpad >> 3);
-    uint32_t *const sl = strips + warp * kStripWords + 32 + lane;  // this lane's word of plane 0
-    const uint16_t *table = reinterpret_cast<const uint16_t *>(d.table);
-    uint16_t *table_w = reinterpret_cast<uint16_t *>(d.table);
+    const int l8 = Lpad >> 3;  // 16-byte pieces per row
+    const bool active = lane < l8;
+    uint32_t *const sl = strips + warp * kStripWords + 31 + lane;  // this lane's word of slot 0
+    uint32_t *const se = strips + warp * kStripWords + (lane == 31 ? 31 : 32 + lane);  // ... of the E slots
+    const int next_lane = (lane + 1) & 31;
+    // rows are addressed in 16-byte pieces from the start of the table (fits 32 bits at every size)
+    const uint4 *const table = reinterpret_cast<const uint4 *>(d.table);
+    uint4 *const table_w = reinterpret_cast<uint4 *>(d.table);
     const uint32_t first = d.level_off[level - 1];
     const uint32_t nmask = d.level_off[level] - first;
     const uint32_t npair = (nmask + 1) >> 1;
     const uint32_t full = (1u << k) - 1u;
-    const int last_lane = (L - 1) >> 3, last_j = (L - 1) & 7;
+    const bool is_last = lane == ((L - 1) >> 3);
+    const int last_j = (L - 1) & 7;
     const uint32_t stride = gridDim.x * kWarps;
     const uint4 inf4 = make_uint4(kInf2, kInf2, kInf2, kInf2);
+    const uint32_t mask_rows = (uint32_t)(k * l8);  // pieces per mask
 
     uint32_t pi = blockIdx.x * kWarps + warp;
-    // sources: voff[0 .. NV-2] the common nodes T, voff[NV-1] = a (S1 only), voffb = b (S2 only)
+    // sources: voff[0 .. NV-2] the common nodes T, voff[NV-1] = a (S1 only), voffb = b (S2 only);
+    // offsets in elements from the start of a rank-table block or a mask's rows
     int voff[NV];
     int voffb = 0;
     uint4 dp1[NV], dp2[NV];
@@ -120,90 +189,119 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
         A = d.masks[first + 2 * p];
         B = (2 * p + 1 < nmask) ? d.masks[first + 2 * p + 1] : A;
     };
-    auto load_rows = [&](uint32_t A, uint32_t B) {
+    // Rows of the pair (A, B).  MODE 0: bring both masks' rows into L2 (one 16-byte piece per lane
+    // covers a row); 1: load the rows of A into dp1; 2: load the rows of B into dp2 and take over
+    // the pair's source offsets.
+    auto touch_rows = [&](uint32_t A, uint32_t B, auto mode) {
+        constexpr int MODE = decltype(mode)::value;
         uint32_t abit = A & ~B;
         if (!abit) abit = A & (0u - A);  // a mask without partner runs as a pair with itself
         const uint32_t T = A & ~abit;
         const uint32_t bbit = B & ~T;
+        const uint4 *s1 = table + A * mask_rows + lane;
+        const uint4 *s2 = table + B * mask_rows + lane;
         uint32_t rem = T;
+        int off[NV];
 #pragma unroll
-        for (int vi = 0; vi < NV - 1; ++vi) {
-            voff[vi] = (__ffs(rem) - 1) * Lpad;
+        for (int vi = 0; vi < NC; ++vi) {
+            off[vi] = (__ffs(rem) - 1) * l8;
             rem &= rem - 1;
         }
-        voff[NV - 1] = (__ffs(abit) - 1) * Lpad;
-        voffb = (__ffs(bbit) - 1) * Lpad;
-        const uint16_t *s1 = table + (size_t)A * k * Lpad + 8 * lane;
-        const uint16_t *s2 = table + (size_t)B * k * Lpad + 8 * lane;
+        off[NV - 1] = (__ffs(abit) - 1) * l8;
+        const int offb = (__ffs(bbit) - 1) * l8;
+        if (MODE == 1) {
 #pragma unroll
-        for (int vi = 0; vi < NV; ++vi) {
-            dp1[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(s1 + voff[vi])) : inf4;
-            dp2[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(s2 + (vi == NV - 1 ? voffb : voff[vi]))) : inf4;
+            for (int vi = 0; vi < NV; ++vi) dp1[vi] = active ? __ldg(s1 + off[vi]) : inf4;
+        } else if (MODE == 2) {
+#pragma unroll
+            for (int vi = 0; vi < NV; ++vi) {
+                voff[vi] = off[vi] * 8;
+                dp2[vi] = active ? __ldg(s2 + (vi == NV - 1 ? offb : off[vi])) : inf4;
+            }
+            voffb = offb * 8;
+            best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
+        } else if (active) {
+#pragma unroll
+            for (int vi = 0; vi < NV; ++vi) {
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(s1 + off[vi]));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(s2 + (vi == NV - 1 ? offb : off[vi])));
+            }
         }
-        best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
     };
     if (pi < npair) {
         fetch_masks(pi, S1, S2);
-        load_rows(S1, S2);
+        touch_rows(S1, S2, Mode<1>{});
+        touch_rows(S1, S2, Mode<2>{});
     }
     best_seen = best_next;
+    uint32_t thr2 = offer_threshold(best_seen);
     while (pi < npair) {
         const uint32_t pi_next = pi + stride;
+        const bool more = pi_next < npair;
         uint32_t S1n = 0, S2n = 0;
-        if (pi_next < npair) fetch_masks(pi_next, S1n, S2n);
+        if (more) fetch_masks(pi_next, S1n, S2n);
         const uint32_t A = S1, B = S2;
-        const bool has2 = A != B;
-        uint32_t wrem = full & ~(A & B);  // every node outside the common part
-        uint16_t *const base1 = table_w + (size_t)A * k * Lpad + 8 * lane;
-        uint16_t *const base2 = table_w + (size_t)B * k * Lpad + 8 * lane;
-        const int ntargets = __popc(wrem);
+        const uint32_t base1 = A * mask_rows + lane, base2 = B * mask_rows + lane;
 
         // 1. both rows relaxed over their sources, two sources per three-input minimum
         auto relax = [&](int w, uint32_t (&r1)[4], uint32_t (&r2)[4]) {
-            const uint16_t *rw = rank_s + w * k * Lpad + 8 * lane;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) r1[j] = r2[j] = kInf2;
-#pragma unroll
-            for (int vi = 0; vi + 1 < NV - 1; vi += 2) {
-                const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[vi]);
-                const uint4 h = *reinterpret_cast<const uint4 *>(rw + voff[vi + 1]);
-                r1[0] = vmin3(r1[0], vmax2(dp1[vi].x, g.x), vmax2(dp1[vi + 1].x, h.x));
-                r1[1] = vmin3(r1[1], vmax2(dp1[vi].y, g.y), vmax2(dp1[vi + 1].y, h.y));
-                r1[2] = vmin3(r1[2], vmax2(dp1[vi].z, g.z), vmax2(dp1[vi + 1].z, h.z));
-                r1[3] = vmin3(r1[3], vmax2(dp1[vi].w, g.w), vmax2(dp1[vi + 1].w, h.w));
-                r2[0] = vmin3(r2[0], vmax2(dp2[vi].x, g.x), vmax2(dp2[vi + 1].x, h.x));
-                r2[1] = vmin3(r2[1], vmax2(dp2[vi].y, g.y), vmax2(dp2[vi + 1].y, h.y));
-                r2[2] = vmin3(r2[2], vmax2(dp2[vi].z, g.z), vmax2(dp2[vi + 1].z, h.z));
-                r2[3] = vmin3(r2[3], vmax2(dp2[vi].w, g.w), vmax2(dp2[vi + 1].w, h.w));
-            }
+            const uint16_t *rw = rank_s + wm[w].rwoff + 8 * lane;
             const uint4 ga = *reinterpret_cast<const uint4 *>(rw + voff[NV - 1]);
             const uint4 gb = *reinterpret_cast<const uint4 *>(rw + voffb);
-            if ((NV - 1) & 1) {  // the last common source shares a minimum with a (resp. b)
-                const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[NV - 2 >= 0 ? NV - 2 : 0]);
-                constexpr int c = NV - 2 >= 0 ? NV - 2 : 0;
-                r1[0] = vmin3(r1[0], vmax2(dp1[c].x, g.x), vmax2(dp1[NV - 1].x, ga.x));
-                r1[1] = vmin3(r1[1], vmax2(dp1[c].y, g.y), vmax2(dp1[NV - 1].y, ga.y));
-                r1[2] = vmin3(r1[2], vmax2(dp1[c].z, g.z), vmax2(dp1[NV - 1].z, ga.z));
-                r1[3] = vmin3(r1[3], vmax2(dp1[c].w, g.w), vmax2(dp1[NV - 1].w, ga.w));
-                r2[0] = vmin3(r2[0], vmax2(dp2[c].x, g.x), vmax2(dp2[NV - 1].x, gb.x));
-                r2[1] = vmin3(r2[1], vmax2(dp2[c].y, g.y), vmax2(dp2[NV - 1].y, gb.y));
-                r2[2] = vmin3(r2[2], vmax2(dp2[c].z, g.z), vmax2(dp2[NV - 1].z, gb.z));
-                r2[3] = vmin3(r2[3], vmax2(dp2[c].w, g.w), vmax2(dp2[NV - 1].w, gb.w));
+            if (NC >= 2) {
+                const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[0]);
+                const uint4 h = *reinterpret_cast<const uint4 *>(rw + voff[NC >= 2 ? 1 : 0]);
+                setmin4(r1, max4(dp1[0], g), max4(dp1[NC >= 2 ? 1 : 0], h));
+                setmin4(r2, max4(dp2[0], g), max4(dp2[NC >= 2 ? 1 : 0], h));
+#pragma unroll
+                for (int vi = 2; vi + 1 < NC; vi += 2) {
+                    const uint4 g2 = *reinterpret_cast<const uint4 *>(rw + voff[vi]);
+                    const uint4 h2 = *reinterpret_cast<const uint4 *>(rw + voff[vi + 1]);
+                    min4(r1, max4(dp1[vi], g2), max4(dp1[vi + 1], h2));
+                    min4(r2, max4(dp2[vi], g2), max4(dp2[vi + 1], h2));
+                }
+                if (NC & 1) {  // the last common source shares a minimum with a (resp. b)
+                    const uint4 g3 = *reinterpret_cast<const uint4 *>(rw + voff[NC - 1]);
+                    min4(r1, max4(dp1[NC - 1], g3), max4(dp1[NV - 1], ga));
+                    min4(r2, max4(dp2[NC - 1], g3), max4(dp2[NV - 1], gb));
+                } else {
+                    min4(r1, max4(dp1[NV - 1], ga));
+                    min4(r2, max4(dp2[NV - 1], gb));
+                }
+            } else if (NC == 1) {
+                const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[0]);
+                setmin4(r1, max4(dp1[0], g), max4(dp1[NV - 1], ga));
+                setmin4(r2, max4(dp2[0], g), max4(dp2[NV - 1], gb));
             } else {
-                r1[0] = vmin2(r1[0], vmax2(dp1[NV - 1].x, ga.x));
-                r1[1] = vmin2(r1[1], vmax2(dp1[NV - 1].y, ga.y));
-                r1[2] = vmin2(r1[2], vmax2(dp1[NV - 1].z, ga.z));
-                r1[3] = vmin2(r1[3], vmax2(dp1[NV - 1].w, ga.w));
-                r2[0] = vmin2(r2[0], vmax2(dp2[NV - 1].x, gb.x));
-                r2[1] = vmin2(r2[1], vmax2(dp2[NV - 1].y, gb.y));
-                r2[2] = vmin2(r2[2], vmax2(dp2[NV - 1].z, gb.z));
-                r2[3] = vmin2(r2[3], vmax2(dp2[NV - 1].w, gb.w));
+                set4(r1, max4(dp1[NV - 1], ga));
+                set4(r2, max4(dp2[NV - 1], gb));
+            }
+        };
+        // one row only (the target is a node of the other mask): sources T and `lastoff`
+        auto relax1 = [&](int w, const uint4 (&dp)[NV], int lastoff, uint32_t (&r)[4]) {
+            const uint16_t *rw = rank_s + wm[w].rwoff + 8 * lane;
+            const uint4 ga = *reinterpret_cast<const uint4 *>(rw + lastoff);
+            if (NC >= 1) {
+                const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[0]);
+                setmin4(r, max4(dp[0], g), max4(dp[NV - 1], ga));
+#pragma unroll
+                for (int vi = 1; vi + 1 < NC; vi += 2) {
+                    const uint4 g2 = *reinterpret_cast<const uint4 *>(rw + voff[vi]);
+                    const uint4 h2 = *reinterpret_cast<const uint4 *>(rw + voff[vi + 1]);
+                    min4(r, max4(dp[vi], g2), max4(dp[vi + 1], h2));
+                }
+                if (!(NC & 1)) {
+                    const uint4 g3 = *reinterpret_cast<const uint4 *>(rw + voff[NC >= 1 ? NC - 1 : 0]);
+                    min4(r, max4(dp[NC >= 1 ? NC - 1 : 0], g3));
+                }
+            } else {
+                set4(r, max4(dp[NV - 1], ga));
             }
         };
         // 2. + 3. window minimum of both rows, write them, offer their last elements as final states
-        auto finish = [&](int w, const uint32_t (&r1)[4], const uint32_t (&r2)[4]) {
+        auto finish = [&](int w, const uint32_t (&r1)[4], const uint32_t (&r2)[4], bool ok1, bool ok2) {
             const uint4 ma = *reinterpret_cast<const uint4 *>(&wm[w].dd[0]);
-            const uint4 mb = *reinterpret_cast<const uint4 *>(&wm[w].d1);
+            const uint4 mb = *reinterpret_cast<const uint4 *>(&wm[w].d1);  // d1, d2, soff, rowoff
             // p[j] = (g1[8l + j], g2[8l + j])
             uint32_t p[8];
 #pragma unroll
@@ -220,104 +318,120 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
             o[1] = p[0];
 #pragma unroll
             for (int j = 2; j < 8; ++j) o[j] = vmin2(o[j - 1], p[j - 1]);
+            // E_i = min(s_i, block minimum of the next lane).  Lane 31 never holds a piece of a row
+            // (its s_i are +inf); it takes the block minimum of lane 0 and writes the entries of the
+            // lane "before lane 0", whose suffixes are empty but whose next block is block 0.
+            const uint32_t Bn = __shfl_sync(0xFFFFFFFFu, s[0], next_lane);
             __syncwarp();  // the previous rows' readers are done
 #pragma unroll
-            for (int j = 0; j < 8; ++j) sl[j * kPlane] = s[j];
+            for (int j = 0; j < 8; ++j) sl[(8 + j) * kPlane] = s[j];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) se[j * kPlane] = vmin2(s[j], Bn);
             __syncwarp();
-            // whole blocks in between: D = min B[l-2^s+1 .. l], T1 = min B[l-q+1 .. l-1], T2 = min B[l-q .. l-1]
+            // whole blocks in between: D = min B[l-2^s+1 .. l], T1 = min B[l-q+1 .. l-1].
+            // A lane without a source lane gets its own value back from the shuffle, which leaves D alone.
             uint32_t D = s[0];
-            min_shfl_up(D, D, (int)ma.x);
-            min_shfl_up(D, D, (int)ma.y);
-            min_shfl_up(D, D, (int)ma.z);
-            min_shfl_up(D, D, (int)ma.w);
-            uint32_t T1 = shfl_up_inf(D, (int)mb.x);
-            min_shfl_up(T1, D, (int)mb.y);
-            uint32_t T2 = T1;
-            min_shfl_up(T2, s[0], (int)mb.z);
-            const int q = (int)(mb.w & 0xFFu), r = (int)(mb.w >> 8);
-            const uint32_t *sp = sl - q;
+            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.x));
+            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.y));
+            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.z));
+            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.w));
+            const uint32_t T1 = vmin2(shfl_up_inf(D, (int)mb.x), shfl_up_inf(D, (int)mb.y));
+            const uint32_t *sp = sl + (int)mb.z;
             uint32_t out[8];
-            switch (r) {
-                case 0: pair_combine<0>(sp, o, T1, T2, out); break;
-                case 1: pair_combine<1>(sp, o, T1, T2, out); break;
-                case 2: pair_combine<2>(sp, o, T1, T2, out); break;
-                case 3: pair_combine<3>(sp, o, T1, T2, out); break;
-                case 4: pair_combine<4>(sp, o, T1, T2, out); break;
-                case 5: pair_combine<5>(sp, o, T1, T2, out); break;
-                case 6: pair_combine<6>(sp, o, T1, T2, out); break;
-                default: pair_combine<7>(sp, o, T1, T2, out); break;
-            }
-            const bool ok1 = !((A >> w) & 1u), ok2 = has2 && !((B >> w) & 1u);
-            const uint32_t rowoff = (uint32_t)(((k << w) + w) * Lpad);  // row (S + w, w) from row (S, 0)
-            if (active && ok1)
-                *reinterpret_cast<uint4 *>(base1 + rowoff) =
-                    make_uint4(__byte_perm(out[0], out[1], 0x5410), __byte_perm(out[2], out[3], 0x5410),
-                               __byte_perm(out[4], out[5], 0x5410), __byte_perm(out[6], out[7], 0x5410));
-            if (active && ok2)
-                *reinterpret_cast<uint4 *>(base2 + rowoff) =
-                    make_uint4(__byte_perm(out[0], out[1], 0x7632), __byte_perm(out[2], out[3], 0x7632),
-                               __byte_perm(out[4], out[5], 0x7632), __byte_perm(out[6], out[7], 0x7632));
+            out[0] = vmin2(sp[0], T1);
+#pragma unroll
+            for (int j = 1; j < 8; ++j) out[j] = vmin3(o[j], sp[j * kPlane], T1);
+            // row (S + w, w) lies rowoff pieces after row (S, 0)
+            if (ok1)
+                st_if(table_w + (base1 + mb.w),
+                      make_uint4(__byte_perm(out[0], out[1], 0x5410), __byte_perm(out[2], out[3], 0x5410),
+                                 __byte_perm(out[4], out[5], 0x5410), __byte_perm(out[6], out[7], 0x5410)),
+                      active);
+            if (ok2)
+                st_if(table_w + (base2 + mb.w),
+                      make_uint4(__byte_perm(out[0], out[1], 0x7632), __byte_perm(out[2], out[3], 0x7632),
+                                 __byte_perm(out[4], out[5], 0x7632), __byte_perm(out[6], out[7], 0x7632)),
+                      active);
             // final states: ranks at or below the best rank seen so far are rare
-            uint32_t x;
-            switch (last_j) {
-                case 0: x = out[0]; break;
-                case 1: x = out[1]; break;
-                case 2: x = out[2]; break;
-                case 3: x = out[3]; break;
-                case 4: x = out[4]; break;
-                case 5: x = out[5]; break;
-                case 6: x = out[6]; break;
-                default: x = out[7]; break;
+            uint32_t x = out[7];
+            if (!L8) {
+                const uint32_t x01 = (last_j & 1) ? out[1] : out[0], x23 = (last_j & 1) ? out[3] : out[2];
+                const uint32_t x45 = (last_j & 1) ? out[5] : out[4], x67 = (last_j & 1) ? out[7] : out[6];
+                const uint32_t x03 = (last_j & 2) ? x23 : x01, x47 = (last_j & 2) ? x67 : x45;
+                x = (last_j & 4) ? x47 : x03;
             }
-            const uint32_t v1 = ok1 ? (x & 0xFFFFu) : 0xFFFFu, v2 = ok2 ? (x >> 16) : 0xFFFFu;
-            if (lane == last_lane && min(v1, v2) <= (uint32_t)(best_seen >> 30)) {
-                if (v1 != 0xFFFFu && v1 <= (uint32_t)(best_seen >> 30))
-                    best_seen = offer_final(d.best, best_seen, v1, level, A | (1u << w), w);
-                if (v2 != 0xFFFFu && v2 <= (uint32_t)(best_seen >> 30))
-                    best_seen = offer_final(d.best, best_seen, v2, level, B | (1u << w), w);
+            if (is_last && vmax2(x, thr2) != x) {
+                best_seen = offer_pair(d.best, best_seen, x, ok1, ok2, level, A, B, w);
+                thr2 = offer_threshold(best_seen);
             }
         };
-        // software pipeline over the target nodes: the relaxation of the next one (independent
-        // loads and min/max) sits in the same straight-line block as the window step of the
-        // current one (dependent shuffle chains)
-        int w = __ffs(wrem) - 1;
-        wrem &= wrem - 1;
         uint32_t r1[4], r2[4];
-        relax(w, r1, r2);
-        for (int it = 1; it < ntargets; ++it) {
-            const int wn = __ffs(wrem) - 1;
-            wrem &= wrem - 1;
-            uint32_t rn1[4], rn2[4];
-            relax(wn, rn1, rn2);
-            finish(w, r1, r2);
-            w = wn;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                r1[j] = rn1[j];
-                r2[j] = rn2[j];
+        if (A != B) {
+            const uint32_t abit = A & ~B, bbit = B & ~A;
+            // targets outside both masks: two rows each
+            uint32_t wrem = full & ~(A | B);
+            // rows of the next pair on their way into L2 while this pair is worked on
+            if (more) touch_rows(S1n, S2n, Mode<0>{});
+            while (wrem) {
+                const int w = __ffs(wrem) - 1;
+                wrem &= wrem - 1;
+                relax(w, r1, r2);
+                finish(w, r1, r2, true, true);
+            }
+            // target b takes the rows of S1 only, target a those of S2; once a mask's rows are dead
+            // the next pair's rows are fetched into their registers, behind the remaining window steps
+            {
+                const int w = __ffs(bbit) - 1;
+                relax1(w, dp1, voff[NV - 1], r1);
+#if PP_PAIR_STAGED
+                if (more) touch_rows(S1n, S2n, Mode<1>{});
+#endif
+                finish(w, r1, r1, true, false);
+            }
+            {
+                const int w = __ffs(abit) - 1;
+                relax1(w, dp2, voffb, r2);
+#if !PP_PAIR_STAGED
+                if (more) touch_rows(S1n, S2n, Mode<1>{});
+#endif
+                if (more) touch_rows(S1n, S2n, Mode<2>{});
+                finish(w, r2, r2, false, true);
+            }
+        } else {
+            // a mask without partner: one row per target
+            uint32_t wrem = full & ~A;
+            if (more) touch_rows(S1n, S2n, Mode<0>{});
+            while (wrem) {
+                const int w = __ffs(wrem) - 1;
+                wrem &= wrem - 1;
+                relax1(w, dp1, voff[NV - 1], r1);
+                finish(w, r1, r1, true, false);
+            }
+            if (more) {
+                touch_rows(S1n, S2n, Mode<1>{});
+                touch_rows(S1n, S2n, Mode<2>{});
             }
         }
-        // the source rows are dead once the last target is relaxed: fetch the next pair's rows
-        // now, so that their latency hides behind the last window step
-        if (pi_next < npair) load_rows(S1n, S2n);
-        finish(w, r1, r2);
-        best_seen = best_next < best_seen ? best_next : best_seen;
+        if (best_next < best_seen) {
+            best_seen = best_next;
+            thr2 = offer_threshold(best_seen);
+        }
         pi = pi_next;
         S1 = S1n;
         S2 = S2n;
     }
 }
 
-size_t pair_smem_bytes(const Dev &d)
+size_t pair_smem_bytes(const Dev &d, int nv)
 {
     return (((size_t)d.k * d.k * d.Lpad * 2 + 512 + 15) & ~(size_t)15) + sizeof(PMeta) * PP_MAX_K +
-           (size_t)kMaxPairWarps * kStripWords * 4;
+           (size_t)(pair_threads(nv) / 32) * kStripWords * 4;
 }
 
-template <int NV>
+template <int NV, bool L8>
 cudaError_t launch_pair_nv(const Dev &d, int level, unsigned grid, size_t sm, cudaStream_t s)
 {
-    cudaError_t e = cudaFuncSetAttribute(k_sweep_pair<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    cudaError_t e = cudaFuncSetAttribute(k_sweep_pair<NV, L8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -329,7 +443,7 @@ cudaError_t launch_pair_nv(const Dev &d, int level, unsigned grid, size_t sm, cu
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_sweep_pair<NV>, d, level, static_cast<const PairMeta *>(d.pair_meta));
+    return cudaLaunchKernelEx(&cfg, k_sweep_pair<NV, L8>, d, level, static_cast<const PairMeta *>(d.pair_meta));
 }
 
 }  // namespace
@@ -357,8 +471,10 @@ bool pair_meta_build(int L, int k, const int16_t *lo, void *out)
         for (int st = 0; st < 4; ++st) m.dd[st] = (n1 >= 1 && st < s) ? (1 << st) : 31;
         m.d1 = n1 >= 1 ? 1 : 31;
         m.d2 = n1 >= 1 ? 1 + n1 - (1 << s) : 31;
-        m.dq = q > 31 ? 31 : q;
-        m.qr = q | (r << 8);
+        m.soff = (8 - r) * kPlane - q;
+        m.rwoff = w * k * Lpad;
+        m.rowoff = ((k << w) + w) * (Lpad / 8);
+        m.pad[0] = m.pad[1] = m.pad[2] = 0;
     }
     return true;
 }
@@ -370,15 +486,15 @@ bool pair_sweep_takes(const Dev &d, int level, bool whenever_possible)
 {
     const int nv = level - 1;
     if (!d.pair_meta || d.elem != 2 || d.Lpad > 240) return false;
-    if (whenever_possible ? (nv < 2 || nv > 12) : (nv < PP_PAIR_MIN_NV || nv > PP_PAIR_MAX_NV)) return false;
+    if (whenever_possible ? (nv < 2 || nv > 13) : (nv < PP_PAIR_MIN_NV || nv > PP_PAIR_MAX_NV)) return false;
     int dev = 0, max_sm = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&max_sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
-    if (pair_smem_bytes(d) > (size_t)max_sm) return false;
+    if (pair_smem_bytes(d, nv) > (size_t)max_sm) return false;
     unsigned long long n = 1;  // source masks of popcount nv
     for (int i = 0; i < nv; ++i) n = n * (unsigned)(d.k - i) / (unsigned)(i + 1);
-    return whenever_possible || (n + 1) / 2 >= (unsigned long long)sms * (pair_threads(nv) / 32);
+    return whenever_possible || (n + 1) / 2 * PP_PAIR_FILL >= (unsigned long long)sms * (pair_threads(nv) / 32);
 }
 
 cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s)
@@ -392,12 +508,13 @@ cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s)
     const unsigned wpb = pair_threads(nv) / 32;
     unsigned long long blocks = ((n + 1) / 2 + wpb - 1) / wpb;
     const unsigned grid = blocks > (unsigned long long)sms ? (unsigned)sms : (unsigned)blocks;
-    const size_t sm = pair_smem_bytes(d);
+    const size_t sm = pair_smem_bytes(d, nv);
     switch (nv) {
 #define PP_CASE(N) \
-    case N: return launch_pair_nv<N>(d, level, grid, sm, s);
+    case N: return (d.L & 7) ? launch_pair_nv<N, false>(d, level, grid, sm, s) \
+                             : launch_pair_nv<N, true>(d, level, grid, sm, s);
         PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6) PP_CASE(7) PP_CASE(8)
-        PP_CASE(9) PP_CASE(10) PP_CASE(11) PP_CASE(12)
+        PP_CASE(9) PP_CASE(10) PP_CASE(11) PP_CASE(12) PP_CASE(13)
 #undef PP_CASE
     }
     return cudaErrorInvalidValue;

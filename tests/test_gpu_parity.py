@@ -146,7 +146,7 @@ def test_register_tiled_sweep_on_uniform_memory_chains():
                 p.force_generic(3)
                 assert_same(inst, p.solve_exact(), want)
                 prof = p.last_solve_profile()
-                assert prof.fast_path == 1 and prof.pair_levels == max(0, min(k, L, 13) - 2), inst.name
+                assert prof.fast_path == 1 and prof.pair_levels == max(0, min(k, L, 14) - 2), inst.name
                 n_pair += prof.pair_levels > 0
                 if want.table is not None:
                     for S in range(1, 1 << k):
