@@ -50,12 +50,16 @@ namespace {
 #ifndef PP_PAIR_STAGED
 #define PP_PAIR_STAGED 1
 #endif
+#ifndef PP_PAIR_PREFETCH
+#define PP_PAIR_PREFETCH 1
+#endif
 #ifndef PP_PAIR_FILL
 #define PP_PAIR_FILL 2
 #endif
 __host__ __device__ constexpr int pair_threads(int nv) { return nv <= PP_PAIR_T512 ? 512 : (nv <= PP_PAIR_T384 ? 384 : 256); }
 constexpr int kPlane = 64;               // words per strip slot
 constexpr int kStripWords = 16 * kPlane;  // per warp
+constexpr int kPlanWords = 32;            // per warp: row offsets of the pair to come
 
 // Per-target-node constants (W = 8q + r), built on the host.  A shuffle distance of 31 means
 // "nothing": rows occupy at most 30 lanes.
@@ -121,10 +125,6 @@ __device__ __noinline__ unsigned long long offer_pair(unsigned long long *best, 
     return best_seen;
 }
 
-template <int M>
-struct Mode {
-    static constexpr int value = M;
-};
 
 // L8: the chain length is a multiple of 8, so the last element of a row is a lane's last position.
 template <int NV, bool L8>
@@ -162,6 +162,7 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
     const int l8 = Lpad >> 3;  // 16-byte pieces per row
     const bool active = lane < l8;
     uint32_t *const sl = strips + warp * kStripWords + 31 + lane;  // this lane's word of slot 0
+    int *const wo = reinterpret_cast<int *>(strips + kWarps * kStripWords) + warp * kPlanWords;  // row offsets of a pair
     uint32_t *const se = strips + warp * kStripWords + (lane == 31 ? 31 : 32 + lane);  // ... of the E slots
     const int next_lane = (lane + 1) & 31;
     // rows are addressed in 16-byte pieces from the start of the table (fits 32 bits at every size)
@@ -189,49 +190,51 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
         A = d.masks[first + 2 * p];
         B = (2 * p + 1 < nmask) ? d.masks[first + 2 * p + 1] : A;
     };
-    // Rows of the pair (A, B).  MODE 0: bring both masks' rows into L2 (one 16-byte piece per lane
-    // covers a row); 1: load the rows of A into dp1; 2: load the rows of B into dp2 and take over
-    // the pair's source offsets.
-    auto touch_rows = [&](uint32_t A, uint32_t B, auto mode) {
-        constexpr int MODE = decltype(mode)::value;
+    // Rows of the pair (A, B).  plan_rows works out where they are (in 16-byte pieces from the first
+    // row of a mask) once, leaves the offsets in the warp's scratch words, and starts the rows on
+    // their way into L2 (one 16-byte piece per lane covers a row); load_rows1 / load_rows2 fetch the
+    // rows of A / of B into the registers later, and load_rows2 takes over the pair's source offsets.
+    auto plan_rows = [&](uint32_t A, uint32_t B, bool prefetch) {
         uint32_t abit = A & ~B;
         if (!abit) abit = A & (0u - A);  // a mask without partner runs as a pair with itself
         const uint32_t T = A & ~abit;
         const uint32_t bbit = B & ~T;
-        const uint4 *s1 = table + A * mask_rows + lane;
-        const uint4 *s2 = table + B * mask_rows + lane;
+        const uint32_t i1 = A * mask_rows + lane, i2 = B * mask_rows + lane;
         uint32_t rem = T;
-        int off[NV];
+        __syncwarp();  // the previous plan has been read
 #pragma unroll
-        for (int vi = 0; vi < NC; ++vi) {
-            off[vi] = (__ffs(rem) - 1) * l8;
-            rem &= rem - 1;
-        }
-        off[NV - 1] = (__ffs(abit) - 1) * l8;
-        const int offb = (__ffs(bbit) - 1) * l8;
-        if (MODE == 1) {
-#pragma unroll
-            for (int vi = 0; vi < NV; ++vi) dp1[vi] = active ? __ldg(s1 + off[vi]) : inf4;
-        } else if (MODE == 2) {
-#pragma unroll
-            for (int vi = 0; vi < NV; ++vi) {
-                voff[vi] = off[vi] * 8;
-                dp2[vi] = active ? __ldg(s2 + (vi == NV - 1 ? offb : off[vi])) : inf4;
-            }
-            voffb = offb * 8;
-            best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
-        } else if (active) {
-#pragma unroll
-            for (int vi = 0; vi < NV; ++vi) {
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(s1 + off[vi]));
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(s2 + (vi == NV - 1 ? offb : off[vi])));
+        for (int vi = 0; vi <= NV; ++vi) {
+            const uint32_t bits = vi < NC ? rem : (vi == NC ? abit : bbit);
+            const int off = (__ffs(bits) - 1) * l8;
+            if (vi < NC) rem &= rem - 1;
+            wo[vi] = off;
+            if (PP_PAIR_PREFETCH && prefetch && active) {
+                if (vi < NV) asm volatile("prefetch.global.L2 [%0];" ::"l"(table + (i1 + off)));
+                if (vi != NC) asm volatile("prefetch.global.L2 [%0];" ::"l"(table + (i2 + off)));
             }
         }
+        __syncwarp();
+    };
+    auto load_rows1 = [&](uint32_t A) {
+        const uint32_t i1 = A * mask_rows + lane;
+#pragma unroll
+        for (int vi = 0; vi < NV; ++vi) dp1[vi] = active ? __ldg(table + (i1 + wo[vi])) : inf4;
+    };
+    auto load_rows2 = [&](uint32_t B) {
+        const uint32_t i2 = B * mask_rows + lane;
+#pragma unroll
+        for (int vi = 0; vi < NV; ++vi) {
+            voff[vi] = wo[vi] * 8;
+            dp2[vi] = active ? __ldg(table + (i2 + wo[vi == NC ? NV : vi])) : inf4;
+        }
+        voffb = wo[NV] * 8;
+        best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
     };
     if (pi < npair) {
         fetch_masks(pi, S1, S2);
-        touch_rows(S1, S2, Mode<1>{});
-        touch_rows(S1, S2, Mode<2>{});
+        plan_rows(S1, S2, false);
+        load_rows1(S1);
+        load_rows2(S2);
     }
     best_seen = best_next;
     uint32_t thr2 = offer_threshold(best_seen);
@@ -371,7 +374,7 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
             // targets outside both masks: two rows each
             uint32_t wrem = full & ~(A | B);
             // rows of the next pair on their way into L2 while this pair is worked on
-            if (more) touch_rows(S1n, S2n, Mode<0>{});
+            if (more) plan_rows(S1n, S2n, true);
             while (wrem) {
                 const int w = __ffs(wrem) - 1;
                 wrem &= wrem - 1;
@@ -384,7 +387,7 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
                 const int w = __ffs(bbit) - 1;
                 relax1(w, dp1, voff[NV - 1], r1);
 #if PP_PAIR_STAGED
-                if (more) touch_rows(S1n, S2n, Mode<1>{});
+                if (more) load_rows1(S1n);
 #endif
                 finish(w, r1, r1, true, false);
             }
@@ -392,15 +395,15 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
                 const int w = __ffs(abit) - 1;
                 relax1(w, dp2, voffb, r2);
 #if !PP_PAIR_STAGED
-                if (more) touch_rows(S1n, S2n, Mode<1>{});
+                if (more) load_rows1(S1n);
 #endif
-                if (more) touch_rows(S1n, S2n, Mode<2>{});
+                if (more) load_rows2(S2n);
                 finish(w, r2, r2, false, true);
             }
         } else {
             // a mask without partner: one row per target
             uint32_t wrem = full & ~A;
-            if (more) touch_rows(S1n, S2n, Mode<0>{});
+            if (more) plan_rows(S1n, S2n, true);
             while (wrem) {
                 const int w = __ffs(wrem) - 1;
                 wrem &= wrem - 1;
@@ -408,8 +411,8 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
                 finish(w, r1, r1, true, false);
             }
             if (more) {
-                touch_rows(S1n, S2n, Mode<1>{});
-                touch_rows(S1n, S2n, Mode<2>{});
+                load_rows1(S1n);
+                load_rows2(S2n);
             }
         }
         if (best_next < best_seen) {
@@ -425,7 +428,7 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
 size_t pair_smem_bytes(const Dev &d, int nv)
 {
     return (((size_t)d.k * d.k * d.Lpad * 2 + 512 + 15) & ~(size_t)15) + sizeof(PMeta) * PP_MAX_K +
-           (size_t)(pair_threads(nv) / 32) * kStripWords * 4;
+           (size_t)(pair_threads(nv) / 32) * (kStripWords + kPlanWords) * 4;
 }
 
 template <int NV, bool L8>
