@@ -39,7 +39,7 @@ UNIT = "relaxations/s"
 # DRAM bytes per sweep launch (18 launches per Large solve, base frontier included) from the ncu
 # capture summarised in profiles/sweep_dram_traffic_large.md; set to None whenever the sweep
 # kernels change after that capture.
-SWEEP_DRAM_BYTES_PER_LAUNCH = 94.69e6
+SWEEP_DRAM_BYTES_PER_LAUNCH = None
 # Issue rate of packed 16-bit min/max measured on this part: 64 lanes per clock per SM, two
 # elements per lane (a three-input min/max issues at the same rate).
 PACKED_MINMAX_LANES_PER_CLK_SM = 64
@@ -310,7 +310,7 @@ def run_ours(args):
                 "frac": achieved / peaks["hbm_gbs"],
                 "traffic": SWEEP_DRAM_BYTES_PER_LAUNCH if prof.fast_path else None,
                 "peak_source": which + " (burst copy figure; the sweep is timed alone)",
-                "kernel": "k_sweep_fast + k_base (%d launches per solve)" % n_launch,
+                "kernel": "k_sweep_pair + k_sweep_fast + k_base (%d launches per solve)" % n_launch,
                 "algorithmic_bytes_per_launch": alg_bytes / n_launch,
                 "ms_per_launch": sweep_t * 1e3 / n_launch,
                 "algorithmic_bytes_per_solve": alg_bytes, "sweep_ms": sweep_t * 1e3,
