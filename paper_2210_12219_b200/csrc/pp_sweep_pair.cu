@@ -9,9 +9,8 @@
 //      together: the rank rows of the common sources T are read from shared memory once for the two
 //      masks;
 //   2. the two rows are re-packed position by position, (g1[c], g2[c]) in one register, so that the
-//      window minimum runs on both at once: in-lane prefix / suffix minima need no permutes, the
-//      shuffles over block minima and the strip traffic are shared, and the last combine is chosen
-//      by a warp-uniform switch on W mod 8, which makes every register index static;
+//      window minimum runs on both at once: in-lane prefix / suffix minima need no permutes, and
+//      the shuffles over block minima and the strip traffic are shared;
 //   3. rows dp[S1 + w][w] and dp[S2 + w][w] are written (w = b only for S1, w = a only for S2).
 // Window decomposition as in the one-mask kernel, blocks of 8 = lanes, W = 8q + r:
 //   out[8l + j] = min( suffix of block l - q (j >= r) or l - q - 1 (j < r) from offset (j - r) mod 8,
@@ -325,25 +324,29 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
             // (its s_i are +inf); it takes the block minimum of lane 0 and writes the entries of the
             // lane "before lane 0", whose suffixes are empty but whose next block is block 0.
             const uint32_t Bn = __shfl_sync(0xFFFFFFFFu, s[0], next_lane);
+            // whole blocks in between: D = min B[l-2^s+1 .. l], T1 = min B[l-q+1 .. l-1].  A lane without
+            // a source lane gets its own value back from the shuffle, which leaves D alone.  The chain of
+            // dependent shuffles is spread over the strip traffic below.
+            uint32_t D = s[0];
+            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.x));
             __syncwarp();  // the previous rows' readers are done
 #pragma unroll
             for (int j = 0; j < 8; ++j) sl[(8 + j) * kPlane] = s[j];
+            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.y));
 #pragma unroll
             for (int j = 1; j < 8; ++j) se[j * kPlane] = vmin2(s[j], Bn);
-            __syncwarp();
-            // whole blocks in between: D = min B[l-2^s+1 .. l], T1 = min B[l-q+1 .. l-1].
-            // A lane without a source lane gets its own value back from the shuffle, which leaves D alone.
-            uint32_t D = s[0];
-            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.x));
-            D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.y));
             D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.z));
+            __syncwarp();
+            const uint32_t *sp = sl + (int)mb.z;
+            uint32_t f[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) f[j] = sp[j * kPlane];
             D = vmin2(D, __shfl_up_sync(0xFFFFFFFFu, D, ma.w));
             const uint32_t T1 = vmin2(shfl_up_inf(D, (int)mb.x), shfl_up_inf(D, (int)mb.y));
-            const uint32_t *sp = sl + (int)mb.z;
             uint32_t out[8];
-            out[0] = vmin2(sp[0], T1);
+            out[0] = vmin2(f[0], T1);
 #pragma unroll
-            for (int j = 1; j < 8; ++j) out[j] = vmin3(o[j], sp[j * kPlane], T1);
+            for (int j = 1; j < 8; ++j) out[j] = vmin3(o[j], f[j], T1);
             // row (S + w, w) lies rowoff pieces after row (S, 0)
             if (ok1)
                 st_if(table_w + (base1 + mb.w),
