@@ -30,7 +30,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(binding.pp_solution) == 8 + 4 + 4 + 4 * 20 + 4 * 20
-    assert ctypes.sizeof(binding.pp_profile) == 32
+    assert ctypes.sizeof(binding.pp_profile) == 36
 
 
 def test_status_strings(lib):
