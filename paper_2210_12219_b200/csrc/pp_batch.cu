@@ -7,7 +7,7 @@
 //   1. stages the inputs, builds the memory prefix sums and the window table lo[w][c'];
 //   2. rank-compresses gamma (Eq. 3): layers sorted by bits, distinct bandwidths listed, one fp64
 //      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, obtained by
-//      a bitonic sort of all quotients in shared memory;
+//      a bitonic sort of all quotients (64-key tiles in registers, the wide strides in shared memory);
 //   3. sweeps the popcount levels with a flat thread <-> (target row, position) mapping:
 //      phase A forms g[c] = min_v max(dp[S'\{w}][v][c], rank[v][w][c]) for every row of the level,
 //      two neighbouring positions per thread as one packed u16x2 word,
@@ -80,6 +80,46 @@ size_t batch_smem_bytes(int L, int k)
 __device__ __forceinline__ uint32_t info_pack(uint32_t P, int w, uint32_t src0)
 {
     return P | ((uint32_t)w << 12) | (src0 << 16);
+}
+
+// (key, payload) pairs in lexicographic order; payloads are distinct, so the order is total
+__device__ __forceinline__ bool pair_gt(unsigned long long ka, uint32_t va, unsigned long long kb, uint32_t vb)
+{
+    return ka > kb || (ka == kb && va > vb);
+}
+
+// Bitonic steps of the size levels size_lo..size_hi whose stride is at most 32, on the 64-key tile
+// that starts at `base` (a multiple of 64): lane l holds keys base+l and base+l+32 in registers.
+__device__ __forceinline__ void sort_tile(unsigned long long *skey, uint16_t *sval, int base, int lane,
+                                          int size_lo, int size_hi)
+{
+    unsigned long long ka = skey[base + lane], kb = skey[base + lane + 32];
+    uint32_t va = sval[base + lane], vb = sval[base + lane + 32];
+    for (int size = size_lo; size <= size_hi; size <<= 1) {
+        const bool upa = ((base + lane) & size) == 0, upb = ((base + lane + 32) & size) == 0;
+        int stride = size >> 1;
+        if (stride >= 32) {  // the two keys of a lane are partners
+            if (pair_gt(ka, va, kb, vb) == upa) {
+                const unsigned long long tk = ka; ka = kb; kb = tk;
+                const uint32_t tv = va; va = vb; vb = tv;
+            }
+            stride = 16;
+        }
+        for (; stride > 0; stride >>= 1) {
+            const bool lower = (lane & stride) == 0;
+            const unsigned long long oka = __shfl_xor_sync(0xFFFFFFFFu, ka, stride);
+            const uint32_t ova = __shfl_xor_sync(0xFFFFFFFFu, va, stride);
+            const unsigned long long okb = __shfl_xor_sync(0xFFFFFFFFu, kb, stride);
+            const uint32_t ovb = __shfl_xor_sync(0xFFFFFFFFu, vb, stride);
+            // the lower partner keeps the smaller pair when the run ascends
+            if (pair_gt(ka, va, oka, ova) == (lower == upa)) { ka = oka; va = ova; }
+            if (pair_gt(kb, vb, okb, ovb) == (lower == upb)) { kb = okb; vb = ovb; }
+        }
+    }
+    skey[base + lane] = ka;
+    skey[base + lane + 32] = kb;
+    sval[base + lane] = (uint16_t)va;
+    sval[base + lane + 32] = (uint16_t)vb;
 }
 
 __global__ void __launch_bounds__(kBatchThreads, 2)
@@ -244,23 +284,52 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                 sval[i] = (uint16_t)i;
             }
             __syncthreads();
-            for (int size = 2; size <= npad; size <<= 1)
-                for (int stride = size >> 1; stride > 0; stride >>= 1) {
-                    for (int t = tid; t < (npad >> 1); t += kBatchThreads) {
-                        const int lo_i = 2 * t - (t & (stride - 1));  // index with the stride bit clear
-                        const int hi_i = lo_i + stride;
-                        const bool up = (lo_i & size) == 0;
-                        const unsigned long long a = skey[lo_i], b = skey[hi_i];
-                        if ((a > b) == up) {
-                            skey[lo_i] = b;
-                            skey[hi_i] = a;
-                            const uint16_t va = sval[lo_i];
-                            sval[lo_i] = sval[hi_i];
-                            sval[hi_i] = va;
+            if (npad >= 64) {
+                // Tiles of 64 keys, two per lane, stay in a warp's registers for every run of steps
+                // with stride <= 32 (shuffles, no block barrier); only strides >= 64 go through
+                // shared memory with a barrier each.
+                const int tiles = npad >> 6;
+                for (int t = wid; t < tiles; t += kBatchWarps) sort_tile(skey, sval, t << 6, lane, 2, 64);
+                __syncthreads();
+                for (int size = 128; size <= npad; size <<= 1) {
+                    for (int stride = size >> 1; stride >= 64; stride >>= 1) {
+                        for (int t = tid; t < (npad >> 1); t += kBatchThreads) {
+                            const int lo_i = 2 * t - (t & (stride - 1));  // index with the stride bit clear
+                            const int hi_i = lo_i + stride;
+                            const bool up = (lo_i & size) == 0;
+                            const unsigned long long a = skey[lo_i], b = skey[hi_i];
+                            const uint16_t va = sval[lo_i], vb = sval[hi_i];
+                            if (pair_gt(a, va, b, vb) == up) {
+                                skey[lo_i] = b;
+                                skey[hi_i] = a;
+                                sval[lo_i] = vb;
+                                sval[hi_i] = va;
+                            }
                         }
+                        __syncthreads();
                     }
+                    for (int t = wid; t < tiles; t += kBatchWarps) sort_tile(skey, sval, t << 6, lane, size, size);
                     __syncthreads();
                 }
+            } else {
+                for (int size = 2; size <= npad; size <<= 1)
+                    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                        for (int t = tid; t < (npad >> 1); t += kBatchThreads) {
+                            const int lo_i = 2 * t - (t & (stride - 1));  // index with the stride bit clear
+                            const int hi_i = lo_i + stride;
+                            const bool up = (lo_i & size) == 0;
+                            const unsigned long long a = skey[lo_i], b = skey[hi_i];
+                            if ((a > b) == up) {
+                                skey[lo_i] = b;
+                                skey[hi_i] = a;
+                                const uint16_t va = sval[lo_i];
+                                sval[lo_i] = sval[hi_i];
+                                sval[hi_i] = va;
+                            }
+                        }
+                        __syncthreads();
+                    }
+            }
             for (int i = tid; i < n; i += kBatchThreads) {
                 int first = i;  // runs of equal quotients are short except in degenerate inputs
                 const unsigned long long key = skey[i];
