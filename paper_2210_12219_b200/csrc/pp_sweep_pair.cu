@@ -100,6 +100,10 @@ __device__ __forceinline__ void min4(uint32_t (&r)[4], const uint4 &a, const uin
     r[0] = vmin3(r[0], a.x, b.x); r[1] = vmin3(r[1], a.y, b.y);
     r[2] = vmin3(r[2], a.z, b.z); r[3] = vmin3(r[3], a.w, b.w);
 }
+__device__ __forceinline__ void setmin4(uint32_t (&r)[4], const uint4 &a, const uint4 &b, const uint4 &c)
+{
+    r[0] = vmin3(a.x, b.x, c.x); r[1] = vmin3(a.y, b.y, c.y); r[2] = vmin3(a.z, b.z, c.z); r[3] = vmin3(a.w, b.w, c.w);
+}
 __device__ __forceinline__ void setmin4(uint32_t (&r)[4], const uint4 &a, const uint4 &b)
 {
     r[0] = vmin2(a.x, b.x); r[1] = vmin2(a.y, b.y); r[2] = vmin2(a.z, b.z); r[3] = vmin2(a.w, b.w);
@@ -251,10 +255,12 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
             const uint4 ga = *reinterpret_cast<const uint4 *>(rw + voff[NV - 1]);
             const uint4 gb = *reinterpret_cast<const uint4 *>(rw + voffb);
             if (NC >= 2) {
+                // the first minimum takes three sources (two common ones and the mask's own), every
+                // further one two more: ceil((NV - 1) / 2) three-input minima per register
                 const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[0]);
                 const uint4 h = *reinterpret_cast<const uint4 *>(rw + voff[NC >= 2 ? 1 : 0]);
-                setmin4(r1, max4(dp1[0], g), max4(dp1[NC >= 2 ? 1 : 0], h));
-                setmin4(r2, max4(dp2[0], g), max4(dp2[NC >= 2 ? 1 : 0], h));
+                setmin4(r1, max4(dp1[0], g), max4(dp1[NC >= 2 ? 1 : 0], h), max4(dp1[NV - 1], ga));
+                setmin4(r2, max4(dp2[0], g), max4(dp2[NC >= 2 ? 1 : 0], h), max4(dp2[NV - 1], gb));
 #pragma unroll
                 for (int vi = 2; vi + 1 < NC; vi += 2) {
                     const uint4 g2 = *reinterpret_cast<const uint4 *>(rw + voff[vi]);
@@ -262,13 +268,10 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
                     min4(r1, max4(dp1[vi], g2), max4(dp1[vi + 1], h2));
                     min4(r2, max4(dp2[vi], g2), max4(dp2[vi + 1], h2));
                 }
-                if (NC & 1) {  // the last common source shares a minimum with a (resp. b)
+                if (NC & 1) {  // one common source is left over
                     const uint4 g3 = *reinterpret_cast<const uint4 *>(rw + voff[NC - 1]);
-                    min4(r1, max4(dp1[NC - 1], g3), max4(dp1[NV - 1], ga));
-                    min4(r2, max4(dp2[NC - 1], g3), max4(dp2[NV - 1], gb));
-                } else {
-                    min4(r1, max4(dp1[NV - 1], ga));
-                    min4(r2, max4(dp2[NV - 1], gb));
+                    min4(r1, max4(dp1[NC - 1], g3));
+                    min4(r2, max4(dp2[NC - 1], g3));
                 }
             } else if (NC == 1) {
                 const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[0]);
@@ -283,19 +286,23 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
         auto relax1 = [&](int w, const uint4 (&dp)[NV], int lastoff, uint32_t (&r)[4]) {
             const uint16_t *rw = rank_s + wm[w].rwoff + 8 * lane;
             const uint4 ga = *reinterpret_cast<const uint4 *>(rw + lastoff);
-            if (NC >= 1) {
+            if (NC >= 2) {
                 const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[0]);
-                setmin4(r, max4(dp[0], g), max4(dp[NV - 1], ga));
+                const uint4 h = *reinterpret_cast<const uint4 *>(rw + voff[NC >= 2 ? 1 : 0]);
+                setmin4(r, max4(dp[0], g), max4(dp[NC >= 2 ? 1 : 0], h), max4(dp[NV - 1], ga));
 #pragma unroll
-                for (int vi = 1; vi + 1 < NC; vi += 2) {
+                for (int vi = 2; vi + 1 < NC; vi += 2) {
                     const uint4 g2 = *reinterpret_cast<const uint4 *>(rw + voff[vi]);
                     const uint4 h2 = *reinterpret_cast<const uint4 *>(rw + voff[vi + 1]);
                     min4(r, max4(dp[vi], g2), max4(dp[vi + 1], h2));
                 }
-                if (!(NC & 1)) {
+                if (NC & 1) {
                     const uint4 g3 = *reinterpret_cast<const uint4 *>(rw + voff[NC >= 1 ? NC - 1 : 0]);
                     min4(r, max4(dp[NC >= 1 ? NC - 1 : 0], g3));
                 }
+            } else if (NC == 1) {
+                const uint4 g = *reinterpret_cast<const uint4 *>(rw + voff[0]);
+                setmin4(r, max4(dp[0], g), max4(dp[NV - 1], ga));
             } else {
                 set4(r, max4(dp[NV - 1], ga));
             }
