@@ -238,6 +238,14 @@ def test_large_config_full_size():
                 assert np.array_equal(p.debug_read_state_row(S, n), table[(1 << size) - 1, j])
         # second solve on the same handle gives the same answer (scratch is reused)
         assert_same(inst, p.solve_exact(), want)
+        # the same instance with every level on the kernel that takes one source mask per warp
+        p.force_generic(2)
+        assert_same(inst, p.solve_exact(), want)
+        prof = p.last_solve_profile()
+        assert prof.fast_path == 1 and prof.pair_levels == 0
+        S = sum(1 << n for n in nodes)
+        for j, n in enumerate(nodes):
+            assert np.array_equal(p.debug_read_state_row(S, n), table[(1 << len(nodes)) - 1, j])
 
 
 def test_maximum_sizes():
