@@ -10,7 +10,8 @@
 //      a bitonic sort of all quotients (64-key tiles in registers, the wide strides in shared memory);
 //   3. sweeps the popcount levels with a flat thread <-> (target row, position) mapping:
 //      phase A forms g[c] = min_v max(dp[S'\{w}][v][c], rank[v][w][c]) for every row of the level,
-//      two neighbouring positions per thread as one packed u16x2 word,
+//      two neighbouring positions per thread as one packed u16x2 word, thread <-> (source mask,
+//      word) with the source words in registers for all target nodes,
 //      phase B takes the window minimum over [lo_w(c'), c'-1];
 //   4. reduces the final states to the smallest (value, popcount, mask, node), walks back with
 //      the threshold rule, and maps the winning rank back to its quotient.
@@ -23,7 +24,7 @@ constexpr int kBatchWarps = kBatchThreads / 32;
 constexpr uint16_t kInf16 = 0xFFFFu;
 
 struct BatchLayout {
-    size_t dp, g, rank, gu, rk, cnt, skey, sval, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, total;
+    size_t dp, g, rank, gu, rk, cnt, skey, sval, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, mlist, moff, total;
 };
 
 __host__ __device__ inline BatchLayout batch_layout(int L, int k)
@@ -56,6 +57,8 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     b.rowoff = take(((size_t)1 << k) * sizeof(uint32_t));
     b.loff = take((size_t)(k + 2) * sizeof(uint32_t));
     b.rowinfo = take(rows * sizeof(uint32_t));
+    b.mlist = take(((size_t)1 << k) * sizeof(uint16_t));
+    b.moff = take((size_t)(k + 2) * sizeof(uint32_t));
     b.dp = take(rows * Ls * sizeof(uint16_t));
     b.g = take(best * Ls * sizeof(uint16_t));
     b.rank = take((size_t)k * k * Ls * sizeof(uint16_t));
@@ -122,6 +125,58 @@ __device__ __forceinline__ void sort_tile(unsigned long long *skey, uint16_t *sv
     sval[base + lane + 32] = (uint16_t)vb;
 }
 
+// Phase A of one level for the sources masks of NV nodes: g[(P + w, w)][c] = min over v in P of
+// max(dp[P][v][c], rank[v][w][c]) for every node w outside P, two positions per 32-bit word.
+struct BatchRelaxArgs {
+    const uint16_t *dp;       // [compact row][Ls]
+    uint16_t *gbuf;           // [row within the target level][Ls]
+    const uint16_t *rank;     // [v][w][Ls]
+    const uint32_t *rowoff;   // compact row of (S, lowest node of S)
+    const uint16_t *masks;    // the source masks of this level
+    uint32_t nmasks;
+    uint32_t row0;            // first compact row of the target level
+    int k, Lh;
+};
+
+template <int NV>
+__device__ __forceinline__ void batch_relax(const BatchRelaxArgs &a, int tid)
+{
+    const int Lh = a.Lh, k = a.k;
+    const uint32_t *dp32 = reinterpret_cast<const uint32_t *>(a.dp);
+    const uint32_t *rank32 = reinterpret_cast<const uint32_t *>(a.rank);
+    uint32_t *g32 = reinterpret_cast<uint32_t *>(a.gbuf);
+    const uint32_t items = a.nmasks * (uint32_t)Lh;
+    const uint32_t full = (1u << k) - 1u;
+    for (uint32_t it = tid; it < items; it += kBatchThreads) {
+        const uint32_t pi = it / (uint32_t)Lh;
+        const int cw = (int)(it - pi * (uint32_t)Lh);
+        const uint32_t P = a.masks[pi];
+        const uint32_t *src = dp32 + (size_t)a.rowoff[P] * Lh + cw;
+        uint32_t d[NV];
+        int roff[NV];  // word offset of rank[v][0][cw]
+        uint32_t rem = P;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int v = __ffs(rem) - 1;
+            rem &= rem - 1;
+            d[i] = src[i * Lh];
+            roff[i] = v * k * Lh + cw;
+        }
+        for (uint32_t wrem = full & ~P; wrem; wrem &= wrem - 1) {
+            const int w = __ffs(wrem) - 1;
+            const uint32_t *rw = rank32 + w * Lh;
+            uint32_t g = __vmaxu2(d[0], rw[roff[0]]);
+#pragma unroll
+            for (int i = 1; i + 1 < NV; i += 2)
+                g = __vimin3_u16x2(g, __vmaxu2(d[i], rw[roff[i]]), __vmaxu2(d[i + 1], rw[roff[i + 1]]));
+            if (!(NV & 1)) g = __vminu2(g, __vmaxu2(d[NV - 1], rw[roff[NV - 1]]));
+            const uint32_t S2 = P | (1u << w);
+            const uint32_t row = a.rowoff[S2] + (uint32_t)__popc(S2 & ((1u << w) - 1u)) - a.row0;
+            g32[row * Lh + cw] = g;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kBatchThreads, 2)
 k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
@@ -141,6 +196,8 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     uint32_t *rowoff = reinterpret_cast<uint32_t *>(smem + lay.rowoff);
     uint32_t *loff = reinterpret_cast<uint32_t *>(smem + lay.loff);    // first compact row of each level
     uint32_t *rowinfo = reinterpret_cast<uint32_t *>(smem + lay.rowinfo);
+    uint16_t *mlist = reinterpret_cast<uint16_t *>(smem + lay.mlist);  // masks by (popcount, value)
+    uint32_t *moff = reinterpret_cast<uint32_t *>(smem + lay.moff);    // first entry of each popcount
     uint16_t *dp = reinterpret_cast<uint16_t *>(smem + lay.dp);        // [compact row][L]
     uint16_t *gbuf = reinterpret_cast<uint16_t *>(smem + lay.g);       // [row within level][L]
     uint16_t *rank = reinterpret_cast<uint16_t *>(smem + lay.rank);    // [v][w][c]
@@ -167,8 +224,13 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     // rowoff[S] = compact row of (S, lowest node of S); loff[j] = first row of level j.
     if (tid <= k + 1) {
         uint32_t cnt = 0;  // rows of all masks with popcount below tid
-        for (uint32_t S = 0; S < nm; ++S) cnt += (__popc(S) < tid) ? __popc(S) : 0;
+        uint32_t masks = 0;
+        for (uint32_t S = 0; S < nm; ++S) {
+            cnt += (__popc(S) < tid) ? __popc(S) : 0;
+            masks += (__popc(S) < tid);
+        }
         loff[tid] = cnt;
+        moff[tid] = masks;
     }
     __syncthreads();
     for (uint32_t S = tid; S < nm; S += kBatchThreads) {
@@ -176,6 +238,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         uint32_t before = 0;  // masks of the same popcount below S
         for (uint32_t T = 0; T < S; ++T) before += (__popc(T) == pc);
         rowoff[S] = loff[pc] + before * pc;
+        mlist[moff[pc] + before] = (uint16_t)S;
     }
     __syncthreads();
     for (uint32_t S = 1 + tid; S < nm; S += kBatchThreads) {
@@ -357,23 +420,17 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                 __syncthreads();
                 continue;
             }
-            {  // phase A: thread <-> (row, word of two positions)
-                int rr = tid / Lh, cw = tid - rr * Lh;
-                while (rr < (int)nrows) {
-                    const uint32_t info = rowinfo[row0 + rr];
-                    const int w = (info >> 12) & 15;
-                    const uint32_t *src = reinterpret_cast<const uint32_t *>(dp + (size_t)(info >> 16) * Ls) + cw;
-                    const uint32_t *rw = reinterpret_cast<const uint32_t *>(rank + w * Ls) + cw;
-                    uint32_t g = 0xFFFFFFFFu;
-                    for (uint32_t rem = info & 0xFFFu; rem; rem &= rem - 1) {
-                        const int v = __ffs(rem) - 1;
-                        g = __vminu2(g, __vmaxu2(*src, rw[v * k * Lh]));
-                        src += Lh;
-                    }
-                    reinterpret_cast<uint32_t *>(gbuf)[rr * Lh + cw] = g;
-                    rr += drA;
-                    cw += dcA;
-                    if (cw >= Lh) { cw -= Lh; ++rr; }
+            // phase A: thread <-> (source mask P, word of two positions); the words of P's rows stay
+            // in registers for all target nodes
+            {
+                const BatchRelaxArgs ra = {dp, gbuf, rank, rowoff, mlist + moff[j - 1], moff[j] - moff[j - 1],
+                                           row0, k, Lh};
+                switch (j - 1) {
+#define PP_CASE(N) case N: batch_relax<N>(ra, tid); break;
+                    PP_CASE(1) PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6)
+                    PP_CASE(7) PP_CASE(8) PP_CASE(9) PP_CASE(10) PP_CASE(11)
+#undef PP_CASE
+                    default: break;
                 }
             }
             __syncthreads();

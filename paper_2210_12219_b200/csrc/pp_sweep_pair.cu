@@ -30,6 +30,8 @@ namespace pp {
 
 namespace {
 
+// Tunables (measured on the k = 18, L = 200 benchmark chain): levels the kernel takes by number of
+// source nodes, how full the machine must be (pairs * FILL >= warps), threads per block.
 #ifndef PP_PAIR_T512
 #define PP_PAIR_T512 6
 #endif
@@ -42,15 +44,6 @@ namespace {
 // threads per block by the number of source rows per mask (2 * NV rows of 4 registers per lane)
 #ifndef PP_PAIR_T384
 #define PP_PAIR_T384 11
-#endif
-#ifndef PP_PAIR_PIPE
-#define PP_PAIR_PIPE 1
-#endif
-#ifndef PP_PAIR_STAGED
-#define PP_PAIR_STAGED 1
-#endif
-#ifndef PP_PAIR_PREFETCH
-#define PP_PAIR_PREFETCH 1
 #endif
 #ifndef PP_PAIR_FILL
 #define PP_PAIR_FILL 2
@@ -211,7 +204,7 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
             const int off = (__ffs(bits) - 1) * l8;
             if (vi < NC) rem &= rem - 1;
             wo[vi] = off;
-            if (PP_PAIR_PREFETCH && prefetch && active) {
+            if (prefetch && active) {
                 if (vi < NV) asm volatile("prefetch.global.L2 [%0];" ::"l"(table + (i1 + off)));
                 if (vi != NC) asm volatile("prefetch.global.L2 [%0];" ::"l"(table + (i2 + off)));
             }
@@ -396,17 +389,12 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
             {
                 const int w = __ffs(bbit) - 1;
                 relax1(w, dp1, voff[NV - 1], r1);
-#if PP_PAIR_STAGED
                 if (more) load_rows1(S1n);
-#endif
                 finish(w, r1, r1, true, false);
             }
             {
                 const int w = __ffs(abit) - 1;
                 relax1(w, dp2, voffb, r2);
-#if !PP_PAIR_STAGED
-                if (more) load_rows1(S1n);
-#endif
                 if (more) load_rows2(S2n);
                 finish(w, r2, r2, false, true);
             }
