@@ -186,6 +186,13 @@ pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out);
  * `mask` must contain node v.  Synchronous. */
 pp_status pp_debug_read_state_row(pp_problem *p, uint32_t mask, int32_t v, double *row_out);
 
+/* Test hook (host only, needs no device): the order in which the sweep lists the non-empty node
+ * sets of k nodes.  masks_out[2^k - 1] receives them level by level (popcount 1, 2, ..., k),
+ * level_off_out[k + 2] the first index of every level (entry 0 is 0, entry k + 1 the total).
+ * Within a level, neighbours differ by one node swapped for another (revolving-door order):
+ * the sweep kernel that takes two node sets per warp relies on it. */
+pp_status pp_debug_mask_order(int32_t k, uint32_t *masks_out, uint32_t *level_off_out);
+
 /* Force (1) or forbid (0) the generic sweep kernel; 2 = automatic choice among the kernels that
  * take one source mask per warp (the two-mask kernel is left out); 3 = the two-mask kernel on every
  * level it can run, however small; -1 restores the automatic choice.  Meant for tests that want every kernel checked on the same instance. */

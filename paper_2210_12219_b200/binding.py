@@ -24,7 +24,7 @@ EXPORTS = (
     "pp_problem_create", "pp_problem_destroy", "pp_problem_set_stream",
     "pp_problem_workspace_bytes", "pp_problem_set_workspace", "pp_solve_exact",
     "pp_solve_exact_dev", "pp_eval_plans", "pp_eval_plans_dev", "pp_solve_exact_batch",
-    "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row",
+    "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row", "pp_debug_mask_order",
     "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str",
 )
 
@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
         L.pp_solve_exact_batch_dev.argtypes = [i64, i32, i32] + [vp] * 10
         L.pp_last_solve_profile.argtypes = [vp, ctypes.POINTER(pp_profile)]
         L.pp_debug_read_state_row.argtypes = [vp, ctypes.c_uint32, i32, vp]
+        L.pp_debug_mask_order.argtypes = [i32, vp, vp]
         L.pp_problem_force_generic.argtypes = [vp, i32]
         L.pp_solve_exact_static.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp]
         L.pp_status_str.argtypes = [ctypes.c_int]
@@ -244,6 +245,15 @@ def solve_exact_batch(L, k, out_bits, mem, node_mem, bw) -> BatchSolution:
                                     (beta, m, cuts, placement, status)))
     _check(st, "pp_solve_exact_batch")
     return BatchSolution(beta, m, cuts[:, : max(k - 1, 0)] if k > 1 else cuts[:, :0], placement, status)
+
+
+def debug_mask_order(k: int):
+    """pp_debug_mask_order: (masks uint32 [2^k - 1], level_off uint32 [k + 2]); needs no device."""
+    masks = np.zeros((1 << k) - 1, dtype=np.uint32)
+    level_off = np.zeros(k + 2, dtype=np.uint32)
+    _check(lib().pp_debug_mask_order(int(k), ctypes.c_void_p(masks.ctypes.data),
+                                     ctypes.c_void_p(level_off.ctypes.data)), "pp_debug_mask_order")
+    return masks, level_off
 
 
 def solve_exact_batch_dev(B, L, k, bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr,

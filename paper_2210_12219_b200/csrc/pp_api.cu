@@ -587,6 +587,20 @@ pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *
     return from_cuda(e2);
 }
 
+pp_status pp_debug_mask_order(int32_t k, uint32_t *masks_out, uint32_t *level_off_out)
+{
+    if (!masks_out || !level_off_out || k < 1) return PP_ERR_ARG;
+    if (k > PP_MAX_K) return PP_ERR_LIMIT;
+    try {
+        const MaskList &ml = mask_list(k);
+        std::copy(ml.masks.begin(), ml.masks.end(), masks_out);
+        std::copy(ml.level_off.begin(), ml.level_off.end(), level_off_out);
+    } catch (const std::bad_alloc &) {
+        return PP_ERR_NOMEM;
+    }
+    return PP_OK;
+}
+
 pp_status pp_debug_read_state_row(pp_problem *p, uint32_t mask, int32_t v, double *row_out)
 {
     if (!p || !row_out || !p->solved) return PP_ERR_ARG;

@@ -3,6 +3,7 @@ and rejects bad arguments before touching a device."""
 from __future__ import annotations
 
 import ctypes
+import math
 import os
 import re
 
@@ -86,3 +87,23 @@ def test_no_cpu_fallback_without_device(lib):
     st, _ = _create(4, np.ones(4, np.uint64), np.ones(4, np.uint64), 2, np.ones(2, np.uint64),
                     np.ones(4, np.uint32))
     assert st in (binding.PP_ERR_CUDA, binding.PP_ERR_NOMEM)
+
+
+def test_mask_order_is_a_revolving_door(lib):
+    # the two-mask sweep kernel pairs neighbours of each level: they must differ by one node
+    # swapped for another, every non-empty node set must appear exactly once, levels by popcount
+    for k in (1, 2, 3, 5, 8, 12, 18):
+        masks, level_off = binding.debug_mask_order(k)
+        assert level_off[0] == 0 and level_off[k + 1] == (1 << k) - 1
+        assert sorted(int(m) for m in masks) == list(range(1, 1 << k))
+        for j in range(1, k + 1):
+            level = [int(m) for m in masks[level_off[j]:level_off[j + 1]]]
+            assert len(level) == math.comb(k, j)
+            assert all(bin(m).count("1") == j for m in level)
+            for a, b in zip(level, level[1:]):
+                assert bin(a ^ b).count("1") == 2, (k, j, a, b)
+    bad = np.zeros(4, np.uint32)
+    assert binding.lib().pp_debug_mask_order(0, ctypes.c_void_p(bad.ctypes.data),
+                                             ctypes.c_void_p(bad.ctypes.data)) == binding.PP_ERR_ARG
+    assert binding.lib().pp_debug_mask_order(21, ctypes.c_void_p(bad.ctypes.data),
+                                             ctypes.c_void_p(bad.ctypes.data)) == binding.PP_ERR_LIMIT
