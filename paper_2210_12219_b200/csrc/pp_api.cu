@@ -328,7 +328,7 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     try {
         if (!has_fast && p->elem == 2 && p->Lpad <= 240 && k >= 2) {
             gmeta.resize((size_t)k * p->Lpad);
-            gen_meta_build(L, k, p->Lpad, p->lo.data(), gmeta.data());
+            p->d.gen_levels = gen_meta_build(L, k, p->Lpad, p->lo.data(), gmeta.data());
         }
     } catch (const std::bad_alloc &) {
         delete p;

@@ -37,6 +37,7 @@ struct Dev {
     int32_t *err;              // device error word (0 = fine)
     const void *fast_meta;     // per-node window constants of the register-tiled sweep, or null
     const uint32_t *gen_meta;  // [k*Lpad] per-(node, position) lookup words of its general-window step, or null
+    int gen_levels;            // levels of that step's sparse table (1 + floor(log2(longest window)))
     const void *pair_meta;     // per-node window constants of the two-mask sweep, or null
 };
 
@@ -54,7 +55,7 @@ cudaError_t launch_base(const Dev &d, cudaStream_t s);
 cudaError_t launch_sweep_generic(const Dev &d, int level, cudaStream_t s);
 size_t fast_meta_bytes();
 bool fast_meta_build(int L, int k, const int16_t *lo, void *out);
-void gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out);
+int gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out);
 bool fast_sweep_supported(const Dev &d);
 cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s);
 size_t pair_meta_bytes();

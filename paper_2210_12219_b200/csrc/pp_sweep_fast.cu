@@ -23,6 +23,8 @@
 // The relaxation of the next target node is issued in the same straight-line block as the window
 // step of the current one, so that independent loads fill the latencies of the dependent chain.
 // Row (S + w, w) has the single source mask S, so no two warps ever write the same row.
+#include <algorithm>
+
 #include "pp_internal.cuh"
 #include "pp_sweep_ops.cuh"
 
@@ -61,7 +63,8 @@ struct FastMeta {
 };
 
 constexpr int NT = PP_FAST_NT;  // target nodes processed together
-constexpr int kStripElems = 256 + 256 + 168;  // per-warp strips of the general window step (u16)
+// per-warp strip of the general window step (u16): the levels of the sparse table, then +inf
+__host__ __device__ constexpr int gen_strip_elems(int levels, int Lpad) { return levels * Lpad + 8; }
 constexpr int kTailWords = 128 + 128;           // per-warp suffix strip of the constant-window step: +inf pad, data
 
 // Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].  tl points at this lane's four
@@ -145,74 +148,59 @@ __device__ __forceinline__ void window_min(const uint32_t (&r)[NT][4], const WMe
     }
 }
 
-// Window minimum for arbitrary (non-decreasing) window starts lo_w(c').  Same block decomposition
-// as above, but the tail of the block that holds lo, and the whole blocks in between, are fetched
-// from per-warp shared-memory strips through lookup words prepared on the host (gen_meta_build):
-//   sfx[i][l]  in-lane inclusive suffix minima of every lane (position-major); entry (0, 30) is
-//              +inf because rows occupy at most 30 lanes,
-//   T[s][l]    minimum of the 2^s block minima ending at lane l (sparse table, s = 0..4);
-//              T[160] is a constant +inf,
-//   g[c]       the relaxed row itself, for the rare window that lies inside one block.
-// Lookup word of (w, c'): sfx index | T index 1 << 8 | T index 2 << 16 | lo << 24.
-__device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const uint32_t *meta_row,
-                                                   uint16_t *sfx, uint16_t *gs, uint16_t *T, int lane,
-                                                   bool active, uint32_t (&o)[4])
+// Window minimum for arbitrary window starts lo_w(c'): a sparse table over the positions of the
+// relaxed row, T[s][c] = min g[c - 2^s + 1 .. c], built in registers level by level (shifts by 1, 2
+// and 4 positions inside a lane's 16-byte vector with one to two registers from the lane below,
+// shifts by 8 and more as whole-lane shuffles) and parked in the warp's strip of shared memory.
+// Output c' is then min(T[s][c' - 1], T[s][lo + 2^s - 1]) with 2^s <= c' - lo < 2^(s+1): two 16-bit
+// loads whose byte offsets come from the lookup word the host prepared for (w, c')
+// (gen_meta_build); an empty window points both at the +inf element behind the last level.
+// Entries that would reach below position 0 hold garbage and are never asked for.
+__device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const uint32_t *meta_row, uint16_t *T,
+                                                   int lane, bool active, int nlev, int Lpad, uint32_t (&o)[4])
 {
-    const uint32_t m0 = vmin2(r[0], __byte_perm(r[0], 0, 0x1032));
-    const uint32_t m1 = vmin2(r[1], __byte_perm(r[1], 0, 0x1032));
-    const uint32_t m2 = vmin2(r[2], __byte_perm(r[2], 0, 0x1032));
-    const uint32_t m3 = vmin2(r[3], __byte_perm(r[3], 0, 0x1032));
-    const uint32_t q1 = vmin2(m0, m1), q2 = vmin2(q1, m2);
-    const uint32_t t2 = vmin2(m2, m3), t1 = vmin2(m1, t2);
-    const uint32_t B = vmin2(q2, m3);
-    // exclusive in-lane prefix minima, one per position
-    uint32_t xp[4];
-    xp[0] = __byte_perm(r[0], kInf2, 0x1044);
-    xp[1] = vmin2(m0, __byte_perm(r[1], kInf2, 0x1044));
-    xp[2] = vmin2(q1, __byte_perm(r[2], kInf2, 0x1044));
-    xp[3] = vmin2(q2, __byte_perm(r[3], kInf2, 0x1044));
-    const uint32_t sv[4] = {vmin2(__byte_perm(m0, r[0], 0x7610), t1), vmin2(__byte_perm(m1, r[1], 0x7610), t2),
-                            vmin2(__byte_perm(m2, r[2], 0x7610), m3), __byte_perm(m3, r[3], 0x7610)};
-    __syncwarp();  // the previous row's readers are done with the strips
+    uint32_t t[4] = {r[0], r[1], r[2], r[3]};
+    uint16_t *mine = T + 8 * lane;
+    __syncwarp();  // the previous row's readers are done with the strip
+    if (active) *reinterpret_cast<uint4 *>(mine) = make_uint4(t[0], t[1], t[2], t[3]);
+    if (nlev > 1) {  // shift by one position
+        const uint32_t below = __shfl_up_sync(0xFFFFFFFFu, t[3], 1);
+        const uint32_t y0 = __byte_perm(below, t[0], 0x5432), y1 = __byte_perm(t[0], t[1], 0x5432);
+        const uint32_t y2 = __byte_perm(t[1], t[2], 0x5432), y3 = __byte_perm(t[2], t[3], 0x5432);
+        t[0] = vmin2(t[0], y0); t[1] = vmin2(t[1], y1); t[2] = vmin2(t[2], y2); t[3] = vmin2(t[3], y3);
+        if (active) *reinterpret_cast<uint4 *>(mine + Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+    }
+    if (nlev > 2) {  // by two positions: one register
+        const uint32_t below = __shfl_up_sync(0xFFFFFFFFu, t[3], 1);
+        const uint32_t a0 = vmin2(t[0], below), a1 = vmin2(t[1], t[0]), a2 = vmin2(t[2], t[1]), a3 = vmin2(t[3], t[2]);
+        t[0] = a0; t[1] = a1; t[2] = a2; t[3] = a3;
+        if (active) *reinterpret_cast<uint4 *>(mine + 2 * Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+    }
+    if (nlev > 3) {  // by four positions: two registers
+        const uint32_t b2 = __shfl_up_sync(0xFFFFFFFFu, t[2], 1), b3 = __shfl_up_sync(0xFFFFFFFFu, t[3], 1);
+        const uint32_t a0 = vmin2(t[0], b2), a1 = vmin2(t[1], b3), a2 = vmin2(t[2], t[0]), a3 = vmin2(t[3], t[1]);
+        t[0] = a0; t[1] = a1; t[2] = a2; t[3] = a3;
+        if (active) *reinterpret_cast<uint4 *>(mine + 3 * Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+    }
+    for (int s = 4; s < nlev; ++s) {  // by 8 * 2^(s-4) positions: whole lanes
+        const int dl = 1 << (s - 4);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) sfx[i * 32 + lane] = (uint16_t)(sv[i >> 1] >> (16 * (i & 1)));
-    *reinterpret_cast<uint4 *>(gs + 8 * lane) = make_uint4(r[0], r[1], r[2], r[3]);
-    uint32_t D = B;
-    T[lane] = (uint16_t)D;
-    min_shfl_up(D, D, 1); T[32 + lane] = (uint16_t)D;
-    min_shfl_up(D, D, 2); T[64 + lane] = (uint16_t)D;
-    min_shfl_up(D, D, 4); T[96 + lane] = (uint16_t)D;
-    min_shfl_up(D, D, 8); T[128 + lane] = (uint16_t)D;
+        for (int j = 0; j < 4; ++j) t[j] = vmin2(t[j], __shfl_up_sync(0xFFFFFFFFu, t[j], dl));
+        if (active) *reinterpret_cast<uint4 *>(mine + s * Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+    }
     __syncwarp();
-    // lanes beyond the row take empty windows whose lookups all hit the +inf entries
-    const uint4 none = make_uint4(0xFFA0A01Eu, 0xFFA0A01Eu, 0xFFA0A01Eu, 0xFFA0A01Eu);
-    const uint4 ma = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane) : none;
-    const uint4 mb = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane + 4) : none;
+    // lanes beyond the row take empty windows
+    const uint32_t none = (uint32_t)(nlev * Lpad * 2) * 0x10001u;
+    const uint4 ma = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane) : make_uint4(none, none, none, none);
+    const uint4 mb = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane + 4) : make_uint4(none, none, none, none);
     const uint32_t mw[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
-    const int base = 8 * lane;
+    const unsigned char *Tb = reinterpret_cast<const unsigned char *>(T);
     uint32_t val[8];
-    bool inblock = false;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const uint32_t w = mw[i];
-        const int a = (int)(w >> 24), c2 = base + i;
-        const uint32_t x = (xp[i >> 1] >> (16 * (i & 1))) & 0xFFFFu;
-        uint32_t v = min(min((uint32_t)sfx[w & 255u], (uint32_t)T[(w >> 8) & 255u]),
-                         min((uint32_t)T[(w >> 16) & 255u], x));
-        if (a >= c2) v = 0xFFFFu;           // empty window
-        else if (a >= base) inblock = true;  // window inside this lane's block: fixed below
-        val[i] = v;
-    }
-    if (__any_sync(0xFFFFFFFFu, inblock)) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int a = (int)(mw[i] >> 24), c2 = base + i;
-            if (a >= base && a < c2) {
-                uint32_t v = 0xFFFFu;
-                for (int c = a; c < c2; ++c) v = min(v, (uint32_t)gs[c]);
-                val[i] = v;
-            }
-        }
+        const uint32_t x = *reinterpret_cast<const uint16_t *>(Tb + (mw[i] & 0xFFFFu));
+        const uint32_t y = *reinterpret_cast<const uint16_t *>(Tb + (mw[i] >> 16));
+        val[i] = min(x, y);
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) o[j] = val[2 * j] | (val[2 * j + 1] << 16);
@@ -254,10 +242,11 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
         uint32_t *pad = gm_s + (threadIdx.x >> 5) * kTailWords;
         for (int i = threadIdx.x & 31; i < kTailWords; i += 32) pad[i] = kInf2;
     }
-    uint16_t *strips = reinterpret_cast<uint16_t *>(gm_s + k * Lpad) + (threadIdx.x >> 5) * kStripElems;
+    uint16_t *strips = reinterpret_cast<uint16_t *>(gm_s + k * Lpad) +
+                       (threadIdx.x >> 5) * gen_strip_elems(d.gen_levels, Lpad);
     if (GEN) {
         for (int i = threadIdx.x; i < k * Lpad; i += kFastThreads) gm_s[i] = d.gen_meta[i];
-        if ((threadIdx.x & 31) == 0) strips[512 + 160] = 0xFFFFu;  // the constant +inf of the T strip
+        if ((threadIdx.x & 31) == 0) strips[d.gen_levels * Lpad] = 0xFFFFu;  // the constant +inf behind the table
     }
     __syncthreads();
     asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
@@ -367,7 +356,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
             for (int t = 0; t < NT; ++t) mp[t] = wm + w[t];
             uint32_t o[NT][4];
             if (GEN)
-                window_min_general(r[0], gm_s + w[0] * Lpad, strips, strips + 256, strips + 512, lane, active, o[0]);
+                window_min_general(r[0], gm_s + w[0] * Lpad, strips, lane, active, d.gen_levels, Lpad, o[0]);
             else
                 window_min(r, mp, tl, o);
 #pragma unroll
@@ -418,7 +407,7 @@ size_t fast_smem_bytes(const Dev &d)
 {
     size_t b = (((size_t)d.k * d.k * d.Lpad * 2 + 512 + 15) & ~(size_t)15) + sizeof(WMeta) * PP_MAX_K;
     if (!d.fast_meta)  // general windows: lookup words + strips
-        b += (size_t)d.k * d.Lpad * 4 + (size_t)(512 / 32) * kStripElems * 2;
+        b += (size_t)d.k * d.Lpad * 4 + (size_t)(512 / 32) * gen_strip_elems(d.gen_levels, d.Lpad) * 2;
     else               // constant windows: suffix strips
         b += (size_t)(kMaxFastThreads / 32) * kTailWords * 4;
     return b;
@@ -478,27 +467,31 @@ bool fast_meta_build(int L, int k, const int16_t *lo, void *out)
     return true;
 }
 
-// Lookup words of the general window step (see window_min_general), row stride Lpad <= 240.
-void gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out)
+// Lookup words of the general window step (see window_min_general), row stride Lpad <= 240:
+// byte offsets into a warp's strip of T[s][c' - 1] (low half) and T[s][lo + 2^s - 1] (high half),
+// both the +inf element for an empty window.  Returns the number of table levels in use.
+int gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out)
 {
+    int maxlen = 1;
+    for (int w = 0; w < k; ++w)
+        for (int c2 = 0; c2 < L; ++c2) maxlen = std::max(maxlen, c2 - (int)lo[w * L + c2]);
+    int levels = 1;
+    while ((1 << levels) <= maxlen) ++levels;  // floor(log2(maxlen)) + 1
+    const uint32_t inf_off = (uint32_t)(levels * Lpad * 2);
     for (int w = 0; w < k; ++w)
         for (int c2 = 0; c2 < Lpad; ++c2) {
             const int a = c2 < L ? lo[w * L + c2] : c2;  // pads: empty window
-            const int lane = c2 >> 3, base = lane * 8;
-            uint32_t sfx = 30, t1 = 160, t2 = 160;      // the +inf entries
-            if (a < c2 && a < base) {
-                const int la = a >> 3, oa = a & 7;
-                sfx = (uint32_t)(oa * 32 + la);
-                const int n = lane - 1 - la;
-                if (n >= 1) {
-                    int s = 0;
-                    while ((2 << s) <= n) ++s;
-                    t1 = (uint32_t)(s * 32 + lane - 1);
-                    t2 = (uint32_t)(s * 32 + la + (1 << s));
-                }
+            const int len = c2 - a;
+            uint32_t o1 = inf_off, o2 = inf_off;
+            if (len > 0) {
+                int s = 0;
+                while ((2 << s) <= len) ++s;
+                o1 = (uint32_t)((s * Lpad + c2 - 1) * 2);
+                o2 = (uint32_t)((s * Lpad + a + (1 << s) - 1) * 2);
             }
-            out[w * Lpad + c2] = sfx | (t1 << 8) | (t2 << 16) | ((uint32_t)a << 24);
+            out[w * Lpad + c2] = o1 | (o2 << 16);
         }
+    return levels;
 }
 
 bool fast_sweep_supported(const Dev &d)

@@ -167,8 +167,9 @@ def test_register_tiled_sweep_on_uniform_memory_chains():
 
 def test_register_tiled_sweep_with_general_windows():
     # arbitrary layer memories: window starts come from the staged window table; includes
-    # windows inside one 8-position block, empty windows, windows reaching layer 0, L from one
-    # lane to 30 lanes, and every state compared on the small ones
+    # windows of one position up to the whole chain (every level count of the sparse table),
+    # empty windows, windows reaching layer 0, L from one lane to 30 lanes, and every state
+    # compared on the small ones
     seed = 0
     for L, k, n in ((5, 3, 8), (9, 4, 10), (17, 5, 10), (33, 6, 10), (64, 6, 6), (100, 7, 5), (150, 5, 5),
                     (199, 4, 5), (240, 4, 4), (12, 8, 6), (50, 10, 2)):
