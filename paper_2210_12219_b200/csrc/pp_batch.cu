@@ -1,5 +1,6 @@
 // Many-instance exact search: one thread block per instance, the whole state table in shared
-// memory as 16-bit ranks.  Same recurrence, final choice and backtrack rule as the
+// memory as 16-bit ranks (the quotients and the sort scratch of the ranking live in the same bytes
+// before the table is written).  Same recurrence, final choice and backtrack rule as the
 // single-instance path (see pp_sweep.cu); global memory sees the inputs once and the result
 // record once.
 //
@@ -19,7 +20,11 @@
 
 namespace pp {
 
-constexpr int kBatchThreads = 512;
+// Three blocks of 384 threads per SM (at k = 8, L = 24: 73 KB of shared memory and at most 56
+// registers per thread): the phases of an instance are short and separated by block barriers, so
+// what keeps an SM busy is the number of instances in flight on it.
+constexpr int kBatchThreads = 384;
+constexpr int kBatchBlocksPerSm = 3;
 constexpr int kBatchWarps = kBatchThreads / 32;
 constexpr uint16_t kInf16 = 0xFFFFu;
 
@@ -42,11 +47,8 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
                                                      // two neighbouring cut positions form one word
     size_t o = 0;
     auto take = [&o](size_t bytes) { size_t at = o; o = (o + bytes + 15) & ~(size_t)15; return at; };
-    b.gu = take(U * L * sizeof(double));
     size_t npad = 1;
     while (npad < U * L) npad <<= 1;
-    b.skey = take(npad * sizeof(unsigned long long));
-    b.sval = take(npad * sizeof(uint16_t));
     b.M = take((size_t)(L + 1) * sizeof(uint64_t));
     b.cap = take((size_t)k * sizeof(uint64_t));
     b.bits = take((size_t)L * sizeof(uint64_t));
@@ -59,11 +61,24 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     b.rowinfo = take(rows * sizeof(uint32_t));
     b.mlist = take(((size_t)1 << k) * sizeof(uint16_t));
     b.moff = take((size_t)(k + 2) * sizeof(uint32_t));
-    b.dp = take(rows * Ls * sizeof(uint16_t));
+    // The quotients, the sort scratch and the per-entry ranks are dead before the first state is
+    // written: they share the bytes of the state table.
+    {
+        auto up16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
+        const size_t scratch = up16(U * L * sizeof(double)) + up16(npad * sizeof(unsigned long long)) +
+                               up16(npad * sizeof(uint16_t)) + up16(U * L * sizeof(uint16_t)) +
+                               up16(U * L * sizeof(uint32_t));
+        const size_t table = rows * Ls * sizeof(uint16_t);
+        b.dp = take(table > scratch ? table : scratch);
+        size_t q = b.dp;
+        b.gu = q;   q += up16(U * L * sizeof(double));
+        b.skey = q; q += up16(npad * sizeof(unsigned long long));
+        b.sval = q; q += up16(npad * sizeof(uint16_t));
+        b.rk = q;   q += up16(U * L * sizeof(uint16_t));
+        b.cnt = q;
+    }
     b.g = take(best * Ls * sizeof(uint16_t));
     b.rank = take((size_t)k * k * Ls * sizeof(uint16_t));
-    b.rk = take(U * L * sizeof(uint16_t));
-    b.cnt = take(U * L * sizeof(uint32_t));
     b.pair_u = take((size_t)k * k * sizeof(int16_t));
     b.pos = take((size_t)L * sizeof(int16_t));
     b.lo = take((size_t)k * L * sizeof(int16_t));
@@ -177,7 +192,7 @@ __device__ __forceinline__ void batch_relax(const BatchRelaxArgs &a, int tid)
     }
 }
 
-__global__ void __launch_bounds__(kBatchThreads, 2)
+__global__ void __launch_bounds__(kBatchThreads, kBatchBlocksPerSm)
 k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
         const uint32_t *__restrict__ g_bw, double *__restrict__ o_beta, int32_t *__restrict__ o_m,
@@ -406,6 +421,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             const int u = pair_u[r];
             rank[e] = (u < 0 || c >= L) ? kInf16 : rk[u * L + pos[c]];
         }
+        __syncthreads();  // the per-entry ranks share their bytes with the state table
         // base frontier
         for (int e = tid; e < k * Ls; e += kBatchThreads) {
             const int v = e / Ls, c = e - v * Ls;
@@ -502,14 +518,17 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             int w = (int)(key & 31), c2 = L - 1;
             double bstar = 0.0;
             if (rstar != 0) {
+                // an entry of the rank table that carries the winning rank names a (node pair, layer)
+                // whose quotient is beta* (equal ranks hold equal doubles)
                 int found = -1;
-                for (int e = lane; e < U * L; e += 32)
-                    if (rk[e] == rstar) found = e;
+                for (int e = lane; e < k * k * Ls; e += 32)
+                    if (rank[e] == rstar) found = e;
                 for (int o = 16; o; o >>= 1) {
                     const int other = __shfl_xor_sync(0xFFFFFFFFu, found, o);
                     found = other > found ? other : found;
                 }
-                bstar = gu[found];  // equal ranks hold equal doubles
+                const int r = found / Ls, c = found - r * Ls;
+                bstar = __ddiv_rn((double)s_sorted[pos[c]], (double)ubw[pair_u[r]]);
             }
             if (lane == 0) {
                 o_beta[inst] = bstar;
