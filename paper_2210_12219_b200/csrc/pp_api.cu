@@ -17,7 +17,7 @@ using namespace pp;
 struct pp_problem {
     int L = 0, k = 0, Lpad = 0, U = 0, elem = 2;
     std::vector<uint64_t> bits, mem, cap, M;
-    std::vector<uint32_t> bw, ubw, masks, level_off;
+    std::vector<uint32_t> bw, ubw;
     std::vector<int16_t> lo, pair_u;
     unsigned char *d_inputs = nullptr;  // one allocation for all small device arrays
     unsigned char *d_work = nullptr;    // exact-search scratch (own or caller's)
@@ -80,6 +80,40 @@ const MaskList &mask_list(int k)
     ml.level_off[k + 1] = (uint32_t)ml.masks.size();
     ml.level_off[0] = 0;
     return cache.emplace(k, std::move(ml)).first->second;
+}
+
+// Device copy of a mask list, uploaded once per (device, k) and kept for the life of the process:
+// masks [2^k - 1] followed (256-byte aligned) by level_off [k + 2].
+struct DeviceMasks {
+    uint32_t *masks = nullptr, *level_off = nullptr;
+};
+cudaError_t device_masks(int k, const MaskList &ml, DeviceMasks *out)
+{
+    static std::mutex mu;
+    static std::map<std::pair<int, int>, DeviceMasks> cache;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find({dev, k});
+    if (it == cache.end()) {
+        const size_t mb = (ml.masks.size() * 4 + 255) / 256 * 256, lb = ml.level_off.size() * 4;
+        unsigned char *buf = nullptr;
+        e = cudaMalloc(reinterpret_cast<void **>(&buf), mb + lb);
+        if (e != cudaSuccess) return e;
+        e = cudaMemcpy(buf, ml.masks.data(), ml.masks.size() * 4, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(buf + mb, ml.level_off.data(), lb, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            cudaFree(buf);
+            return e;
+        }
+        DeviceMasks dm;
+        dm.masks = reinterpret_cast<uint32_t *>(buf);
+        dm.level_off = reinterpret_cast<uint32_t *>(buf + mb);
+        it = cache.emplace(std::make_pair(dev, k), dm).first;
+    }
+    *out = it->second;
+    return cudaSuccess;
 }
 
 // Staging buffers of the host-pointer entry points come from a pool of the library's own that
@@ -294,8 +328,6 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         p->Lpad = (L + per32 - 1) / per32 * per32;
         // masks by (popcount, value)
         const MaskList &ml = mask_list(k);
-        p->masks = ml.masks;
-        p->level_off = ml.level_off;
         p->mask_swaps = ml.swaps;
         p->pair_lvl.assign(k + 2, -1);
     } catch (const std::bad_alloc &) {
@@ -341,7 +373,7 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
         {p->cap.data(), p->cap.size() * 8, 0},         {p->bw.data(), p->bw.size() * 4, 0},
         {p->lo.data(), p->lo.size() * 2, 0},           {p->pair_u.data(), p->pair_u.size() * 2, 0},
         {p->ubw.data(), p->ubw.size() * 4, 0},
-        {p->masks.data(), p->masks.size() * 4, 0},     {p->level_off.data(), p->level_off.size() * 4, 0},
+        {nullptr, 0, 0} /* masks: shared */,           {nullptr, 0, 0} /* level_off: shared */,
         {nullptr, 8, 0} /* best */,                    {nullptr, 4, 0} /* err */,
         {nullptr, sizeof(pp_solution), 0} /* solution */,
         {fmeta.data(), fmeta.size(), 0},
@@ -359,7 +391,9 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     }
     for (auto &q : parts)
         if (q.src && q.bytes) std::memcpy(staging.data() + q.off, q.src, q.bytes);
-    cudaError_t e = staging_alloc(reinterpret_cast<void **>(&p->d_inputs), total, nullptr);
+    DeviceMasks dmasks;
+    cudaError_t e = device_masks(k, mask_list(k), &dmasks);
+    if (e == cudaSuccess) e = staging_alloc(reinterpret_cast<void **>(&p->d_inputs), total, nullptr);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_inputs, staging.data(), total, cudaMemcpyHostToDevice);
     for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreate(&p->ev[i]);
     if (e != cudaSuccess) {
@@ -377,8 +411,8 @@ pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
     d.lo = reinterpret_cast<int16_t *>(b + parts[4].off);
     d.pair_u = reinterpret_cast<int16_t *>(b + parts[5].off);
     d.ubw = reinterpret_cast<uint32_t *>(b + parts[6].off);
-    d.masks = reinterpret_cast<uint32_t *>(b + parts[7].off);
-    d.level_off = reinterpret_cast<uint32_t *>(b + parts[8].off);
+    d.masks = dmasks.masks;  // shared by every problem of this k on this device
+    d.level_off = dmasks.level_off;
     d.best = reinterpret_cast<unsigned long long *>(b + parts[9].off);
     d.err = reinterpret_cast<int32_t *>(b + parts[10].off);
     p->d_sol = reinterpret_cast<pp_solution *>(b + parts[11].off);
