@@ -100,6 +100,8 @@ typedef struct {
  * Validates, builds the uint64 memory prefix sums and the per-node window table (for each
  * node w and segment end c', the earliest segment start that still fits), uploads them.
  * *out receives the handle; free it with pp_problem_destroy.
+ * The list of node sets the search walks depends on k only: its device copy (4 * 2^k bytes) is
+ * made by the first problem of that k on a device and kept until the process ends.
  */
 pp_status pp_problem_create(int32_t L, const uint64_t *layer_out_bits,
                             const uint64_t *layer_mem_bytes, int32_t k,
