@@ -266,7 +266,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
     const int last_lane = (L - 1) >> 3, last_reg = ((L - 1) & 7) >> 1, last_sh = ((L - 1) & 1) * 16;
     const uint32_t stride = gridDim.x * (kFastThreads / 32);
 
-    uint32_t mi = blockIdx.x * (kFastThreads / 32) + warp;
+    uint32_t mi = warp * gridDim.x + blockIdx.x;  // items go round the blocks: a partial last round spreads over all SMs
     uint32_t S = mi < nmask ? d.masks[first + mi / split] : 0u;
     int voff[NV];
     uint4 dp[NV];

@@ -174,7 +174,9 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
     const uint4 inf4 = make_uint4(kInf2, kInf2, kInf2, kInf2);
     const uint32_t mask_rows = (uint32_t)(k * l8);  // pieces per mask
 
-    uint32_t pi = blockIdx.x * kWarps + warp;
+    // pair p goes to block p mod gridDim (round by round over the warp slots): the last, partial
+    // round is then spread over all SMs instead of filling a few of them
+    uint32_t pi = warp * gridDim.x + blockIdx.x;
     // sources: voff[0 .. NV-2] the common nodes T, voff[NV-1] = a (S1 only), voffb = b (S2 only);
     // offsets in elements from the start of a rank-table block or a mask's rows
     int voff[NV];
