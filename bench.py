@@ -39,7 +39,7 @@ UNIT = "relaxations/s"
 # DRAM bytes per sweep launch (18 launches per Large solve, base frontier included) from the ncu
 # capture summarised in profiles/sweep_dram_traffic_large.md; set to None whenever the sweep
 # kernels change after that capture.
-SWEEP_DRAM_BYTES_PER_LAUNCH = 94.81e6
+SWEEP_DRAM_BYTES_PER_LAUNCH = 94.83e6
 # Issue rate of packed 16-bit min/max measured on this part: 64 lanes per clock per SM, two
 # elements per lane (a three-input min/max issues at the same rate).
 PACKED_MINMAX_LANES_PER_CLK_SM = 64
