@@ -188,6 +188,7 @@ def run_ours(args):
     o_place = torch.empty(N_BATCH * BATCH_K, dtype=torch.int32, device=dev)
     o_stat = torch.empty(N_BATCH, dtype=torch.int8, device=dev)
     d_sol = torch.zeros(ctypes.sizeof(pp.pp_solution) // 8, dtype=torch.float64, device=dev)
+    d_sol2 = torch.zeros_like(d_sol)  # result record of the smaller configurations
 
     def batch_device():
         pp.solve_exact_batch_dev(N_BATCH, BATCH_L, BATCH_K, d_bb.data_ptr(), d_bm.data_ptr(),
@@ -256,6 +257,19 @@ def run_ours(args):
             stream.synchronize()
             batch_ms.append(e0.elapsed_time(e1))
             eval_ms.append(e1.elapsed_time(e2))
+
+        # the smaller named configurations (parity-test cases, not part of the timed step): device
+        # time of one exact solve each, for context
+        other = {}
+        for name, inst in (("tiny_k6_L12", W.config_tiny()), ("resnet50_shaped_k10_L50", W.config_resnet50_shaped()),
+                           ("deeper_cnn_k14_L100", W.config_deeper_cnn())):
+            with pp.Problem.from_instance(inst) as q:
+                q.set_stream(stream.cuda_stream)
+                ts = []
+                for _ in range(6):
+                    q.solve_exact_dev(d_sol2.data_ptr())
+                    ts.append(q.last_solve_profile().ms_total)
+                other[name] = {"solve_ms": min(ts[2:]), "relaxations_per_s": n_relax(inst.k, inst.L) / (min(ts[2:]) * 1e-3)}
 
     sol_rec = pp.pp_solution.from_buffer_copy(d_sol.cpu().numpy().tobytes())
     ms_per_step = ms_total / args.steps
@@ -340,6 +354,7 @@ def run_ours(args):
             "batch_ms": med(batch_ms), "instances_per_s": N_BATCH / (med(batch_ms) * 1e-3),
             "eval_ms": med(eval_ms), "plans_per_s": N_PLANS / (med(eval_ms) * 1e-3),
             "fast_path": prof.fast_path, "beta_ms": sol_rec.beta_ms, "segments": sol_rec.m,
+            "other_configs": other,
         },
     }
     if rank == 0 and world == 1 and not args.no_cpu:
