@@ -9,27 +9,33 @@
 
 namespace pp {
 
-// One block: order[] = layers sorted by (bits, index), pos[] = inverse permutation, then
+// order[] = layers sorted by (bits, index), pos[] = inverse permutation, then
 // gu[u][i] = bits[order[i]] / ubw[u], one correctly rounded fp64 division per entry (never
-// contracted, no fast math).
+// contracted, no fast math).  Every block works out the order for itself in shared memory (L is at
+// most 1024) and takes its share of the U * L quotients; block 0 also writes order[] and pos[].
 __global__ void __launch_bounds__(1024) k_order_quotients(Dev d)
 {
     extern __shared__ unsigned char smem_raw[];
-    uint64_t *sorted = reinterpret_cast<uint64_t *>(smem_raw);  // [L]
+    uint64_t *raw = reinterpret_cast<uint64_t *>(smem_raw);  // [L] bits by layer
+    uint64_t *sorted = raw + d.L;                            // [L] bits ascending
+    for (int c = threadIdx.x; c < d.L; c += blockDim.x) raw[c] = d.bits[c];
+    __syncthreads();
     for (int c = threadIdx.x; c < d.L; c += blockDim.x) {
-        uint64_t b = d.bits[c];
+        const uint64_t b = raw[c];
         int p = 0;
         for (int o = 0; o < d.L; ++o) {
-            uint64_t x = d.bits[o];
+            const uint64_t x = raw[o];
             p += (x < b) || (x == b && o < c);
         }
-        d.pos[c] = (int16_t)p;
-        d.order[p] = (int16_t)c;
         sorted[p] = b;
+        if (blockIdx.x == 0) {
+            d.pos[c] = (int16_t)p;
+            d.order[p] = (int16_t)c;
+        }
     }
     __syncthreads();
     const int n = d.U * d.L;
-    for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
         int u = e / d.L, i = e - u * d.L;
         d.gu[e] = __ddiv_rn((double)sorted[i], (double)d.ubw[u]);
     }
@@ -98,7 +104,13 @@ __global__ void k_expand(Dev d)
 cudaError_t launch_rank_build(const Dev &d, cudaStream_t s, int *launches)
 {
     *launches = 0;
-    k_order_quotients<<<1, 1024, (size_t)d.L * sizeof(uint64_t), s>>>(d);
+    {
+        const int n = d.U * d.L;
+        int blocks = (n + 1023) / 1024;
+        if (blocks < 1) blocks = 1;
+        if (blocks > 64) blocks = 64;
+        k_order_quotients<<<blocks, 1024, 2 * (size_t)d.L * sizeof(uint64_t), s>>>(d);
+    }
     ++*launches;
     if (d.U > 0) {
         int tile_lists = kRankTileBytes / (int)(d.L * sizeof(double));
