@@ -461,9 +461,13 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                     const bool has1 = c2 + 1 < L;
                     const int l1 = has1 ? lo[w * L + c2 + 1] : c2 + 1;
                     uint32_t head = kInf16, common = kInf16;
-                    const int split = l1 < c2 ? l1 : c2;
-                    for (int c = l0; c < split; ++c) head = min(head, (uint32_t)gr[c]);
-                    for (int c = l1; c < c2; ++c) common = min(common, (uint32_t)gr[c]);
+                    // one plain loop over [l0, c2-1]: the runs are a few positions long and differ from
+                    // lane to lane, so unrolled and split loops only add instructions
+#pragma unroll 1
+                    for (int c = l0; c < c2; ++c) {
+                        const uint32_t x = gr[c];
+                        if (c < l1) head = min(head, x); else common = min(common, x);
+                    }
                     const uint32_t out0 = min(head, common);
                     const uint32_t out1 = (has1 && l1 <= c2) ? min(common, (uint32_t)gr[c2]) : (uint32_t)kInf16;
                     reinterpret_cast<uint32_t *>(dp + (size_t)(row0 + rr) * Ls)[cw] = out0 | (out1 << 16);
