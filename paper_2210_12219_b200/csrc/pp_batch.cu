@@ -81,7 +81,7 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     b.rank = take((size_t)k * k * Ls * sizeof(uint16_t));
     b.pair_u = take((size_t)k * k * sizeof(int16_t));
     b.pos = take((size_t)L * sizeof(int16_t));
-    b.lo = take((size_t)k * L * sizeof(int16_t));
+    b.lo = take((size_t)k * Ls * sizeof(int16_t));  // row stride Ls: two window starts per 32-bit word
     b.total = o;
     return b;
 }
@@ -338,11 +338,11 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             for (int u2 = 0; u2 < U; ++u2) at += (ubw[u2] < ubw[u]);
             uord[at] = (int16_t)u;
         }
-        for (int e = tid; e < k * L; e += kBatchThreads) {
-            const int w = e / L, c2 = e - w * L;
+        for (int e = tid; e < k * Ls; e += kBatchThreads) {
+            const int w = e / Ls, c2 = e - w * Ls;
             int c = c2;  // step down while the segment starting at layer c (previous cut c-1) fits
-            while (c > 0 && M[c2 + 1] - M[c] <= cap[w]) --c;
-            lo[e] = (int16_t)c;
+            while (c2 < L && c > 0 && M[c2 + 1] - M[c] <= cap[w]) --c;
+            lo[e] = (int16_t)c;  // the pad of an odd L keeps c2: an empty window
         }
         // ---- 2. quotients and their ranks ----
         for (int e = tid; e < U * L; e += kBatchThreads) {
@@ -457,9 +457,8 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                     const int w = (rowinfo[row0 + rr] >> 12) & 15;
                     const uint16_t *gr = gbuf + rr * Ls;
                     const int c2 = 2 * cw;
-                    const int l0 = lo[w * L + c2];
-                    const bool has1 = c2 + 1 < L;
-                    const int l1 = has1 ? lo[w * L + c2 + 1] : c2 + 1;
+                    const uint32_t ll = reinterpret_cast<const uint32_t *>(lo)[w * Lh + cw];  // starts of c2, c2+1
+                    const int l0 = (int)(ll & 0xFFFFu), l1 = (int)(ll >> 16);
                     uint32_t head = kInf16, common = kInf16;
                     // one plain loop over [l0, c2-1]: the runs are a few positions long and differ from
                     // lane to lane, so unrolled and split loops only add instructions
@@ -469,8 +468,8 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                         if (c < l1) head = min(head, x); else common = min(common, x);
                     }
                     const uint32_t out0 = min(head, common);
-                    const uint32_t out1 = (has1 && l1 <= c2) ? min(common, (uint32_t)gr[c2]) : (uint32_t)kInf16;
-                    reinterpret_cast<uint32_t *>(dp + (size_t)(row0 + rr) * Ls)[cw] = out0 | (out1 << 16);
+                    const uint32_t out1 = l1 <= c2 ? min(common, (uint32_t)gr[c2]) : (uint32_t)kInf16;
+                    reinterpret_cast<uint32_t *>(dp)[(row0 + rr) * Lh + cw] = out0 | (out1 << 16);
                     rr += drA;
                     cw += dcA;
                     if (cw >= Lh) { cw -= Lh; ++rr; }
@@ -546,7 +545,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                 }
                 if (j == 0) break;
                 const uint32_t P = S & ~(1u << w);
-                const int l0 = lo[w * L + c2];
+                const int l0 = lo[w * Ls + c2];
                 unsigned int pick = 0xFFFFFFFFu;
                 for (int it = lane; it < (c2 - l0) * k; it += 32) {
                     const int c = l0 + it / k, v = it - (it / k) * k;
