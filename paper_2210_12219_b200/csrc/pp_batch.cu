@@ -29,8 +29,19 @@ constexpr int kBatchWarps = kBatchThreads / 32;
 constexpr uint16_t kInf16 = 0xFFFFu;
 
 struct BatchLayout {
-    size_t dp, g, rank, gu, rk, cnt, skey, sval, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, mlist, moff, total;
+    size_t dp, g, rank, rk, cnt, skey, sval, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, mlist, moff, total;
 };
+
+// Sort slots that one list of L quotients takes.  A list is ascending as it is computed, so for
+// L <= 32 it is laid out as a sorted run of the next power of two (padded with +inf keys) and the
+// sorting network starts at twice that size; longer lists are sorted from single keys.
+__host__ __device__ inline int batch_run_slots(int L)
+{
+    if (L > 32) return L;
+    int R = 1;
+    while (R < L) R <<= 1;
+    return R;
+}
 
 __host__ __device__ inline BatchLayout batch_layout(int L, int k)
 {
@@ -48,7 +59,7 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     size_t o = 0;
     auto take = [&o](size_t bytes) { size_t at = o; o = (o + bytes + 15) & ~(size_t)15; return at; };
     size_t npad = 1;
-    while (npad < U * L) npad <<= 1;
+    while (npad < U * batch_run_slots(L)) npad <<= 1;
     b.M = take((size_t)(L + 1) * sizeof(uint64_t));
     b.cap = take((size_t)k * sizeof(uint64_t));
     b.bits = take((size_t)L * sizeof(uint64_t));
@@ -61,17 +72,16 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     b.rowinfo = take(rows * sizeof(uint32_t));
     b.mlist = take(((size_t)1 << k) * sizeof(uint16_t));
     b.moff = take((size_t)(k + 2) * sizeof(uint32_t));
-    // The quotients, the sort scratch and the per-entry ranks are dead before the first state is
+    // The sort scratch and the per-entry ranks are dead before the first state is
     // written: they share the bytes of the state table.
     {
         auto up16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
-        const size_t scratch = up16(U * L * sizeof(double)) + up16(npad * sizeof(unsigned long long)) +
+        const size_t scratch = up16(npad * sizeof(unsigned long long)) +
                                up16(npad * sizeof(uint16_t)) + up16(U * L * sizeof(uint16_t)) +
                                up16(U * L * sizeof(uint32_t));
         const size_t table = rows * Ls * sizeof(uint16_t);
         b.dp = take(table > scratch ? table : scratch);
         size_t q = b.dp;
-        b.gu = q;   q += up16(U * L * sizeof(double));
         b.skey = q; q += up16(npad * sizeof(unsigned long long));
         b.sval = q; q += up16(npad * sizeof(uint16_t));
         b.rk = q;   q += up16(U * L * sizeof(uint16_t));
@@ -200,7 +210,6 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const BatchLayout lay = batch_layout(L, k);
-    double *gu = reinterpret_cast<double *>(smem + lay.gu);          // [U][L] ascending in i
     uint64_t *M = reinterpret_cast<uint64_t *>(smem + lay.M);
     uint64_t *cap = reinterpret_cast<uint64_t *>(smem + lay.cap);
     uint64_t *s_bits = reinterpret_cast<uint64_t *>(smem + lay.bits);
@@ -345,21 +354,35 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             lo[e] = (int16_t)c;  // the pad of an odd L keeps c2: an empty window
         }
         // ---- 2. quotients and their ranks ----
-        for (int e = tid; e < U * L; e += kBatchThreads) {
-            const int u = e / L, i = e - u * L;
-            gu[e] = __ddiv_rn((double)s_sorted[i], (double)ubw[u]);
-        }
-        __syncthreads();
         // Rank = 1 + number of quotients strictly below: bitonic sort of the bit patterns (positive
         // doubles order like unsigned integers) with the entry index as payload, then every run of
         // equal keys takes the position of its first element.
         {
+            // Entry e = u * L + i is bits[order[i]] / ubw[u], ascending in i.  With runs, list u takes
+            // the R slots from u * R, in descending order when u is odd: the network then starts
+            // from bitonic blocks of 2 R keys.  Pads carry the largest key and end up behind the
+            // n real entries; they all compare equal, which a compare-exchange leaves alone.
             const int n = U * L;
+            const int R = batch_run_slots(L);
+            const bool runs = L <= 32;
+            const int rshift = 31 - __clz(R);
             int npad = 1;
-            while (npad < n) npad <<= 1;
+            while (npad < U * R) npad <<= 1;
             for (int i = tid; i < npad; i += kBatchThreads) {
-                skey[i] = i < n ? (unsigned long long)__double_as_longlong(gu[i]) : ~0ull;
-                sval[i] = (uint16_t)i;
+                int u, ii;
+                if (runs) {
+                    u = i >> rshift;
+                    ii = i & (R - 1);
+                    if (u & 1) ii = R - 1 - ii;
+                } else {
+                    u = i / L;
+                    ii = i - u * L;
+                }
+                const bool real = u < U && ii < L;
+                skey[i] = real ? (unsigned long long)__double_as_longlong(
+                                     __ddiv_rn((double)s_sorted[ii], (double)ubw[u]))
+                               : ~0ull;
+                sval[i] = real ? (uint16_t)(u * L + ii) : kInf16;
             }
             __syncthreads();
             if (npad >= 64) {
@@ -367,7 +390,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
                 // with stride <= 32 (shuffles, no block barrier); only strides >= 64 go through
                 // shared memory with a barrier each.
                 const int tiles = npad >> 6;
-                for (int t = wid; t < tiles; t += kBatchWarps) sort_tile(skey, sval, t << 6, lane, 2, 64);
+                for (int t = wid; t < tiles; t += kBatchWarps) sort_tile(skey, sval, t << 6, lane, runs ? 2 * R : 2, 64);
                 __syncthreads();
                 for (int size = 128; size <= npad; size <<= 1) {
                     for (int stride = size >> 1; stride >= 64; stride >>= 1) {
