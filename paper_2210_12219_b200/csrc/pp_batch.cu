@@ -1,5 +1,5 @@
 // Many-instance exact search: one thread block per instance, the whole state table in shared
-// memory as 16-bit ranks (the quotients and the sort scratch of the ranking live in the same bytes
+// memory as 16-bit ranks (the sort scratch and the per-entry ranks of the ranking live in the same bytes
 // before the table is written).  Same recurrence, final choice and backtrack rule as the
 // single-instance path (see pp_sweep.cu); global memory sees the inputs once and the result
 // record once.
@@ -8,7 +8,8 @@
 //   1. stages the inputs, builds the memory prefix sums and the window table lo[w][c'];
 //   2. rank-compresses gamma (Eq. 3): layers sorted by bits, distinct bandwidths listed, one fp64
 //      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, obtained by
-//      a bitonic sort of all quotients (64-key tiles in registers, the wide strides in shared memory);
+//      a bitonic sort of all quotients (64-key tiles in registers, the wide strides in shared memory;
+//      chains of up to 32 layers enter as the sorted runs they already are);
 //   3. sweeps the popcount levels with a flat thread <-> (target row, position) mapping:
 //      phase A forms g[c] = min_v max(dp[S'\{w}][v][c], rank[v][w][c]) for every row of the level,
 //      two neighbouring positions per thread as one packed u16x2 word, thread <-> (source mask,
