@@ -167,7 +167,7 @@ pp_status pp_eval_plans_dev(pp_problem *p, int64_t B, const uint8_t *nseg, const
  *   or PP_ERR_LIMIT for an instance with a value above the limits)
  * Returns PP_ERR_LIMIT without touching outputs when the instance shape does not fit one block:
  * k > 12, k*(k-1)*L + 1 > 65534 (ranks are 16-bit), or k * 2^(k-1) * L 16-bit states plus the
- * rank and quotient tables beyond the shared memory of a block (k = 8, L = 24 needs 90 KB).  Host variant is synchronous and uses the
+ * rank tables beyond the shared memory of a block (k = 8, L = 24 needs 73 KB).  Host variant is synchronous and uses the
  * legacy default stream; the _dev variant takes device pointers and a stream and is
  * asynchronous.  cuts may be NULL when k == 1.
  */
@@ -179,6 +179,30 @@ pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64
                                    const uint64_t *mem, const uint64_t *node_mem,
                                    const uint32_t *bw, double *beta_ms, int32_t *m, int32_t *cuts,
                                    int32_t *placement, int8_t *status, void *cuda_stream);
+
+/*
+ * Greedy comparison baseline of Section 4 (second algorithm of the paper's comparison list), for
+ * many independent instances of the same shape; arguments, layouts and outputs as for
+ * pp_solve_exact_batch, any L <= PP_MAX_L and k <= PP_MAX_K.  For every start node n: (a) on the
+ * current node, among the segments that start at the next unassigned layer and fit the node's
+ * memory, take the one with the smallest outgoing transfer; (b) move to the unused node behind
+ * the current node's fastest outgoing link; repeat until the chain is used up; (c) keep the start
+ * node with the smallest bottleneck latency (Eq. 2, Eq. 3).  Where the paper is silent: a segment
+ * that reaches the last layer transfers nothing and is taken as soon as it fits; equal transfers
+ * take the longer segment, equal links the lower node, equal bottlenecks the lower start node;
+ * bandwidth 0 is no link.  status[b] is PP_OK, or PP_INFEASIBLE when every walk gets stuck (the
+ * heuristic found no plan; the exact search may still find one); then beta_ms = +inf, m = 0 and
+ * the plan rows are -1.  Host variant: synchronous, legacy default stream.  _dev variant: device
+ * pointers, asynchronous on `cuda_stream`.  cuts may be NULL when k == 1.
+ */
+pp_status pp_greedy_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                          const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
+                          double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
+                          int8_t *status);
+pp_status pp_greedy_batch_dev(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                              const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
+                              double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
+                              int8_t *status, void *cuda_stream);
 
 /* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream. */
 pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out);

@@ -25,7 +25,8 @@ EXPORTS = (
     "pp_problem_workspace_bytes", "pp_problem_set_workspace", "pp_solve_exact",
     "pp_solve_exact_dev", "pp_eval_plans", "pp_eval_plans_dev", "pp_solve_exact_batch",
     "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row", "pp_debug_mask_order",
-    "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str",
+    "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str", "pp_greedy_batch",
+    "pp_greedy_batch_dev",
 )
 
 
@@ -72,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.pp_eval_plans_dev.argtypes = [vp, i64, vp, vp, vp, vp, vp]
         L.pp_solve_exact_batch.argtypes = [i64, i32, i32] + [vp] * 9
         L.pp_solve_exact_batch_dev.argtypes = [i64, i32, i32] + [vp] * 10
+        L.pp_greedy_batch.argtypes = [i64, i32, i32] + [vp] * 9
+        L.pp_greedy_batch_dev.argtypes = [i64, i32, i32] + [vp] * 10
         L.pp_last_solve_profile.argtypes = [vp, ctypes.POINTER(pp_profile)]
         L.pp_debug_read_state_row.argtypes = [vp, ctypes.c_uint32, i32, vp]
         L.pp_debug_mask_order.argtypes = [i32, vp, vp]
@@ -230,6 +233,15 @@ class BatchSolution:
 
 def solve_exact_batch(L, k, out_bits, mem, node_mem, bw) -> BatchSolution:
     """Host arrays [B, L], [B, L], [B, k], [B, k, k] -> BatchSolution (synchronous)."""
+    return _batch_from_host("pp_solve_exact_batch", L, k, out_bits, mem, node_mem, bw)
+
+
+def greedy_batch(L, k, out_bits, mem, node_mem, bw) -> BatchSolution:
+    """pp_greedy_batch: the greedy comparison baseline on the same host arrays (synchronous)."""
+    return _batch_from_host("pp_greedy_batch", L, k, out_bits, mem, node_mem, bw)
+
+
+def _batch_from_host(entry, L, k, out_bits, mem, node_mem, bw) -> BatchSolution:
     out_bits, p0 = _host(out_bits, np.uint64)
     B = out_bits.shape[0]
     mem, p1 = _host(mem, np.uint64)
@@ -241,9 +253,9 @@ def solve_exact_batch(L, k, out_bits, mem, node_mem, bw) -> BatchSolution:
     cuts = np.full((B, max(k - 1, 1)), -1, dtype=np.int32)
     placement = np.empty((B, k), dtype=np.int32)
     status = np.empty(B, dtype=np.int8)
-    st = lib().pp_solve_exact_batch(B, L, k, p0, p1, p2, p3, *(ctypes.c_void_p(a.ctypes.data) for a in
-                                    (beta, m, cuts, placement, status)))
-    _check(st, "pp_solve_exact_batch")
+    st = getattr(lib(), entry)(B, L, k, p0, p1, p2, p3, *(ctypes.c_void_p(a.ctypes.data) for a in
+                                                          (beta, m, cuts, placement, status)))
+    _check(st, entry)
     return BatchSolution(beta, m, cuts[:, : max(k - 1, 0)] if k > 1 else cuts[:, :0], placement, status)
 
 
@@ -262,6 +274,14 @@ def solve_exact_batch_dev(B, L, k, bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta
         bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr, placement_ptr, status_ptr,
         cuda_stream)))
     _check(st, "pp_solve_exact_batch_dev")
+
+
+def greedy_batch_dev(B, L, k, bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr,
+                     placement_ptr, status_ptr, cuda_stream: int = 0):
+    st = lib().pp_greedy_batch_dev(int(B), int(L), int(k), *(ctypes.c_void_p(x) for x in (
+        bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr, placement_ptr, status_ptr,
+        cuda_stream)))
+    _check(st, "pp_greedy_batch_dev")
 
 
 def solve_exact_static(L, layer_out_bits, layer_mem_bytes, k, node_mem_bytes, bw_kbps,

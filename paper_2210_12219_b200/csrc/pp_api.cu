@@ -571,10 +571,16 @@ pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64
     return PP_OK;
 }
 
-pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
-                               const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
-                               double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
-                               int8_t *status)
+// Host-pointer form of a batched entry point: stage the inputs, run the device-pointer form on
+// the legacy default stream, bring the results back.
+typedef pp_status (*batch_dev_fn)(int64_t, int32_t, int32_t, const uint64_t *, const uint64_t *,
+                                  const uint64_t *, const uint32_t *, double *, int32_t *, int32_t *,
+                                  int32_t *, int8_t *, void *);
+
+static pp_status batch_from_host(batch_dev_fn run_dev, int64_t B, int32_t L, int32_t k,
+                                 const uint64_t *out_bits, const uint64_t *mem, const uint64_t *node_mem,
+                                 const uint32_t *bw, double *beta_ms, int32_t *m, int32_t *cuts,
+                                 int32_t *placement, int8_t *status)
 {
     if (B < 0 || L < 1 || k < 1) return PP_ERR_ARG;
     if (L > PP_MAX_L || k > PP_MAX_K) return PP_ERR_LIMIT;
@@ -597,15 +603,11 @@ pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *
         e = cudaMemcpyAsync(buf + off[i], src[i], sz[i], cudaMemcpyHostToDevice, s);
     pp_status st = PP_OK;
     if (e == cudaSuccess)
-        st = pp_solve_exact_batch_dev(B, L, k, reinterpret_cast<uint64_t *>(buf + off[0]),
-                                      reinterpret_cast<uint64_t *>(buf + off[1]),
-                                      reinterpret_cast<uint64_t *>(buf + off[2]),
-                                      reinterpret_cast<uint32_t *>(buf + off[3]),
-                                      reinterpret_cast<double *>(buf + off[4]),
-                                      reinterpret_cast<int32_t *>(buf + off[5]),
-                                      reinterpret_cast<int32_t *>(buf + off[6]),
-                                      reinterpret_cast<int32_t *>(buf + off[7]),
-                                      reinterpret_cast<int8_t *>(buf + off[8]), s);
+        st = run_dev(B, L, k, reinterpret_cast<uint64_t *>(buf + off[0]),
+                     reinterpret_cast<uint64_t *>(buf + off[1]), reinterpret_cast<uint64_t *>(buf + off[2]),
+                     reinterpret_cast<uint32_t *>(buf + off[3]), reinterpret_cast<double *>(buf + off[4]),
+                     reinterpret_cast<int32_t *>(buf + off[5]), reinterpret_cast<int32_t *>(buf + off[6]),
+                     reinterpret_cast<int32_t *>(buf + off[7]), reinterpret_cast<int8_t *>(buf + off[8]), s);
     if (e == cudaSuccess && st == PP_OK) {
         void *dst[5] = {beta_ms, m, cuts, placement, status};
         for (int i = 0; i < 5 && e == cudaSuccess; ++i) {
@@ -619,6 +621,39 @@ pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *
     if (st != PP_OK) return st;
     if (e != cudaSuccess) return from_cuda(e);
     return from_cuda(e2);
+}
+
+pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                               const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
+                               double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
+                               int8_t *status)
+{
+    return batch_from_host(pp_solve_exact_batch_dev, B, L, k, out_bits, mem, node_mem, bw, beta_ms, m, cuts,
+                           placement, status);
+}
+
+pp_status pp_greedy_batch_dev(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                              const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
+                              double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
+                              int8_t *status, void *cuda_stream)
+{
+    if (B < 0 || L < 1 || k < 1) return PP_ERR_ARG;
+    if (L > PP_MAX_L || k > PP_MAX_K) return PP_ERR_LIMIT;
+    if (B == 0) return PP_OK;
+    if (!out_bits || !mem || !node_mem || !bw || !beta_ms || !m || !placement || !status ||
+        (!cuts && k > 1))
+        return PP_ERR_ARG;
+    PP_CUDA(launch_greedy(B, L, k, out_bits, mem, node_mem, bw, beta_ms, m, cuts, placement, status,
+                          static_cast<cudaStream_t>(cuda_stream)));
+    return PP_OK;
+}
+
+pp_status pp_greedy_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
+                          const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
+                          double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement, int8_t *status)
+{
+    return batch_from_host(pp_greedy_batch_dev, B, L, k, out_bits, mem, node_mem, bw, beta_ms, m, cuts,
+                           placement, status);
 }
 
 pp_status pp_debug_mask_order(int32_t k, uint32_t *masks_out, uint32_t *level_off_out)

@@ -1,0 +1,126 @@
+// Greedy comparison baseline of Section 4 (the "joint-optimization" algorithm of the paper's
+// comparison list), many instances per launch: one warp per instance, lane n walks from start
+// node n.
+//
+// A walk alternates two steps until the chain is used up: (a) on the current node, among the
+// segments that start at the next unassigned layer and fit the node's memory, take the one whose
+// outgoing transfer is smallest; (b) move to the unused node behind the current node's fastest
+// outgoing link.  Step (c) keeps the walk with the smallest bottleneck latency (Eq. 2 with one
+// correctly rounded fp64 division per cut, Eq. 3).  Where the paper is silent: a segment that
+// reaches the last layer transfers nothing and is taken as soon as it fits; equal transfers take
+// the longer segment, equal links the lower node, equal bottlenecks the lower start node; a link
+// of bandwidth 0 is no link; a walk that gets stuck contributes no plan.
+//
+// The work of an instance is a few hundred dependent scalar steps, so the kernel is bound by
+// latency, not by bandwidth or arithmetic; instances in flight hide it.
+#include "pp_internal.cuh"
+
+namespace pp {
+
+constexpr int kGreedyWarps = 4;
+
+__global__ void __launch_bounds__(kGreedyWarps * 32)
+k_greedy_batch(int64_t B, int L, int k, const uint64_t *__restrict__ bits, const uint64_t *__restrict__ mem,
+               const uint64_t *__restrict__ cap, const uint32_t *__restrict__ bw, double *o_beta,
+               int32_t *o_m, int32_t *o_cuts, int32_t *o_place, int8_t *o_status)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t inst = (int64_t)blockIdx.x * kGreedyWarps + (threadIdx.x >> 5);
+    if (inst >= B) return;  // the whole warp leaves together
+    const uint64_t *b = bits + inst * L, *mm = mem + inst * L, *cp = cap + inst * k;
+    const uint32_t *links = bw + inst * k * k;
+    int cuts[PP_MAX_K], nodes[PP_MAX_K];
+    int nseg = 0;
+    double beta = 0.0;
+    bool arrived = false;
+    if (lane < k) {
+        uint32_t used = 1u << lane;
+        int node = lane, first = 0;
+        nodes[0] = lane;
+        nseg = 1;
+        for (;;) {
+            // (a) held never exceeds the capacity, so the sum cannot wrap
+            const uint64_t room = cp[node];
+            uint64_t held = 0, transfer = 0;
+            int chosen = -1;
+            for (int e = first; e < L; ++e) {
+                const uint64_t need = mm[e];
+                if (need > room - held) break;
+                held += need;
+                const uint64_t x = b[e];
+                if (e == L - 1 || chosen < 0 || x <= transfer) {
+                    chosen = e;
+                    transfer = x;
+                }
+            }
+            if (chosen < 0) break;
+            if (chosen == L - 1) {
+                arrived = true;
+                break;
+            }
+            // (b) strictly faster links only: the lowest node wins a tie, a zero link never wins
+            int next = -1;
+            uint32_t fastest = 0;
+            for (int w = 0; w < k; ++w) {
+                const uint32_t x = links[node * k + w];
+                if (!((used >> w) & 1u) && x > fastest) {
+                    next = w;
+                    fastest = x;
+                }
+            }
+            if (next < 0) break;
+            const double g = __ddiv_rn((double)transfer, (double)fastest);
+            beta = g > beta ? g : beta;
+            cuts[nseg - 1] = chosen;
+            nodes[nseg] = next;
+            ++nseg;
+            used |= 1u << next;
+            node = next;
+            first = chosen + 1;
+        }
+    }
+    // (c) smallest (beta, start node); beta >= +0.0, so its bit pattern orders like the value
+    unsigned long long key = arrived ? (unsigned long long)__double_as_longlong(beta) : ~0ull;
+    int who = lane;
+    for (int o = 16; o; o >>= 1) {
+        const unsigned long long okey = __shfl_xor_sync(0xFFFFFFFFu, key, o);
+        const int owho = __shfl_xor_sync(0xFFFFFFFFu, who, o);
+        if (okey < key || (okey == key && owho < who)) {
+            key = okey;
+            who = owho;
+        }
+    }
+    int32_t *oc = o_cuts ? o_cuts + inst * (k - 1) : nullptr;
+    int32_t *op = o_place + inst * k;
+    if (key == ~0ull) {
+        if (lane == 0) {
+            o_beta[inst] = __longlong_as_double(0x7FF0000000000000ll);
+            o_m[inst] = 0;
+            o_status[inst] = (int8_t)PP_INFEASIBLE;
+        }
+        if (lane < k) op[lane] = -1;
+        if (oc && lane < k - 1) oc[lane] = -1;
+        return;
+    }
+    if (lane == who) {
+        o_beta[inst] = beta;
+        o_m[inst] = nseg;
+        o_status[inst] = (int8_t)PP_OK;
+        for (int i = 0; i < k; ++i) op[i] = i < nseg ? nodes[i] : -1;
+        if (oc)
+            for (int i = 0; i < k - 1; ++i) oc[i] = i < nseg - 1 ? cuts[i] : -1;
+    }
+}
+
+cudaError_t launch_greedy(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                          const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m, int32_t *cuts,
+                          int32_t *place, int8_t *status, cudaStream_t s)
+{
+    const int64_t blocks = (B + kGreedyWarps - 1) / kGreedyWarps;
+    if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    k_greedy_batch<<<(unsigned)blocks, kGreedyWarps * 32, 0, s>>>(B, L, k, bits, mem, cap, bw, beta, m, cuts,
+                                                                  place, status);
+    return cudaGetLastError();
+}
+
+}  // namespace pp

@@ -78,6 +78,10 @@ def test_null_handles_are_rejected(lib):
     assert lib.pp_solve_exact_batch(-1, 4, 2, *([None] * 9)) == binding.PP_ERR_ARG
     assert lib.pp_solve_exact_batch(1, 4, 30, *([None] * 9)) == binding.PP_ERR_LIMIT
     assert lib.pp_solve_exact_batch(0, 4, 2, *([None] * 9)) == binding.PP_OK
+    assert lib.pp_greedy_batch(-1, 4, 2, *([None] * 9)) == binding.PP_ERR_ARG
+    assert lib.pp_greedy_batch(1, 4, 30, *([None] * 9)) == binding.PP_ERR_LIMIT
+    assert lib.pp_greedy_batch(0, 4, 2, *([None] * 9)) == binding.PP_OK
+    assert lib.pp_greedy_batch_dev(1, 4, 2, *([None] * 10)) == binding.PP_ERR_ARG
 
 
 def test_no_cpu_fallback_without_device(lib):
