@@ -258,6 +258,28 @@ def run_ours(args):
             batch_ms.append(e0.elapsed_time(e1))
             eval_ms.append(e1.elapsed_time(e2))
 
+        # the paper's greedy comparison baseline on the batched instances (not part of the timed
+        # step): device time of one launch, and how far its plans are from the exact optimum
+        g_beta, g_m, g_stat = torch.empty_like(o_beta), torch.empty_like(o_m), torch.empty_like(o_stat)
+        g_cuts, g_place = torch.empty_like(o_cuts), torch.empty_like(o_place)
+        greedy_ms = []
+        for _ in range(7):
+            e0.record(stream)
+            pp.greedy_batch_dev(N_BATCH, BATCH_L, BATCH_K, d_bb.data_ptr(), d_bm.data_ptr(), d_bc.data_ptr(),
+                                d_bbw.data_ptr(), g_beta.data_ptr(), g_m.data_ptr(), g_cuts.data_ptr(),
+                                g_place.data_ptr(), g_stat.data_ptr(), stream.cuda_stream)
+            e1.record(stream)
+            stream.synchronize()
+            greedy_ms.append(e0.elapsed_time(e1))
+        both = (g_stat == 0) & (o_stat == 0) & (o_beta > 0)
+        ratio = (g_beta[both] / o_beta[both]).cpu().numpy()
+        greedy = {"launch_ms": min(greedy_ms[2:]), "instances_per_s": N_BATCH / (min(greedy_ms[2:]) * 1e-3),
+                  "plans_found": int((g_stat == 0).sum().item()),
+                  "plans_found_by_exact_search": int((o_stat == 0).sum().item()),
+                  "beta_over_optimum_median": float(np.median(ratio)) if ratio.size else None,
+                  "beta_over_optimum_mean": float(ratio.mean()) if ratio.size else None,
+                  "optimal_fraction": float((ratio == 1.0).mean()) if ratio.size else None}
+
         # the smaller named configurations (parity-test cases, not part of the timed step): device
         # time of one exact solve each, for context
         other = {}
@@ -354,6 +376,7 @@ def run_ours(args):
             "batch_ms": med(batch_ms), "instances_per_s": N_BATCH / (med(batch_ms) * 1e-3),
             "eval_ms": med(eval_ms), "plans_per_s": N_PLANS / (med(eval_ms) * 1e-3),
             "fast_path": prof.fast_path, "beta_ms": sol_rec.beta_ms, "segments": sol_rec.m,
+            "greedy_baseline_batched": greedy,
             "other_configs": other,
         },
     }

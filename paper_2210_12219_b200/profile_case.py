@@ -2,6 +2,7 @@
 
     python -m paper_2210_12219_b200.profile_case --k 16 --solves 2
     python -m paper_2210_12219_b200.profile_case --batch 4096 --solves 1
+    python -m paper_2210_12219_b200.profile_case --batch 65536 --greedy --solves 1
 
 With k = 16 the state table is 0.44 GB (still far above the 126 MB L2), small enough for a
 multi-pass counter capture of single sweep launches.
@@ -26,15 +27,17 @@ def main():
     ap.add_argument("--solves", type=int, default=2)
     ap.add_argument("--generic", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="solve this many batched instances instead")
+    ap.add_argument("--greedy", action="store_true", help="with --batch: the greedy comparison baseline")
     args = ap.parse_args()
     build.build()
     if args.batch:
         insts = W.config_batched(args.batch)
         stack = lambda f: np.stack([f(i) for i in insts])
+        entry = pp.greedy_batch if args.greedy else pp.solve_exact_batch
         for _ in range(args.solves):
-            got = pp.solve_exact_batch(24, 8, stack(lambda i: i.layer_out_bits), stack(lambda i: i.layer_mem_bytes),
-                                       stack(lambda i: i.node_mem_bytes), stack(lambda i: i.bw_kbps))
-        print("batch of %d: %d feasible" % (args.batch, int((got.status == 0).sum())))
+            got = entry(24, 8, stack(lambda i: i.layer_out_bits), stack(lambda i: i.layer_mem_bytes),
+                        stack(lambda i: i.node_mem_bytes), stack(lambda i: i.bw_kbps))
+        print("batch of %d: %d with a plan" % (args.batch, int((got.status == 0).sum())))
         return
     large = W.config_large()
     k = args.k
