@@ -181,6 +181,26 @@ pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64
                                    int32_t *placement, int8_t *status, void *cuda_stream);
 
 /*
+ * Random comparison baseline of Section 4 (first algorithm of the paper's comparison list) as a
+ * generator of P candidate plans of one problem, in the evaluator's input layout.  Step s of a
+ * plan takes a random node among the nodes not used yet and a random segment among those that
+ * start at the next unassigned layer and fit that node's memory, until the chain is used up.
+ *   draws [P*2k]  32-bit random numbers supplied by the caller; row p, word 2s chooses the node of
+ *                 step s, word 2s+1 its segment; a draw d picks index floor(d * n / 2^32) among n
+ *                 candidates in ascending order (both choices uniform: the paper does not say)
+ *   nseg [P], ends [P*k], nodes [P*k]   out: as pp_eval_plans reads them, unused entries -1;
+ *                 nseg = 0 (a row the evaluator flags PP_PLAN_BAD_NSEG) when the chosen node holds
+ *                 not even the next layer or when all k nodes are used and layers are left over
+ * Bandwidths play no part; score the plans with pp_eval_plans.  pp_random_plans takes host
+ * pointers and is synchronous; pp_random_plans_dev takes device pointers and is asynchronous on
+ * the problem's stream.  P == 0 is a no-op.
+ */
+pp_status pp_random_plans(pp_problem *p, int64_t P, const uint32_t *draws, uint8_t *nseg, int32_t *ends,
+                          int32_t *nodes);
+pp_status pp_random_plans_dev(pp_problem *p, int64_t P, const uint32_t *draws, uint8_t *nseg,
+                              int32_t *ends, int32_t *nodes);
+
+/*
  * Greedy comparison baseline of Section 4 (second algorithm of the paper's comparison list), for
  * many independent instances of the same shape; arguments, layouts and outputs as for
  * pp_solve_exact_batch, any L <= PP_MAX_L and k <= PP_MAX_K.  For every start node n: (a) on the

@@ -26,7 +26,7 @@ EXPORTS = (
     "pp_solve_exact_dev", "pp_eval_plans", "pp_eval_plans_dev", "pp_solve_exact_batch",
     "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row", "pp_debug_mask_order",
     "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str", "pp_greedy_batch",
-    "pp_greedy_batch_dev",
+    "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev",
 )
 
 
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.pp_solve_exact_batch.argtypes = [i64, i32, i32] + [vp] * 9
         L.pp_solve_exact_batch_dev.argtypes = [i64, i32, i32] + [vp] * 10
         L.pp_greedy_batch.argtypes = [i64, i32, i32] + [vp] * 9
+        L.pp_random_plans.argtypes = [vp, i64] + [vp] * 4
+        L.pp_random_plans_dev.argtypes = [vp, i64] + [vp] * 4
         L.pp_greedy_batch_dev.argtypes = [i64, i32, i32] + [vp] * 10
         L.pp_last_solve_profile.argtypes = [vp, ctypes.POINTER(pp_profile)]
         L.pp_debug_read_state_row.argtypes = [vp, ctypes.c_uint32, i32, vp]
@@ -215,6 +217,23 @@ class Problem:
         _check(lib().pp_eval_plans_dev(self._h, int(B), *(ctypes.c_void_p(x) for x in
                                        (nseg_ptr, ends_ptr, nodes_ptr, beta_ptr, status_ptr))),
                "pp_eval_plans_dev")
+
+    # -- random comparison baseline -------------------------------------------------------
+    def random_plans(self, draws):
+        """pp_random_plans: uint32 draws [P, 2k] -> (nseg uint8 [P], ends int32 [P, k], nodes int32 [P, k])."""
+        draws, p0 = _host(draws, np.uint32)
+        assert draws.ndim == 2 and draws.shape[1] == 2 * self.k
+        P = draws.shape[0]
+        nseg = np.empty(P, dtype=np.uint8)
+        ends = np.empty((P, self.k), dtype=np.int32)
+        nodes = np.empty((P, self.k), dtype=np.int32)
+        _check(lib().pp_random_plans(self._h, P, p0, *(ctypes.c_void_p(a.ctypes.data) for a in (nseg, ends, nodes))),
+               "pp_random_plans")
+        return nseg, ends, nodes
+
+    def random_plans_dev(self, P, draws_ptr, nseg_ptr, ends_ptr, nodes_ptr):
+        _check(lib().pp_random_plans_dev(self._h, int(P), *(ctypes.c_void_p(x) for x in
+                                         (draws_ptr, nseg_ptr, ends_ptr, nodes_ptr))), "pp_random_plans_dev")
 
 
 @dataclass

@@ -551,6 +551,43 @@ pp_status pp_eval_plans(pp_problem *p, int64_t B, const uint8_t *nseg, const int
     return from_cuda(e2);
 }
 
+pp_status pp_random_plans_dev(pp_problem *p, int64_t P, const uint32_t *draws, uint8_t *nseg, int32_t *ends,
+                              int32_t *nodes)
+{
+    if (!p || P < 0) return PP_ERR_ARG;
+    if (P == 0) return PP_OK;
+    if (!draws || !nseg || !ends || !nodes) return PP_ERR_ARG;
+    PP_CUDA(launch_random_plans(p->d, P, draws, nseg, ends, nodes, p->stream));
+    return PP_OK;
+}
+
+pp_status pp_random_plans(pp_problem *p, int64_t P, const uint32_t *draws, uint8_t *nseg, int32_t *ends,
+                          int32_t *nodes)
+{
+    if (!p || P < 0) return PP_ERR_ARG;
+    if (P == 0) return PP_OK;
+    if (!draws || !nseg || !ends || !nodes) return PP_ERR_ARG;
+    const size_t k = p->k;
+    const size_t b_draws = (size_t)P * 2 * k * 4, b_rows = (size_t)P * k * 4;
+    const size_t o_ends = align_up(b_draws, 256), o_nodes = align_up(o_ends + b_rows, 256);
+    const size_t o_nseg = align_up(o_nodes + b_rows, 256), total = o_nseg + (size_t)P;
+    unsigned char *buf = nullptr;
+    cudaStream_t s = p->stream;
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), total, s));
+    cudaError_t e = cudaMemcpyAsync(buf, draws, b_draws, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+        e = launch_random_plans(p->d, P, reinterpret_cast<uint32_t *>(buf), buf + o_nseg,
+                                reinterpret_cast<int32_t *>(buf + o_ends),
+                                reinterpret_cast<int32_t *>(buf + o_nodes), s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(nseg, buf + o_nseg, (size_t)P, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ends, buf + o_ends, b_rows, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(nodes, buf + o_nodes, b_rows, cudaMemcpyDeviceToHost, s);
+    cudaFreeAsync(buf, s);
+    cudaError_t e2 = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return from_cuda(e);
+    return from_cuda(e2);
+}
+
 pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
                                    const uint64_t *mem, const uint64_t *node_mem,
                                    const uint32_t *bw, double *beta_ms, int32_t *m, int32_t *cuts,

@@ -69,6 +69,9 @@ size_t batch_smem_bytes(int L, int k);
 cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
                          const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
                          int32_t *cuts, int32_t *placement, int8_t *status, cudaStream_t s);
+// Random comparison baseline (Section 4): P plans of problem d from 2 k draws each.
+cudaError_t launch_random_plans(const Dev &d, int64_t P, const uint32_t *draws, uint8_t *nseg, int32_t *ends,
+                                int32_t *nodes, cudaStream_t s);
 // Greedy comparison baseline (Section 4), one warp per instance.
 cudaError_t launch_greedy(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
                           const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m, int32_t *cuts,

@@ -75,6 +75,8 @@ def test_null_handles_are_rejected(lib):
     assert lib.pp_problem_workspace_bytes(None, ctypes.byref(n)) == binding.PP_ERR_ARG
     assert lib.pp_solve_exact(None, None, None, None, None) == binding.PP_ERR_ARG
     assert lib.pp_eval_plans(None, 1, None, None, None, None, None) == binding.PP_ERR_ARG
+    assert lib.pp_random_plans(None, 1, None, None, None, None) == binding.PP_ERR_ARG
+    assert lib.pp_random_plans_dev(None, 1, None, None, None, None) == binding.PP_ERR_ARG
     assert lib.pp_solve_exact_batch(-1, 4, 2, *([None] * 9)) == binding.PP_ERR_ARG
     assert lib.pp_solve_exact_batch(1, 4, 30, *([None] * 9)) == binding.PP_ERR_LIMIT
     assert lib.pp_solve_exact_batch(0, 4, 2, *([None] * 9)) == binding.PP_OK
