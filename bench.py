@@ -280,6 +280,36 @@ def run_ours(args):
                   "beta_over_optimum_mean": float(ratio.mean()) if ratio.size else None,
                   "optimal_fraction": float((ratio == 1.0).mean()) if ratio.size else None}
 
+        # the paper's random comparison baseline on the Large instance (not part of the timed step):
+        # N_PLANS plans generated on the device from seeded draws, scored by the evaluator
+        h_draws = np.random.default_rng(4242).integers(0, 2**32, size=(N_PLANS, 2 * k), dtype=np.uint64)
+        d_draws = torch.from_numpy(h_draws.astype(np.uint32).view(np.int32)).to(dev)
+        r_nseg = torch.empty(N_PLANS, dtype=torch.uint8, device=dev)
+        r_ends = torch.empty(N_PLANS * k, dtype=torch.int32, device=dev)
+        r_nodes = torch.empty(N_PLANS * k, dtype=torch.int32, device=dev)
+        r_beta, r_stat = torch.empty_like(d_beta), torch.empty_like(d_pstat)
+        random_ms = []
+        for _ in range(7):
+            e0.record(stream)
+            prob.random_plans_dev(N_PLANS, d_draws.data_ptr(), r_nseg.data_ptr(), r_ends.data_ptr(),
+                                  r_nodes.data_ptr())
+            e1.record(stream)
+            stream.synchronize()
+            random_ms.append(e0.elapsed_time(e1))
+        prob.eval_plans_dev(N_PLANS, r_nseg.data_ptr(), r_ends.data_ptr(), r_nodes.data_ptr(),
+                            r_beta.data_ptr(), r_stat.data_ptr())
+        stream.synchronize()
+        r_ok = r_beta[r_stat == 0]
+        r_ms = min(random_ms[2:])
+        r_bytes = N_PLANS * (2 * k * 4 + 1 + 2 * k * 4)  # draws in, nseg + two rows out
+        random_base = {"launch_ms": r_ms, "plans_per_s": N_PLANS / (r_ms * 1e-3),
+                       "algorithmic_GBps": r_bytes / (r_ms * 1e-3) / 1e9,
+                       "frac_of_hbm_peak": r_bytes / (r_ms * 1e-3) / 1e9 / measured_peaks()[0]["hbm_gbs"],
+                       "rows_with_a_plan": int((r_nseg > 0).sum().item()),
+                       "plans_scored_finite": int(r_ok.numel()),
+                       "best_beta_ms": float(r_ok.min().item()) if r_ok.numel() else None,
+                       "median_beta_ms": float(r_ok.median().item()) if r_ok.numel() else None}
+
         # the smaller named configurations (parity-test cases, not part of the timed step): device
         # time of one exact solve each, for context
         other = {}
@@ -377,6 +407,7 @@ def run_ours(args):
             "eval_ms": med(eval_ms), "plans_per_s": N_PLANS / (med(eval_ms) * 1e-3),
             "fast_path": prof.fast_path, "beta_ms": sol_rec.beta_ms, "segments": sol_rec.m,
             "greedy_baseline_batched": greedy,
+            "random_baseline_large": random_base,
             "other_configs": other,
         },
     }

@@ -3,6 +3,7 @@
     python -m paper_2210_12219_b200.profile_case --k 16 --solves 2
     python -m paper_2210_12219_b200.profile_case --batch 4096 --solves 1
     python -m paper_2210_12219_b200.profile_case --batch 65536 --greedy --solves 1
+    python -m paper_2210_12219_b200.profile_case --k 18 --random-plans 262144 --solves 1
 
 With k = 16 the state table is 0.44 GB (still far above the 126 MB L2), small enough for a
 multi-pass counter capture of single sweep launches.
@@ -28,6 +29,8 @@ def main():
     ap.add_argument("--generic", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="solve this many batched instances instead")
     ap.add_argument("--greedy", action="store_true", help="with --batch: the greedy comparison baseline")
+    ap.add_argument("--random-plans", type=int, default=0,
+                    help="generate this many random plans (random comparison baseline) instead of solving")
     args = ap.parse_args()
     build.build()
     if args.batch:
@@ -43,6 +46,13 @@ def main():
     k = args.k
     inst = W.Instance(large.L, k, large.layer_out_bits, large.layer_mem_bytes,
                       large.node_mem_bytes[:k].copy(), np.ascontiguousarray(large.bw_kbps[:k, :k]))
+    if args.random_plans:
+        draws = np.random.default_rng(4242).integers(0, 2**32, size=(args.random_plans, 2 * k), dtype=np.uint64)
+        with pp.Problem.from_instance(inst) as p:
+            for _ in range(args.solves):
+                nseg, _, _ = p.random_plans(draws.astype(np.uint32))
+        print("%d random plans: %d rows with a plan" % (args.random_plans, int((nseg > 0).sum())))
+        return
     sol = torch.zeros(ctypes.sizeof(pp.pp_solution) // 8, dtype=torch.float64, device="cuda")
     with pp.Problem.from_instance(inst) as p:
         if args.generic:
