@@ -203,14 +203,17 @@ pp_status pp_random_plans_dev(pp_problem *p, int64_t P, const uint32_t *draws, u
 /*
  * Greedy comparison baseline of Section 4 (second algorithm of the paper's comparison list), for
  * many independent instances of the same shape; arguments, layouts and outputs as for
- * pp_solve_exact_batch, any L <= PP_MAX_L and k <= PP_MAX_K.  For every start node n: (a) on the
- * current node, among the segments that start at the next unassigned layer and fit the node's
- * memory, take the one with the smallest outgoing transfer; (b) move to the unused node behind
- * the current node's fastest outgoing link; repeat until the chain is used up; (c) keep the start
- * node with the smallest bottleneck latency (Eq. 2, Eq. 3).  Where the paper is silent: a segment
- * that reaches the last layer transfers nothing and is taken as soon as it fits; equal transfers
- * take the longer segment, equal links the lower node, equal bottlenecks the lower start node;
- * bandwidth 0 is no link.  status[b] is PP_OK, or PP_INFEASIBLE when every walk gets stuck (the
+ * pp_solve_exact_batch, any L <= PP_MAX_L and k <= PP_MAX_K.  A walk starts on one node and
+ * repeats two choices until the chain is used up: on the current node, among the segments that
+ * start at the next unassigned layer and fit the node's memory, it takes the one with the
+ * smallest outgoing transfer; then it moves to the unused node behind the current node's fastest
+ * outgoing link.  One walk is made per start node and the one with the smallest bottleneck
+ * latency is returned (Eq. 2, Eq. 3).  Where the paper is silent: a segment that reaches the last
+ * layer transfers nothing and is taken as soon as it fits; equal transfers take the longer
+ * segment, equal links the lower node, equal bottlenecks the lower start node; bandwidth 0 is no
+ * link.  Values are not range-checked here (no PP_ERR_LIMIT per instance): the walk compares
+ * integers and divides once per cut, which is exact in the sense of Eq. 3 for bit counts below
+ * 2^53.  status[b] is PP_OK, or PP_INFEASIBLE when every walk gets stuck (the
  * heuristic found no plan; the exact search may still find one); then beta_ms = +inf, m = 0 and
  * the plan rows are -1.  Host variant: synchronous, legacy default stream.  _dev variant: device
  * pointers, asynchronous on `cuda_stream`.  cuts may be NULL when k == 1.
@@ -239,6 +242,15 @@ pp_status pp_debug_read_state_row(pp_problem *p, uint32_t mask, int32_t v, doubl
  * the sweep kernel that takes two node sets per warp relies on it. */
 pp_status pp_debug_mask_order(int32_t k, uint32_t *masks_out, uint32_t *level_off_out);
 
+/* Measurement hook: issue rate of the packed 16-bit min/max instructions the sweep consists of, on
+ * the current device.  One block of 1024 threads per SM runs `iters` trips of 64 dependent-chain
+ * instructions per thread on registers only, timed with the SM's own cycle counter; the median over
+ * the SMs gives *warp_instr_per_clk_per_sm (host).  op: 0 = two-input packed minimum, 1 = two-input
+ * packed maximum, 2 = three-input packed minimum.  The ALU bound of the search's roofline is this
+ * rate x 32 lanes x 2 elements x SMs x clock.  Synchronous, legacy default stream; allocates and
+ * frees a few hundred bytes of device memory. */
+pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm);
+
 /* Force (1) or forbid (0) the generic sweep kernel; 2 = automatic choice among the kernels that
  * take one source mask per warp (the two-mask kernel is left out); 3 = the two-mask kernel on every
  * level it can run, however small; -1 restores the automatic choice.  Meant for tests that want every kernel checked on the same instance. */
@@ -249,8 +261,7 @@ pp_status pp_problem_force_generic(pp_problem *p, int32_t mode);
  * for the library's users, not for the method).
  *
  * Who needs it: code that must not, or cannot, call cudaMalloc at this point -- a process
- * whose whole device heap was handed to a framework's caching allocator at start-up, a
- * serving loop that cannot afford the device-wide synchronisation an allocation implies, a
+ * whose whole device heap was handed to a framework's caching allocator at start-up, or a
  * plug-in that is only allowed to launch work.  pp_problem_create / pp_solve_exact allocate
  * device and pinned memory; this call does not.  It performs the same search with the same
  * kernels (the generic sweep) and gives bit-identical results, but every byte of device
@@ -260,16 +271,20 @@ pp_status pp_problem_force_generic(pp_problem *p, int32_t mode);
  *
  *   layer_out_bits, layer_mem_bytes  host [L];  node_mem_bytes host [k];  bw_kbps host [k*k]
  *   solution_dev   device, sizeof(pp_solution), 8-byte aligned: receives the result record
- *   cuda_stream    a cudaStream_t (NULL = legacy default stream); the inputs are copied from
- *                  pageable host memory with cudaMemcpyAsync (the host buffers may be reused
- *                  as soon as the call returns); kernels are queued on the stream and the call
+ *   cuda_stream    a cudaStream_t (NULL = legacy default stream).  The inputs, and a few small
+ *                  tables this call prepares on its own stack, are pageable host memory: each
+ *                  cudaMemcpyAsync of them is a staged copy that blocks the host until the
+ *                  bytes have left the host buffer (the buffers may be reused as soon as the
+ *                  call returns).  The kernels are then queued on the stream and the call
  *                  returns without waiting for them.
  * Limits: k <= 14, L <= PP_MAX_L, and the scratch the instance needs (dominated by the state
  * table, k * 2^k rows of L elements of 2 or 4 bytes) must fit PP_STATIC_SCRATCH_BYTES; anything
  * larger returns PP_ERR_LIMIT before any work is queued (k = 10, L = 50 needs about 1.1 MB;
  * k = 14, L = 100 about 52 MB).  Host-side preparation uses about 100 KB of stack.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress,
- * with that device current) and caches it; make that first call outside any stream capture.
+ * with that device current) and caches it; that first call should come before any stream
+ * capture.  Nothing in this call was written for, or tried under, stream capture: the host-side
+ * staging above and the per-launch attribute calls are ordinary eager-mode work.
  * All calls share the one array and it keeps the previous call's contents; the library resets
  * the words that must start clean itself.  Two calls whose GPU work overlaps (different
  * streams, or different host threads) race on the array: serialise them.

@@ -4,12 +4,14 @@
 Plain Python, exact integers for the memory sums and one binary64 division per transfer.
 Nothing in the product package imports this module; it shares no code with the CUDA path.
 
-The steps, in the paper's order, for every start node n:
-  (a) on the current node take, among the segments that start at the next unassigned layer and
-      fit the node's memory, the one whose outgoing transfer is smallest;
-  (b) move to the unused neighbour of the current node whose link from it has the highest
-      bandwidth; repeat (a) there, and so on until the chain is used up;
-  (c) keep the (segments, nodes) of the start node with the smallest bottleneck latency (Eq. 2).
+What it computes (Section 4, second comparison algorithm).  A walk starts on one node and
+repeats two choices until the chain is used up:
+  * segment choice: among the segments that start at the next unassigned layer and fit the
+    memory of the node the walk stands on, the one that sends the fewest bits onward;
+  * next-node choice: among the nodes not used yet, the one reached from the current node over
+    the link of highest bandwidth; the segment choice is then made there.
+One walk is made from every start node, and the result is the walk with the smallest
+bottleneck latency (Eq. 2).
 
 Where the paper is silent, the readings are:
   * a segment that reaches the last layer transfers nothing, so it is taken as soon as it fits;
@@ -39,7 +41,7 @@ class GreedyPlan:
 
 
 def walk_from(inst, start: int):
-    """Steps (a) and (b) from one start node: (beta_ms, cuts, nodes) or None when stuck."""
+    """One walk (segment choice, next-node choice, repeated) from one start node: (beta_ms, cuts, nodes) or None when stuck."""
     L, k = int(inst.L), int(inst.k)
     bits = [int(x) for x in inst.layer_out_bits]
     mem = [int(x) for x in inst.layer_mem_bytes]
@@ -50,7 +52,7 @@ def walk_from(inst, start: int):
     node, first = start, 0
     cuts, nodes, beta = [], [start], 0.0
     while True:
-        # (a) smallest outgoing transfer among the segments [first, e] that fit `node`
+        # segment choice: smallest outgoing transfer among the segments [first, e] that fit `node`
         chosen, held = -1, 0
         for e in range(first, L):
             held += mem[e]
@@ -62,7 +64,7 @@ def walk_from(inst, start: int):
             return None
         if chosen == L - 1:
             return beta, tuple(cuts), tuple(nodes)
-        # (b) highest-bandwidth link from `node` to a node not used yet
+        # next-node choice: highest-bandwidth link from `node` to a node not used yet
         nxt = -1
         for w in range(k):
             if used[w] or bw[node][w] == 0:
@@ -79,7 +81,7 @@ def walk_from(inst, start: int):
 
 
 def greedy_joint(inst) -> GreedyPlan:
-    """Step (c): the best walk over all start nodes."""
+    """The best walk over all start nodes."""
     best = None
     for n in range(int(inst.k)):
         got = walk_from(inst, n)

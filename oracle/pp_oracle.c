@@ -8,7 +8,7 @@
  *
  * Problem (paper, Section 1 and Section 3.2): a chain of L layers is cut into
  * m >= 1 contiguous, non-empty segments; segment j runs on its own edge node n_j
- * (all nodes different: "each partition is assigned to a different edge device");
+ * (Section 1: no two segments share a node, so the n_j are pairwise different);
  * a segment fits when the memory of its layers is within the node's capacity (the
  * omega(P) vs kappa predicate of the partition-graph definition, read as <=).
  * The tensor that crosses cut j is the output of the last layer of segment j, and

@@ -26,7 +26,7 @@ EXPORTS = (
     "pp_solve_exact_dev", "pp_eval_plans", "pp_eval_plans_dev", "pp_solve_exact_batch",
     "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row", "pp_debug_mask_order",
     "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str", "pp_greedy_batch",
-    "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev",
+    "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev", "pp_debug_minmax_rate",
 )
 
 
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.pp_debug_mask_order.argtypes = [i32, vp, vp]
         L.pp_problem_force_generic.argtypes = [vp, i32]
         L.pp_solve_exact_static.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp]
+        L.pp_debug_minmax_rate.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
         L.pp_status_str.argtypes = [ctypes.c_int]
         L.pp_status_str.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -285,6 +286,13 @@ def debug_mask_order(k: int):
     _check(lib().pp_debug_mask_order(int(k), ctypes.c_void_p(masks.ctypes.data),
                                      ctypes.c_void_p(level_off.ctypes.data)), "pp_debug_mask_order")
     return masks, level_off
+
+
+def debug_minmax_rate(op: int, iters: int = 2048) -> float:
+    """pp_debug_minmax_rate: warp instructions per clock per SM of one packed min/max form."""
+    rate = ctypes.c_double()
+    _check(lib().pp_debug_minmax_rate(int(op), int(iters), ctypes.byref(rate)), "pp_debug_minmax_rate")
+    return float(rate.value)
 
 
 def solve_exact_batch_dev(B, L, k, bits_ptr, mem_ptr, node_mem_ptr, bw_ptr, beta_ptr, m_ptr, cuts_ptr,

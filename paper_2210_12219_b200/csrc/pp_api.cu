@@ -693,6 +693,35 @@ pp_status pp_greedy_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_b
                            placement, status);
 }
 
+pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm)
+{
+    if (!warp_instr_per_clk_per_sm || op < 0 || op > 2 || iters < 1 || iters > (1 << 20)) return PP_ERR_ARG;
+    int dev = 0, sms = 0;
+    PP_CUDA(cudaGetDevice(&dev));
+    PP_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    unsigned char *buf = nullptr;
+    PP_CUDA(cudaMalloc(reinterpret_cast<void **>(&buf), (size_t)sms * 8 + 256));
+    long long *cycles = reinterpret_cast<long long *>(buf);
+    uint32_t *sink = reinterpret_cast<uint32_t *>(buf + (size_t)sms * 8);
+    std::vector<long long> h;
+    cudaError_t e = cudaSuccess;
+    try {
+        h.resize(sms);
+    } catch (const std::bad_alloc &) {
+        cudaFree(buf);
+        return PP_ERR_NOMEM;
+    }
+    for (int rep = 0; rep < 3 && e == cudaSuccess; ++rep) e = launch_probe(op, iters, sms, cycles, sink, nullptr);
+    if (e == cudaSuccess) e = cudaMemcpy(h.data(), cycles, (size_t)sms * 8, cudaMemcpyDeviceToHost);
+    cudaFree(buf);
+    if (e != cudaSuccess) return from_cuda(e);
+    std::sort(h.begin(), h.end());
+    const long long med = h[sms / 2];
+    if (med <= 0) return PP_ERR_CUDA;
+    *warp_instr_per_clk_per_sm = probe_instr_per_block(iters) / (double)med;
+    return PP_OK;
+}
+
 pp_status pp_debug_mask_order(int32_t k, uint32_t *masks_out, uint32_t *level_off_out)
 {
     if (!masks_out || !level_off_out || k < 1) return PP_ERR_ARG;

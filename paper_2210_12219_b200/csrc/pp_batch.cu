@@ -293,7 +293,11 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         if (tid == 0) {
             uint64_t acc = 0;
             M[0] = 0;
-            for (int i = 1; i <= L; ++i) { acc += M[i]; M[i] = acc; }
+            for (int i = 1; i <= L; ++i) {
+                if (M[i] > ~0ull - acc) s_bad = 1;  // the 64-bit sum would wrap: PP_ERR_LIMIT, as in pp_problem_create
+                acc += M[i];
+                M[i] = acc;
+            }
         }
         // distinct usable bandwidths in order of first appearance, one thread per node pair:
         // first_p[p] = earliest pair with the same bandwidth, then its index among the firsts

@@ -2,14 +2,15 @@
 // comparison list), many instances per launch: a group of G lanes per instance (G = k rounded up
 // to a power of two, so a warp holds 32 / G instances), lane n of the group walks from start node n.
 //
-// A walk alternates two steps until the chain is used up: (a) on the current node, among the
-// segments that start at the next unassigned layer and fit the node's memory, take the one whose
-// outgoing transfer is smallest; (b) move to the unused node behind the current node's fastest
-// outgoing link.  Step (c) keeps the walk with the smallest bottleneck latency (Eq. 2 with one
-// correctly rounded fp64 division per cut, Eq. 3).  Where the paper is silent: a segment that
-// reaches the last layer transfers nothing and is taken as soon as it fits; equal transfers take
-// the longer segment, equal links the lower node, equal bottlenecks the lower start node; a link
-// of bandwidth 0 is no link; a walk that gets stuck contributes no plan.
+// A walk alternates two choices until the chain is used up.  Segment choice: on the current node,
+// among the segments that start at the next unassigned layer and fit the node's memory, the one
+// whose outgoing transfer is smallest.  Next-node choice: the unused node behind the current
+// node's fastest outgoing link.  The result is the walk with the smallest bottleneck latency over
+// all start nodes (Eq. 2 with one correctly rounded fp64 division per cut, Eq. 3).  Where the
+// paper is silent: a segment that reaches the last layer transfers nothing and is taken as soon
+// as it fits; equal transfers take the longer segment, equal links the lower node, equal
+// bottlenecks the lower start node; a link of bandwidth 0 is no link; a walk that gets stuck
+// contributes no plan.
 //
 // The work of an instance is a few hundred dependent scalar steps per walk, data-dependent in
 // length: with enough instances in flight the kernel is bound by instruction issue (scalar integer
@@ -43,7 +44,7 @@ k_greedy_batch(int64_t B, int L, int k, int group, const uint64_t *__restrict__ 
         nodes[0] = lane;
         nseg = 1;
         for (;;) {
-            // (a) held never exceeds the capacity, so the sum cannot wrap
+            // segment choice; held never exceeds the capacity, so the sum cannot wrap
             const uint64_t room = cp[node];
             uint64_t held = 0, transfer = 0;
             int chosen = -1;
@@ -62,7 +63,7 @@ k_greedy_batch(int64_t B, int L, int k, int group, const uint64_t *__restrict__ 
                 arrived = true;
                 break;
             }
-            // (b) strictly faster links only: the lowest node wins a tie, a zero link never wins
+            // next-node choice; strictly faster links only: the lowest node wins a tie, a zero link never wins
             int next = -1;
             uint32_t fastest = 0;
             for (int w = 0; w < k; ++w) {
@@ -83,7 +84,7 @@ k_greedy_batch(int64_t B, int L, int k, int group, const uint64_t *__restrict__ 
             first = chosen + 1;
         }
     }
-    // (c) smallest (beta, start node); beta >= +0.0, so its bit pattern orders like the value
+    // best walk: smallest (beta, start node); beta >= +0.0, so its bit pattern orders like the value
     unsigned long long key = arrived ? (unsigned long long)__double_as_longlong(beta) : ~0ull;
     int who = lane;
     for (int o = group >> 1; o; o >>= 1) {

@@ -77,4 +77,8 @@ cudaError_t launch_greedy(int64_t B, int L, int k, const uint64_t *bits, const u
                           const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m, int32_t *cuts,
                           int32_t *place, int8_t *status, cudaStream_t s);
 
+// Issue-rate probe (pp_probe.cu): `blocks` blocks of 1024 threads, cycles[b] = SM clocks block b took.
+cudaError_t launch_probe(int op, int iters, int blocks, long long *cycles, uint32_t *sink, cudaStream_t s);
+double probe_instr_per_block(int iters);
+
 }  // namespace pp

@@ -202,7 +202,10 @@ __global__ void k_finalize(Dev d, pp_solution *out)
         __syncthreads();
         const unsigned int pick = s_pick;
         if (pick == 0xFFFFFFFFu) {  // cannot happen on a consistent table; report, do not trap
-            if (tid == 0) atomicExch(d.err, 1);
+            if (tid == 0) {
+                atomicExch(d.err, 1);
+                out->status = PP_ERR_CUDA;  // readers of the record must not take a half-written plan for a result
+            }
             return;
         }
         S = P;

@@ -32,19 +32,11 @@ namespace pp {
 
 namespace {
 
-#ifndef PP_NV768
-#define PP_NV768 6
-#endif
-#ifndef PP_NV640
-#define PP_NV640 9
-#endif
-#ifndef PP_FAST_NT
-#define PP_FAST_NT 1
-#endif
 // Threads per block by the number of source rows a warp keeps in registers: fewer rows leave room
 // for more resident warps (the register file holds 64K registers per SM).
 constexpr int kMaxFastThreads = 768;
-__host__ __device__ constexpr int fast_threads(int nv, bool gen) { return gen ? 512 : (nv <= PP_NV768 ? 768 : (nv <= PP_NV640 ? 640 : 512)); }
+constexpr int kFastNv768 = 6, kFastNv640 = 9;  // 768 threads up to NV = 6, 640 up to 9, 512 above
+__host__ __device__ constexpr int fast_threads(int nv, bool gen) { return gen ? 512 : (nv <= kFastNv768 ? 768 : (nv <= kFastNv640 ? 640 : 512)); }
 // Per-target-node constants of the window step (W = 8q + r), built on the host.
 // A shuffle distance of 31 means "nothing": rows occupy at most 30 lanes, so no lane that holds
 // data finds a source and +inf (or the untouched accumulator) results.
@@ -62,7 +54,7 @@ struct FastMeta {
     WMeta w[PP_MAX_K];
 };
 
-constexpr int NT = PP_FAST_NT;  // target nodes processed together
+constexpr int NT = 1;  // target nodes processed together
 // per-warp strip of the general window step (u16): the levels of the sparse table, then +inf
 __host__ __device__ constexpr int gen_strip_elems(int levels, int Lpad) { return levels * Lpad + 8; }
 constexpr int kTailWords = 128 + 128;           // per-warp suffix strip of the constant-window step: +inf pad, data

@@ -31,24 +31,12 @@ namespace pp {
 namespace {
 
 // Tunables (measured on the k = 18, L = 200 benchmark chain): levels the kernel takes by number of
-// source nodes, how full the machine must be (pairs * FILL >= warps), threads per block.
-#ifndef PP_PAIR_T512
-#define PP_PAIR_T512 6
-#endif
-#ifndef PP_PAIR_MIN_NV
-#define PP_PAIR_MIN_NV 3
-#endif
-#ifndef PP_PAIR_MAX_NV
-#define PP_PAIR_MAX_NV 12
-#endif
-// threads per block by the number of source rows per mask (2 * NV rows of 4 registers per lane)
-#ifndef PP_PAIR_T384
-#define PP_PAIR_T384 11
-#endif
-#ifndef PP_PAIR_FILL
-#define PP_PAIR_FILL 2
-#endif
-__host__ __device__ constexpr int pair_threads(int nv) { return nv <= PP_PAIR_T512 ? 512 : (nv <= PP_PAIR_T384 ? 384 : 256); }
+// source nodes, how full the machine must be (pairs * kPairFill >= warps), and threads per block by
+// the number of source rows per mask (2 * NV rows of 4 registers per lane).
+constexpr int kPairMinNv = 3, kPairMaxNv = 12;
+constexpr int kPairT512 = 6, kPairT384 = 11;  // 512 threads up to NV = 6, 384 up to 11, 256 above
+constexpr int kPairFill = 2;
+__host__ __device__ constexpr int pair_threads(int nv) { return nv <= kPairT512 ? 512 : (nv <= kPairT384 ? 384 : 256); }
 constexpr int kPlane = 64;               // words per strip slot
 constexpr int kStripWords = 16 * kPlane;  // per warp
 constexpr int kPlanWords = 32;            // per warp: row offsets of the pair to come
@@ -489,7 +477,7 @@ bool pair_sweep_takes(const Dev &d, int level, bool whenever_possible)
 {
     const int nv = level - 1;
     if (!d.pair_meta || d.elem != 2 || d.Lpad > 240) return false;
-    if (whenever_possible ? (nv < 2 || nv > 13) : (nv < PP_PAIR_MIN_NV || nv > PP_PAIR_MAX_NV)) return false;
+    if (whenever_possible ? (nv < 2 || nv > 13) : (nv < kPairMinNv || nv > kPairMaxNv)) return false;
     int dev = 0, max_sm = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess) return false;
     if (cudaDeviceGetAttribute(&max_sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
@@ -497,7 +485,7 @@ bool pair_sweep_takes(const Dev &d, int level, bool whenever_possible)
     if (pair_smem_bytes(d, nv) > (size_t)max_sm) return false;
     unsigned long long n = 1;  // source masks of popcount nv
     for (int i = 0; i < nv; ++i) n = n * (unsigned)(d.k - i) / (unsigned)(i + 1);
-    return whenever_possible || (n + 1) / 2 * PP_PAIR_FILL >= (unsigned long long)sms * (pair_threads(nv) / 32);
+    return whenever_possible || (n + 1) / 2 * kPairFill >= (unsigned long long)sms * (pair_threads(nv) / 32);
 }
 
 cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s)
