@@ -475,6 +475,51 @@ def run_reference(args):
     }))
 
 
+def run_only(args):
+    """Small single-part runs for profilers (no timing, no JSON line): the Large instance restricted
+    to its first --k nodes (k = 16: a 0.44 GB state table, far above the L2 and small enough for a
+    multi-pass counter capture of single sweep launches), the batched solve, or one of the two
+    comparison baselines."""
+    import torch
+
+    import paper_2210_12219_b200 as pp
+    from paper_2210_12219_b200 import build as pp_build
+
+    pp_build.build()
+    if args.only in ("batch", "greedy"):
+        insts = W.config_batched(args.batch)
+        b_bits, b_mem, b_cap, b_bw = stack(insts)
+        entry = pp.greedy_batch if args.only == "greedy" else pp.solve_exact_batch
+        for _ in range(args.solves):
+            got = entry(BATCH_L, BATCH_K, b_bits, b_mem, b_cap, b_bw)
+        print("%s of %d: %d with a plan" % (args.only, args.batch, int((got.status == 0).sum())))
+        return
+    large = W.config_large()
+    k = args.k
+    inst = W.Instance(large.L, k, large.layer_out_bits, large.layer_mem_bytes,
+                      large.node_mem_bytes[:k].copy(), np.ascontiguousarray(large.bw_kbps[:k, :k]))
+    if args.only == "unequal":  # same sizes, layers of unequal memory: the general-window kernels
+        inst = W.large_unequal_layers(k)
+    if args.only == "random":
+        draws = np.random.default_rng(4242).integers(0, 2**32, size=(args.plans, 2 * k), dtype=np.uint64)
+        with pp.Problem.from_instance(inst) as p:
+            for _ in range(args.solves):
+                nseg, _, _ = p.random_plans(draws.astype(np.uint32))
+        print("%d random plans: %d rows with a plan" % (args.plans, int((nseg > 0).sum())))
+        return
+    sol = torch.zeros(ctypes.sizeof(pp.pp_solution) // 8, dtype=torch.float64, device="cuda")
+    with pp.Problem.from_instance(inst) as p:
+        if args.mode is not None:
+            p.force_generic(args.mode)
+        for _ in range(args.solves):
+            p.solve_exact_dev(sol.data_ptr())
+        torch.cuda.synchronize()
+        prof = p.last_solve_profile()
+        rec = pp.pp_solution.from_buffer_copy(sol.cpu().numpy().tobytes())
+        print("k=%d L=%d beta=%.6f m=%d sweep=%.3f ms total=%.3f ms fast=%d pair_levels=%d" %
+              (k, inst.L, rec.beta_ms, rec.m, prof.ms_sweep, prof.ms_total, prof.fast_path, prof.pair_levels))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -482,8 +527,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    ap.add_argument("--only", choices=["sweep", "unequal", "batch", "greedy", "random"],
+                    help="profiler helper: run one part a few times and exit (see run_only)")
+    ap.add_argument("--k", type=int, default=16, help="--only sweep/unequal/random: nodes kept of the Large instance")
+    ap.add_argument("--solves", type=int, default=2, help="--only: repetitions")
+    ap.add_argument("--mode", type=int, default=None, help="--only sweep: pp_problem_force_generic mode")
+    ap.add_argument("--batch", type=int, default=N_BATCH, help="--only batch/greedy: instances")
+    ap.add_argument("--plans", type=int, default=N_PLANS, help="--only random: plans")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.only:
+        run_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

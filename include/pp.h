@@ -69,7 +69,7 @@ typedef enum {
 /* Result record of the exact search as the device writes it. */
 typedef struct {
     double beta_ms;              /* beta*, +inf if infeasible */
-    int32_t status;              /* PP_OK or PP_INFEASIBLE */
+    int32_t status;              /* PP_OK or PP_INFEASIBLE; PP_ERR_CUDA when the backtrack broke off */
     int32_t m;                   /* number of segments, 0 if infeasible */
     int32_t cuts[PP_MAX_K];      /* e_1 .. e_{m-1}; unused slots are -1 */
     int32_t placement[PP_MAX_K]; /* n_1 .. n_m;     unused slots are -1 */
@@ -77,11 +77,11 @@ typedef struct {
 
 /* Device-time breakdown of the last pp_solve_exact / pp_solve_exact_dev of a problem. */
 typedef struct {
-    float ms_rank;     /* gamma table and rank compression (Eq. 3) */
-    float ms_sweep;    /* base frontier plus all popcount levels of the (min,max) sweep */
+    float ms_rank;     /* gamma table, rank compression (Eq. 3) and the base frontier (one node used) */
+    float ms_sweep;    /* all popcount levels (two nodes and more) of the (min,max) sweep */
     float ms_finalize; /* final choice and backtrack */
     float ms_total;
-    int32_t sweep_launches;  /* kernels launched for the sweep, base frontier included */
+    int32_t sweep_launches;  /* kernels launched for the sweep: one per popcount level from 2 up */
     int32_t total_launches;  /* all kernels of the solve */
     int32_t state_bytes;     /* bytes of one state element: 2 (16-bit ranks) or 4 */
     int32_t fast_path;       /* register-tiled sweep: 1 = constant-width windows, 2 = general
@@ -227,8 +227,12 @@ pp_status pp_greedy_batch_dev(int64_t B, int32_t L, int32_t k, const uint64_t *o
                               double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
                               int8_t *status, void *cuda_stream);
 
-/* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream. */
+/* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream.
+ * ms_total is always measured.  ms_rank, ms_sweep and ms_finalize need events between the
+ * phases, which keep one phase's kernels from being launched under the tail of the previous
+ * one: they are recorded only after pp_problem_set_profiling(p, 1) and read 0 otherwise. */
 pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out);
+pp_status pp_problem_set_profiling(pp_problem *p, int32_t on);
 
 /* Test hook: after a solve, copy one row of the state table to the host as latencies:
  * row_out[c] = value of state (mask, v, c) in milliseconds (+inf if unreachable), c = 0..L-1.
@@ -253,7 +257,8 @@ pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per
 
 /* Force (1) or forbid (0) the generic sweep kernel; 2 = automatic choice among the kernels that
  * take one source mask per warp (the two-mask kernel is left out); 3 = the two-mask kernel on every
- * level it can run, however small; -1 restores the automatic choice.  Meant for tests that want every kernel checked on the same instance. */
+ * level it can run, however small; -1 restores the automatic choice.  Meant for tests that want
+ * every kernel checked on the same instance. */
 pp_status pp_problem_force_generic(pp_problem *p, int32_t mode);
 
 /*

@@ -27,6 +27,7 @@ EXPORTS = (
     "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row", "pp_debug_mask_order",
     "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str", "pp_greedy_batch",
     "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev", "pp_debug_minmax_rate",
+    "pp_problem_set_profiling",
 )
 
 
@@ -81,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.pp_debug_read_state_row.argtypes = [vp, ctypes.c_uint32, i32, vp]
         L.pp_debug_mask_order.argtypes = [i32, vp, vp]
         L.pp_problem_force_generic.argtypes = [vp, i32]
+        L.pp_problem_set_profiling.argtypes = [vp, i32]
         L.pp_solve_exact_static.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp]
         L.pp_debug_minmax_rate.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
         L.pp_status_str.argtypes = [ctypes.c_int]
@@ -170,6 +172,9 @@ class Problem:
                                               tensor.numel() * tensor.element_size()),
                "pp_problem_set_workspace")
         self._workspace = tensor
+
+    def set_profiling(self, on: bool):
+        _check(lib().pp_problem_set_profiling(self._h, int(bool(on))), "pp_problem_set_profiling")
 
     def force_generic(self, mode: int):
         _check(lib().pp_problem_force_generic(self._h, int(mode)), "pp_problem_force_generic")

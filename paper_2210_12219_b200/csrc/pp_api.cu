@@ -31,9 +31,10 @@ struct pp_problem {
     pp_solution *d_sol = nullptr;
     int32_t *h_err = &h_err_buf;
     Dev d{};
-    bool solved = false;
+    bool solved = false, profiled = false;
     int sweep_launches = 0, total_launches = 0, fast_used = 0, pair_levels = 0;
     int force_generic = -1;
+    bool profiling = false;             // record events between the phases of a solve
     bool mask_swaps = false;            // the mask list pairs up (see mask_list)
     std::vector<signed char> pair_lvl;  // per level: 1 = two-mask kernel, 0 = one-mask, -1 = not decided yet
 };
@@ -160,7 +161,7 @@ pp_status from_cuda(cudaError_t e)
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkLayout {
-    size_t pos, order, gu, rk, inv, rank, table, total;
+    size_t pos, order, gu, cnt, rk, inv, rank, table, total;
 };
 
 WorkLayout work_layout(int L, int k, int Lpad, int U, int elem)
@@ -170,6 +171,7 @@ WorkLayout work_layout(int L, int k, int Lpad, int U, int elem)
     w.pos = o;   o = align_up(o + (size_t)L * 2, 256);
     w.order = o; o = align_up(o + (size_t)L * 2, 256);
     w.gu = o;    o = align_up(o + (size_t)std::max(U, 1) * L * 8, 256);
+    w.cnt = o;   o = align_up(o + (size_t)std::max(U, 1) * L * 4, 256);
     w.rk = o;    o = align_up(o + (size_t)std::max(U, 1) * L * 4, 256);
     w.inv = o;   o = align_up(o + ((size_t)std::max(U, 1) * L + 2) * 4, 256);
     w.rank = o;  o = align_up(o + (size_t)k * k * Lpad * elem, 256);
@@ -203,6 +205,7 @@ void bind_work(pp_problem *p)
     p->d.pos = reinterpret_cast<int16_t *>(b + w.pos);
     p->d.order = reinterpret_cast<int16_t *>(b + w.order);
     p->d.gu = reinterpret_cast<double *>(b + w.gu);
+    p->d.cnt = reinterpret_cast<uint32_t *>(b + w.cnt);
     p->d.rk = reinterpret_cast<uint32_t *>(b + w.rk);
     p->d.inv = reinterpret_cast<uint32_t *>(b + w.inv);
     p->d.rank = b + w.rank;
@@ -227,34 +230,36 @@ pp_status queue_solve(pp_problem *p, pp_solution *sol_dev)
     pp_status st = ensure_work(p);
     if (st != PP_OK) return st;
     cudaStream_t s = p->stream;
+    bool fast = fast_sweep_supported(p->d);
+    if (p->force_generic == 1) fast = false;
     const Dev &d = p->d;
     int launches = 0;
     PP_CUDA(cudaEventRecord(p->ev[0], s));
-    PP_CUDA(launch_rank_build(d, s, &launches));
-    PP_CUDA(cudaEventRecord(p->ev[1], s));
-    PP_CUDA(launch_base(d, s));
-    int sweep = 1, pairs = 0;
+    PP_CUDA(launch_rank_base(d, s, &launches));
+    // an event between two kernels ends the programmatic overlap of their launches: only on request
+    if (p->profiling) PP_CUDA(cudaEventRecord(p->ev[1], s));
+    int sweep = 0, pairs = 0;
     const int top = std::min(p->k, p->L);
-    bool fast = fast_sweep_supported(d);
-    if (p->force_generic == 1) fast = false;
     for (int level = 2; level <= top; ++level) {
+        const bool first = level == 2;
         if (fast && p->force_generic != 2) {
             if (p->pair_lvl[level] < 0) p->pair_lvl[level] = pair_sweep_takes(d, level, p->force_generic == 3) ? 1 : 0;
-            PP_CUDA(p->pair_lvl[level] ? launch_sweep_pair(d, level, s) : launch_sweep_fast(d, level, s));
+            PP_CUDA(p->pair_lvl[level] ? launch_sweep_pair(d, level, s, first) : launch_sweep_fast(d, level, s, first));
             pairs += p->pair_lvl[level];
         } else {
-            PP_CUDA(fast ? launch_sweep_fast(d, level, s) : launch_sweep_generic(d, level, s));
+            PP_CUDA(fast ? launch_sweep_fast(d, level, s, first) : launch_sweep_generic(d, level, s));
         }
         ++sweep;
     }
-    PP_CUDA(cudaEventRecord(p->ev[2], s));
-    PP_CUDA(launch_finalize(d, sol_dev, s));
+    if (p->profiling) PP_CUDA(cudaEventRecord(p->ev[2], s));
+    PP_CUDA(launch_finalize(d, sol_dev, s, true));
     PP_CUDA(cudaEventRecord(p->ev[3], s));
     p->sweep_launches = sweep;
     p->pair_levels = pairs;
     p->total_launches = launches + sweep + 1;
     p->fast_used = fast ? (p->d.fast_meta ? 1 : 2) : 0;
     p->solved = true;
+    p->profiled = p->profiling;
     return PP_OK;
 }
 
@@ -472,6 +477,13 @@ pp_status pp_problem_force_generic(pp_problem *p, int32_t mode)
     return PP_OK;
 }
 
+pp_status pp_problem_set_profiling(pp_problem *p, int32_t on)
+{
+    if (!p) return PP_ERR_ARG;
+    p->profiling = on != 0;
+    return PP_OK;
+}
+
 pp_status pp_solve_exact_dev(pp_problem *p, pp_solution *solution_dev)
 {
     if (!p || !solution_dev) return PP_ERR_ARG;
@@ -500,9 +512,12 @@ pp_status pp_last_solve_profile(pp_problem *p, pp_profile *out)
 {
     if (!p || !out || !p->solved) return PP_ERR_ARG;
     PP_CUDA(cudaStreamSynchronize(p->stream));
-    PP_CUDA(cudaEventElapsedTime(&out->ms_rank, p->ev[0], p->ev[1]));
-    PP_CUDA(cudaEventElapsedTime(&out->ms_sweep, p->ev[1], p->ev[2]));
-    PP_CUDA(cudaEventElapsedTime(&out->ms_finalize, p->ev[2], p->ev[3]));
+    out->ms_rank = out->ms_sweep = out->ms_finalize = 0.0f;
+    if (p->profiled) {
+        PP_CUDA(cudaEventElapsedTime(&out->ms_rank, p->ev[0], p->ev[1]));
+        PP_CUDA(cudaEventElapsedTime(&out->ms_sweep, p->ev[1], p->ev[2]));
+        PP_CUDA(cudaEventElapsedTime(&out->ms_finalize, p->ev[2], p->ev[3]));
+    }
     PP_CUDA(cudaEventElapsedTime(&out->ms_total, p->ev[0], p->ev[3]));
     out->sweep_launches = p->sweep_launches;
     out->total_launches = p->total_launches;

@@ -29,12 +29,13 @@ struct Dev {
     int16_t *pos;              // [L] position of layer c in the ascending order of bits
     int16_t *order;            // [L] layer at each position
     double *gu;                // [U*L] gu[u*L+i] = bits[order[i]] / ubw[u]  (ascending in i)
-    uint32_t *rk;              // [U*L] rank of gu[u*L+i]
+    uint32_t *cnt;             // [U*L] number of quotients below gu[u*L+i] (accumulated by the rank build)
+    uint32_t *rk;              // [U*L] rank of gu[u*L+i] = 1 + cnt
     uint32_t *inv;             // [U*L+2] inv[r] = some entry e with rk[e] == r (equal ranks hold equal doubles)
     void *rank;                // [k*k*Lpad] rank[(w*k+v)*Lpad + c] of gamma[c][v][w], element type
     void *table;               // [2^k * k * Lpad] state rows, row (S, v) at (S*k+v)*Lpad
     unsigned long long *best;  // packed (rank, popcount, mask, v) of the best final state
-    int32_t *err;              // device error word (0 = fine)
+    int32_t *err;              // device error word (0 = fine, kErrBacktrack)
     const void *fast_meta;     // per-node window constants of the register-tiled sweep, or null
     const uint32_t *gen_meta;  // [k*Lpad] per-(node, position) lookup words of its general-window step, or null
     int gen_levels;            // levels of that step's sparse table (1 + floor(log2(longest window)))
@@ -42,6 +43,7 @@ struct Dev {
 };
 
 static constexpr unsigned long long kNoBest = ~0ull;
+static constexpr int32_t kErrBacktrack = 1;  // the backtrack found no predecessor (inconsistent table)
 
 // final-state key: smaller is better; rank in the high bits, then popcount, mask, node
 __host__ __device__ inline unsigned long long pack_best(uint32_t rank, int popc, uint32_t mask, int v)
@@ -50,19 +52,19 @@ __host__ __device__ inline unsigned long long pack_best(uint32_t rank, int popc,
            ((unsigned long long)mask << 5) | (unsigned long long)v;
 }
 
-cudaError_t launch_rank_build(const Dev &d, cudaStream_t s, int *launches);
-cudaError_t launch_base(const Dev &d, cudaStream_t s);
+cudaError_t launch_rank_base(const Dev &d, cudaStream_t s, int *launches);
 cudaError_t launch_sweep_generic(const Dev &d, int level, cudaStream_t s);
 size_t fast_meta_bytes();
 bool fast_meta_build(int L, int k, const int16_t *lo, void *out);
 int gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out);
 bool fast_sweep_supported(const Dev &d);
-cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s);
+// first_level: the kernel follows the rank build directly and must wait for it before reading anything
+cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s, bool first_level);
 size_t pair_meta_bytes();
 bool pair_meta_build(int L, int k, const int16_t *lo, void *out);
 bool pair_sweep_takes(const Dev &d, int level, bool whenever_possible);
-cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s);
-cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s);
+cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s, bool first_level);
+cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s, bool dependent);
 cudaError_t launch_eval(const Dev &d, int64_t B, const uint8_t *nseg, const int32_t *ends,
                         const int32_t *nodes, double *beta, uint8_t *status, cudaStream_t s);
 size_t batch_smem_bytes(int L, int k);

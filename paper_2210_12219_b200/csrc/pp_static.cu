@@ -99,6 +99,7 @@ extern "C" pp_status pp_solve_exact_static(int32_t L, const uint64_t *layer_out_
     const size_t o_pos = o;   o = up256(o + (size_t)L * 2);
     const size_t o_order = o; o = up256(o + (size_t)L * 2);
     const size_t o_gu = o;    o = up256(o + (size_t)(U > 0 ? U : 1) * L * 8);
+    const size_t o_cnt = o;   o = up256(o + (size_t)(U > 0 ? U : 1) * L * 4);
     const size_t o_rk = o;    o = up256(o + (size_t)(U > 0 ? U : 1) * L * 4);
     const size_t o_inv = o;   o = up256(o + ((size_t)(U > 0 ? U : 1) * L + 2) * 4);
     const size_t o_rank = o;  o = up256(o + (size_t)k * k * Lpad * elem);
@@ -141,7 +142,8 @@ extern "C" pp_status pp_solve_exact_static(int32_t L, const uint64_t *layer_out_
         if (e != cudaSuccess) { cudaGetLastError(); return PP_ERR_CUDA; }
     }
     // the array keeps whatever the previous call left: reset the words that must start clean
-    // (the best-state key is reset by launch_base; every table row is written before it is read)
+    // (the best-state key and the per-quotient counts are reset by the rank build; every table row
+    // is written before it is read)
     e = cudaMemsetAsync(b + o_err, 0, 4, s);
     if (e != cudaSuccess) { cudaGetLastError(); return PP_ERR_CUDA; }
 
@@ -161,17 +163,17 @@ extern "C" pp_status pp_solve_exact_static(int32_t L, const uint64_t *layer_out_
     d.pos = reinterpret_cast<int16_t *>(b + o_pos);
     d.order = reinterpret_cast<int16_t *>(b + o_order);
     d.gu = reinterpret_cast<double *>(b + o_gu);
+    d.cnt = reinterpret_cast<uint32_t *>(b + o_cnt);
     d.rk = reinterpret_cast<uint32_t *>(b + o_rk);
     d.inv = reinterpret_cast<uint32_t *>(b + o_inv);
     d.rank = b + o_rank;
     d.table = b + o_table;
 
     int launches = 0;
-    e = launch_rank_build(d, s, &launches);
-    if (e == cudaSuccess) e = launch_base(d, s);
+    e = launch_rank_base(d, s, &launches);
     const int top = k < L ? k : L;
     for (int level = 2; level <= top && e == cudaSuccess; ++level) e = launch_sweep_generic(d, level, s);
-    if (e == cudaSuccess) e = launch_finalize(d, solution_dev, s);
+    if (e == cudaSuccess) e = launch_finalize(d, solution_dev, s, false);
     if (e != cudaSuccess) { cudaGetLastError(); return PP_ERR_CUDA; }
     return PP_OK;
 }

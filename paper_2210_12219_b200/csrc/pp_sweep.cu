@@ -1,4 +1,4 @@
-// Base frontier, the generic popcount-level sweep, and the final choice + backtrack.
+// The generic popcount-level sweep, and the final choice + backtrack.
 //
 // State (S, v, c): layers 0..c are placed on exactly the nodes of S, one segment each, the
 // last segment on v ending at layer c.  Its value is the smallest bottleneck (Eq. 2) any such
@@ -20,33 +20,6 @@ __device__ __forceinline__ void offer_best(const Dev &d, T val, uint32_t mask, i
     unsigned long long key = pack_best((uint32_t)val, __popc(mask), mask, v);
     // read first: almost every offer loses, and a plain load is far cheaper than an atomic
     if (key < *reinterpret_cast<volatile unsigned long long *>(d.best)) atomicMin(d.best, key);
-}
-
-template <typename T>
-__global__ void k_base(Dev d)
-{
-    const T kInf = (T)~(T)0;
-    T *table = reinterpret_cast<T *>(d.table);
-    int v = blockIdx.x;
-    uint32_t S = 1u << v;
-    T *row = table + ((size_t)S * d.k + v) * d.Lpad;
-    uint64_t cap = d.cap[v];
-    for (int c = threadIdx.x; c < d.Lpad; c += blockDim.x) {
-        T x = (c < d.L && d.M[c + 1] <= cap) ? (T)0 : kInf;
-        row[c] = x;
-        if (c == d.L - 1) offer_best<T>(d, x, S, v);
-    }
-}
-
-cudaError_t launch_base(const Dev &d, cudaStream_t s)
-{
-    cudaError_t e = cudaMemsetAsync(d.best, 0xFF, sizeof(unsigned long long), s);
-    if (e != cudaSuccess) return e;
-    if (d.elem == 2)
-        k_base<uint16_t><<<d.k, 128, 0, s>>>(d);
-    else
-        k_base<uint32_t><<<d.k, 128, 0, s>>>(d);
-    return cudaGetLastError();
 }
 
 // Generic sweep of one level: one block per source mask S of popcount level-1.  Works for any
@@ -126,16 +99,18 @@ cudaError_t launch_sweep_generic(const Dev &d, int level, cudaStream_t s)
 // One block.  The best final state was collected by offer_best during the sweep.  Walking
 // back from (S', w, c'), the predecessor is the lowest c, then the lowest v, among
 // v in S'\{w}, c in [lo_w(c'), c'-1] with max(dp[S'\{w}][v][c], gamma[c][v][w]) <= beta*.
+// Warp i scans the candidates of the i-th node of S'\{w} in ascending c and stops at its first hit.
 template <typename T>
-__global__ void k_finalize(Dev d, pp_solution *out)
+__global__ void __launch_bounds__(1024) k_finalize(Dev d, pp_solution *out)
 {
     __shared__ unsigned int s_key[32];
     __shared__ unsigned int s_pick;
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // a no-op unless launched as a dependent
     const T *table = reinterpret_cast<const T *>(d.table);
     const T *rank = reinterpret_cast<const T *>(d.rank);
     const int k = d.k, L = d.L, Lpad = d.Lpad;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const unsigned long long key = *d.best;
+    const unsigned long long key = *reinterpret_cast<volatile unsigned long long *>(d.best);
 
     if (tid < PP_MAX_K) {
         out->cuts[tid] = -1;
@@ -171,23 +146,28 @@ __global__ void k_finalize(Dev d, pp_solution *out)
         if (j == 0) break;
         const uint32_t P = S & ~(1u << w);
         const int lo = d.lo[w * L + c2];
-        const int span = c2 - lo;  // candidates c = lo .. c2-1
-        unsigned int bestk = 0xFFFFFFFFu;
         const int np = __popc(P);
-        for (int item = tid; item < span * np; item += blockDim.x) {
-            const int vi = item / span, c = lo + (item - vi * span);
+        unsigned int bestk = 0xFFFFFFFFu;
+        for (int vi = wid; vi < np; vi += (int)(blockDim.x >> 5)) {
             const int v = __fns(P, 0, vi + 1);
-            T a = table[((size_t)P * k + v) * Lpad + c];
-            T b = rank[((size_t)w * k + v) * Lpad + c];
-            T mx = a > b ? a : b;
-            if ((uint32_t)mx <= rstar && mx != (T)~(T)0) {
-                unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
-                bestk = kk < bestk ? kk : bestk;
+            const T *trow = table + ((size_t)P * k + v) * Lpad;
+            const T *rrow = rank + ((size_t)w * k + v) * Lpad;
+            for (int c0 = lo; c0 < c2; c0 += 32) {
+                const int c = c0 + lane;
+                bool hit = false;
+                if (c < c2) {
+                    const T a = trow[c];
+                    const T b = rrow[c];
+                    const T mx = a > b ? a : b;
+                    hit = (uint32_t)mx <= rstar && mx != (T)~(T)0;
+                }
+                const unsigned int hits = __ballot_sync(0xFFFFFFFFu, hit);
+                if (hits) {
+                    const unsigned int kk = ((unsigned)(c0 + __ffs(hits) - 1) << 5) | (unsigned)v;
+                    bestk = kk < bestk ? kk : bestk;
+                    break;
+                }
             }
-        }
-        for (int o = 16; o; o >>= 1) {
-            unsigned int other = __shfl_xor_sync(0xFFFFFFFFu, bestk, o);
-            bestk = other < bestk ? other : bestk;
         }
         if (lane == 0) s_key[wid] = bestk;
         __syncthreads();
@@ -203,7 +183,7 @@ __global__ void k_finalize(Dev d, pp_solution *out)
         const unsigned int pick = s_pick;
         if (pick == 0xFFFFFFFFu) {  // cannot happen on a consistent table; report, do not trap
             if (tid == 0) {
-                atomicExch(d.err, 1);
+                atomicExch(d.err, kErrBacktrack);
                 out->status = PP_ERR_CUDA;  // readers of the record must not take a half-written plan for a result
             }
             return;
@@ -215,13 +195,19 @@ __global__ void k_finalize(Dev d, pp_solution *out)
     }
 }
 
-cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s)
+cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s, bool dependent)
 {
-    if (d.elem == 2)
-        k_finalize<uint16_t><<<1, 1024, 0, s>>>(d, out);
-    else
-        k_finalize<uint32_t><<<1, 1024, 0, s>>>(d, out);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(1024);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return d.elem == 2 ? cudaLaunchKernelEx(&cfg, k_finalize<uint16_t>, d, out)
+                       : cudaLaunchKernelEx(&cfg, k_finalize<uint32_t>, d, out);
 }
 
 }  // namespace pp

@@ -200,9 +200,12 @@ __device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const
 
 template <int NV, bool GEN>
 __global__ void __launch_bounds__(fast_threads(NV, GEN), 1)
-k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
+k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split, int first_level)
 {
     constexpr int kFastThreads = fast_threads(NV, GEN);
+    // The first level of a solve follows the kernel that writes the rank table and the base
+    // frontier: nothing may be read before that kernel is complete.
+    if (first_level) asm volatile("griddepcontrol.wait;" ::: "memory");
     // Programmatic dependent launch: let the next level's blocks be scheduled as soon as this
     // level's blocks retire, so that their prologue (rank table -> shared memory) overlaps our
     // tail.  Nothing the previous level wrote is touched before griddepcontrol.wait below.
@@ -241,7 +244,7 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split)
         if ((threadIdx.x & 31) == 0) strips[d.gen_levels * Lpad] = 0xFFFFu;  // the constant +inf behind the table
     }
     __syncthreads();
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
+    if (!first_level) asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -406,7 +409,8 @@ size_t fast_smem_bytes(const Dev &d)
 }
 
 template <int NV, bool GEN>
-cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned grid, int split, size_t sm, cudaStream_t s)
+cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned grid, int split, size_t sm, cudaStream_t s,
+                      int first_level)
 {
     cudaError_t e = cudaFuncSetAttribute(k_sweep_fast<NV, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
@@ -420,7 +424,7 @@ cudaError_t launch_nv(const Dev &d, int level, const FastMeta *meta, unsigned gr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_sweep_fast<NV, GEN>, d, level, meta, split);
+    return cudaLaunchKernelEx(&cfg, k_sweep_fast<NV, GEN>, d, level, meta, split, first_level);
 }
 
 }  // namespace
@@ -495,7 +499,7 @@ bool fast_sweep_supported(const Dev &d)
     return fast_smem_bytes(d) <= (size_t)max_sm;
 }
 
-cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s)
+cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s, bool first_level)
 {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
@@ -515,8 +519,8 @@ cudaError_t launch_sweep_fast(const Dev &d, int level, cudaStream_t s)
     const FastMeta *meta = static_cast<const FastMeta *>(d.fast_meta);
     switch (level - 1) {
 #define PP_CASE(N) \
-    case N: return meta ? launch_nv<N, false>(d, level, meta, grid, split, sm, s) \
-                        : launch_nv<N, true>(d, level, meta, grid, split, sm, s);
+    case N: return meta ? launch_nv<N, false>(d, level, meta, grid, split, sm, s, first_level) \
+                        : launch_nv<N, true>(d, level, meta, grid, split, sm, s, first_level);
         PP_CASE(1) PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6) PP_CASE(7) PP_CASE(8)
         PP_CASE(9) PP_CASE(10) PP_CASE(11) PP_CASE(12) PP_CASE(13) PP_CASE(14) PP_CASE(15)
         PP_CASE(16) PP_CASE(17) PP_CASE(18) PP_CASE(19)

@@ -113,11 +113,14 @@ __device__ __noinline__ unsigned long long offer_pair(unsigned long long *best, 
 // L8: the chain length is a multiple of 8, so the last element of a row is a lane's last position.
 template <int NV, bool L8>
 __global__ void __launch_bounds__(pair_threads(NV), 1)
-k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
+k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g, int first_level)
 {
     constexpr int kThreads = pair_threads(NV);
     constexpr int kWarps = kThreads / 32;
     constexpr int NC = NV - 1;  // sources common to both masks
+    // The first level of a solve follows the kernel that writes the rank table and the base
+    // frontier: nothing may be read before that kernel is complete.
+    if (first_level) asm volatile("griddepcontrol.wait;" ::: "memory");
     // the next level's prologue (rank table -> shared memory) may overlap this level's tail
     asm volatile("griddepcontrol.launch_dependents;");
     extern __shared__ uint4 smem4[];
@@ -139,7 +142,7 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
         for (int i = threadIdx.x; i < kWarps * kStripWords; i += kThreads) strips[i] = kInf2;
     }
     __syncthreads();
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
+    if (!first_level) asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -216,8 +219,11 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
         voffb = wo[NV] * 8;
         best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
     };
+    // the masks of a pair are fetched two pairs ahead: their latency never meets a dependent instruction
+    uint32_t S1n = 0, S2n = 0;
     if (pi < npair) {
         fetch_masks(pi, S1, S2);
+        if (pi + stride < npair) fetch_masks(pi + stride, S1n, S2n);
         plan_rows(S1, S2, false);
         load_rows1(S1);
         load_rows2(S2);
@@ -227,8 +233,8 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
     while (pi < npair) {
         const uint32_t pi_next = pi + stride;
         const bool more = pi_next < npair;
-        uint32_t S1n = 0, S2n = 0;
-        if (more) fetch_masks(pi_next, S1n, S2n);
+        uint32_t S1nn = 0, S2nn = 0;
+        if (pi_next + stride < npair) fetch_masks(pi_next + stride, S1nn, S2nn);
         const uint32_t A = S1, B = S2;
         const uint32_t base1 = A * mask_rows + lane, base2 = B * mask_rows + lane;
 
@@ -410,6 +416,8 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g)
         pi = pi_next;
         S1 = S1n;
         S2 = S2n;
+        S1n = S1nn;
+        S2n = S2nn;
     }
 }
 
@@ -420,7 +428,7 @@ size_t pair_smem_bytes(const Dev &d, int nv)
 }
 
 template <int NV, bool L8>
-cudaError_t launch_pair_nv(const Dev &d, int level, unsigned grid, size_t sm, cudaStream_t s)
+cudaError_t launch_pair_nv(const Dev &d, int level, unsigned grid, size_t sm, cudaStream_t s, int first_level)
 {
     cudaError_t e = cudaFuncSetAttribute(k_sweep_pair<NV, L8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
@@ -434,7 +442,8 @@ cudaError_t launch_pair_nv(const Dev &d, int level, unsigned grid, size_t sm, cu
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_sweep_pair<NV, L8>, d, level, static_cast<const PairMeta *>(d.pair_meta));
+    return cudaLaunchKernelEx(&cfg, k_sweep_pair<NV, L8>, d, level, static_cast<const PairMeta *>(d.pair_meta),
+                              first_level);
 }
 
 }  // namespace
@@ -488,7 +497,7 @@ bool pair_sweep_takes(const Dev &d, int level, bool whenever_possible)
     return whenever_possible || (n + 1) / 2 * kPairFill >= (unsigned long long)sms * (pair_threads(nv) / 32);
 }
 
-cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s)
+cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s, bool first_level)
 {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
@@ -502,8 +511,8 @@ cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s)
     const size_t sm = pair_smem_bytes(d, nv);
     switch (nv) {
 #define PP_CASE(N) \
-    case N: return (d.L & 7) ? launch_pair_nv<N, false>(d, level, grid, sm, s) \
-                             : launch_pair_nv<N, true>(d, level, grid, sm, s);
+    case N: return (d.L & 7) ? launch_pair_nv<N, false>(d, level, grid, sm, s, first_level) \
+                             : launch_pair_nv<N, true>(d, level, grid, sm, s, first_level);
         PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6) PP_CASE(7) PP_CASE(8)
         PP_CASE(9) PP_CASE(10) PP_CASE(11) PP_CASE(12) PP_CASE(13)
 #undef PP_CASE

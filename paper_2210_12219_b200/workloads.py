@@ -191,6 +191,17 @@ def config_large() -> Instance:
     return Instance(L, k, bits, mem, cap, bw, "large")
 
 
+def large_unequal_layers(k: int = 18) -> Instance:
+    """The Large chain with layers of unequal memory (what a real model chain looks like): the same
+    bits, capacities and bandwidths (the first k nodes), each layer's 6 MB scaled by U[0.5, 1.5).
+    The sliding memory windows then differ from position to position."""
+    base = config_large()
+    u = stream(5, 1, F_MEM).uniform01(base.L)
+    mem = np.rint(base.layer_mem_bytes.astype(np.float64) * (0.5 + u)).astype(np.uint64)
+    return Instance(base.L, k, base.layer_out_bits, mem, base.node_mem_bytes[:k].copy(),
+                    np.ascontiguousarray(base.bw_kbps[:k, :k]), "large_unequal_layers")
+
+
 def random_small(seed: int, L: int, k: int, *, tight: bool = False, dead_links: float = 0.0,
                  ties: bool = False) -> Instance:
     """Small random instance for parity sweeps.  tight=True shrinks capacities so that some
