@@ -5,7 +5,8 @@ One step = one pass of the whole hot path over one batch of synthetic input:
   1. exact search on the Large instance (k = 18 nodes, L = 200 layers): gamma/rank tables,
      base frontier, every popcount level of the (min,max) sweep, final choice, backtrack;
   2. the batched many-instance search on 4096 instances (k = 8, L = 24);
-  3. the batched beta evaluator on 262144 candidate plans of the Large instance.
+  3. the batched beta evaluator on 262144 candidate plans of the Large instance (compressed rows:
+     16-bit cuts, 8-bit nodes, one offset per plan).
 The headline number is DP relaxations per second, where one relaxation is
 g = min(g, max(dp, gamma)) and an instance has k(k-1)2^(k-2) L of them (a closed form of
 the sizes, not of the data).
@@ -36,13 +37,10 @@ from paper_2210_12219_b200 import workloads as W  # noqa: E402
 
 METRIC = "exact-plan DP relaxations/s"
 UNIT = "relaxations/s"
-# DRAM bytes per sweep launch (18 launches per Large solve, base frontier included) from the ncu
-# capture summarised in profiles/sweep_dram_traffic_large.md; set to None whenever the sweep
-# kernels change after that capture.
-SWEEP_DRAM_BYTES_PER_LAUNCH = 94.83e6
-# Issue rate of packed 16-bit min/max measured on this part: 64 lanes per clock per SM, two
-# elements per lane (a three-input min/max issues at the same rate).
-PACKED_MINMAX_LANES_PER_CLK_SM = 64
+# DRAM bytes (read + write) per sweep launch of the Large solve from an ncu capture of the sweep
+# kernels as they stand; None whenever those kernels have changed since the counters were taken.
+SWEEP_DRAM_BYTES_PER_LAUNCH = None
+NOMINAL_HBM_GBS = 8000.0  # the "about 8 TB/s" the roofline is also quoted against
 N_PLANS = 262144
 N_BATCH = 4096
 BATCH_L, BATCH_K = 24, 8
@@ -167,6 +165,8 @@ def run_ours(args):
     batch = W.config_batched(N_BATCH, BATCH_L, BATCH_K)
     b_bits, b_mem, b_cap, b_bw = stack(batch)
     nseg, ends, nodes = W.random_plans(large, N_PLANS, seed=77, invalid_fraction=0.05)
+    p_off, p_ends, p_nodes = W.pack_plans(nseg, ends, nodes)
+    n_entries = int(p_ends.size)
     k, L = large.k, large.L
     relax_large = n_relax(k, L)
     relax_batch = N_BATCH * n_relax(BATCH_K, BATCH_L)
@@ -179,6 +179,7 @@ def run_ours(args):
     prob.set_workspace(ws)
     tt = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
     d_nseg, d_ends, d_nodes = tt(nseg), tt(ends), tt(nodes)
+    d_off, d_pends, d_pnodes = tt(p_off.view(np.int32)), tt(p_ends.view(np.int16)), tt(p_nodes)
     d_beta = torch.empty(N_PLANS, dtype=torch.float64, device=dev)
     d_pstat = torch.empty(N_PLANS, dtype=torch.uint8, device=dev)
     d_bb, d_bm, d_bc, d_bbw = tt(b_bits), tt(b_mem), tt(b_cap), tt(b_bw)
@@ -197,6 +198,10 @@ def run_ours(args):
                                  stream.cuda_stream)
 
     def eval_device():
+        prob.eval_plans_packed_dev(N_PLANS, n_entries, d_nseg.data_ptr(), d_off.data_ptr(), d_pends.data_ptr(),
+                                   d_pnodes.data_ptr(), d_beta.data_ptr(), d_pstat.data_ptr())
+
+    def eval_device_int32():
         prob.eval_plans_dev(N_PLANS, d_nseg.data_ptr(), d_ends.data_ptr(), d_nodes.data_ptr(),
                             d_beta.data_ptr(), d_pstat.data_ptr())
 
@@ -237,17 +242,25 @@ def run_ours(args):
         prof = prob.last_solve_profile()
         launches_per_step = prof.total_launches + 2
 
-        # per-part device times (same launch configuration, measured after the timed region)
+        # per-part device times (same launch configuration, measured after the timed region): the
+        # whole solve as the timed step runs it, then its phases with events between them (which
+        # cost a few microseconds: a phase's kernels are then no longer launched under the tail of
+        # the previous phase)
         sweep_ms, rank_ms, fin_ms, solve_ms = [], [], [], []
+        for _ in range(9):
+            prob.solve_exact_dev(d_sol.data_ptr())
+            solve_ms.append(prob.last_solve_profile().ms_total)
+        prob.set_profiling(True)
         for _ in range(7):
             prob.solve_exact_dev(d_sol.data_ptr())
             pr = prob.last_solve_profile()
             sweep_ms.append(pr.ms_sweep)
             rank_ms.append(pr.ms_rank)
             fin_ms.append(pr.ms_finalize)
-            solve_ms.append(pr.ms_total)
+        prob.set_profiling(False)
         e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-        batch_ms, eval_ms = [], []
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # larger than the 126 MB L2
+        batch_ms, eval_ms, eval_cold_ms = [], [], []
         for _ in range(7):
             e0.record(stream)
             batch_device()
@@ -257,6 +270,40 @@ def run_ours(args):
             stream.synchronize()
             batch_ms.append(e0.elapsed_time(e1))
             eval_ms.append(e1.elapsed_time(e2))
+        eval32_cold_ms = []
+        for _ in range(7):  # the evaluator alone with its plans evicted from L2 first; both row layouts
+            flush.fill_(1)
+            e0.record(stream)
+            eval_device()
+            e1.record(stream)
+            stream.synchronize()
+            eval_cold_ms.append(e0.elapsed_time(e1))
+            flush.fill_(1)
+            e0.record(stream)
+            eval_device_int32()
+            e1.record(stream)
+            stream.synchronize()
+            eval32_cold_ms.append(e0.elapsed_time(e1))
+
+        # sustained leg: the Large solve back to back for about two seconds, clocks sampled meanwhile
+        # (the sweep is bound by an ALU pipe, so its time follows the SM clock the part settles at)
+        n_sus = max(50, int(2000.0 / statistics.median(solve_ms)))
+        with ClockSampler(local) as sus_clocks:
+            e0.record(stream)
+            for _ in range(n_sus):
+                prob.solve_exact_dev(d_sol.data_ptr())
+            e1.record(stream)
+            stream.synchronize()
+        sus_ms = e0.elapsed_time(e1) / n_sus
+        sus_clk = sus_clocks.summary()
+        sustained = {"solves": n_sus, "large_solve_ms_sustained": sus_ms,
+                     "sm_mhz_median": sus_clk["sm_mhz"] if sus_clk else None,
+                     "ms_times_mhz": sus_ms * sus_clk["sm_mhz"] if sus_clk else None,
+                     "reasons": sus_clk["reasons"] if sus_clk else None}
+
+        # issue rate of the packed min/max forms the sweep is made of, measured now on this part
+        rates = {"minmax_u16x2": pp.debug_minmax_rate(0), "min3_u16x2": pp.debug_minmax_rate(1),
+                 "max3_u16x2": pp.debug_minmax_rate(2)}
 
         # the paper's greedy comparison baseline on the batched instances (not part of the timed
         # step): device time of one launch, and how far its plans are from the exact optimum
@@ -314,14 +361,19 @@ def run_ours(args):
         # time of one exact solve each, for context
         other = {}
         for name, inst in (("tiny_k6_L12", W.config_tiny()), ("resnet50_shaped_k10_L50", W.config_resnet50_shaped()),
-                           ("deeper_cnn_k14_L100", W.config_deeper_cnn())):
+                           ("deeper_cnn_k14_L100", W.config_deeper_cnn()),
+                           ("large_unequal_layer_memory_k18_L200", W.large_unequal_layers())):
             with pp.Problem.from_instance(inst) as q:
                 q.set_stream(stream.cuda_stream)
+                if inst.k == k:
+                    q.set_workspace(ws)  # the Large problem is idle here
                 ts = []
                 for _ in range(6):
                     q.solve_exact_dev(d_sol2.data_ptr())
                     ts.append(q.last_solve_profile().ms_total)
-                other[name] = {"solve_ms": min(ts[2:]), "relaxations_per_s": n_relax(inst.k, inst.L) / (min(ts[2:]) * 1e-3)}
+                qp = q.last_solve_profile()
+                other[name] = {"solve_ms": min(ts[2:]), "relaxations_per_s": n_relax(inst.k, inst.L) / (min(ts[2:]) * 1e-3),
+                               "state_bytes": qp.state_bytes, "fast_path": qp.fast_path, "pair_levels": qp.pair_levels}
 
     sol_rec = pp.pp_solution.from_buffer_copy(d_sol.cpu().numpy().tobytes())
     ms_per_step = ms_total / args.steps
@@ -329,7 +381,7 @@ def run_ours(args):
 
     # ---- end to end through the host-pointer entry points ----
     h2d = (large.layer_out_bits.nbytes + large.layer_mem_bytes.nbytes + large.node_mem_bytes.nbytes
-           + large.bw_kbps.nbytes + nseg.nbytes + ends.nbytes + nodes.nbytes
+           + large.bw_kbps.nbytes + nseg.nbytes + p_off.nbytes + p_ends.nbytes + p_nodes.nbytes
            + b_bits.nbytes + b_mem.nbytes + b_cap.nbytes + b_bw.nbytes)
     d2h = (ctypes.sizeof(pp.pp_solution) + N_PLANS * 9
            + N_BATCH * (8 + 4 + 4 * (BATCH_K - 1) + 4 * BATCH_K + 1))
@@ -338,7 +390,8 @@ def run_ours(args):
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory().numpy()
     h_bits, h_mem, h_cap, h_bw = (pin(a) for a in (large.layer_out_bits, large.layer_mem_bytes,
                                                     large.node_mem_bytes, large.bw_kbps))
-    h_nseg, h_ends, h_nodes = pin(nseg), pin(ends), pin(nodes)
+    h_nseg, h_off, h_pends, h_pnodes = pin(nseg), pin(p_off.view(np.int32)).view(np.uint32), \
+        pin(p_ends.view(np.int16)).view(np.uint16), pin(p_nodes)
     hb_bits, hb_mem, hb_cap, hb_bw = pin(b_bits), pin(b_mem), pin(b_cap), pin(b_bw)
 
     def step_host():
@@ -346,7 +399,7 @@ def run_ours(args):
             p2.set_workspace(ws)
             s = p2.solve_exact()
             bsol = pp.solve_exact_batch(BATCH_L, BATCH_K, hb_bits, hb_mem, hb_cap, hb_bw)
-            beta, pstat = p2.eval_plans(h_nseg, h_ends, h_nodes)
+            beta, pstat = p2.eval_plans_packed(h_nseg, h_off, h_pends, h_pnodes)
         return s, bsol, beta, pstat
 
     for _ in range(2):
@@ -361,29 +414,76 @@ def run_ours(args):
     e2e_value, e2e_s = aggregate_over_ranks(relax_step, e2e_local, dist, dev)
     assert host_out[0].beta_ms == sol_rec.beta_ms and host_out[0].m == sol_rec.m
 
-    # ---- roofline of the dominant kernel (the popcount sweep of the Large instance) ----
+    # ---- roofline ----
+    # The DP roofline is the slower of (state bytes at HBM bandwidth) and (min/max element-ops at the
+    # ALU rate): every state is written once and read once (2 * states * element bytes); a
+    # relaxation is one max and one min, the window step about three more ops per state.  The ALU
+    # rate is the packed min/max issue rate measured above x 32 lanes x 2 elements x SMs x max clock.
     peaks, which = measured_peaks()
+    med = statistics.median
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    clock_hz = peaks.get("sm_max_mhz", 1965.0) * 1e6
+    minmax_rate = min(rates["minmax_u16x2"], rates["min3_u16x2"])  # warp instructions per clock per SM
+    alu_peak = minmax_rate * 32 * 2 * sms * clock_hz             # element-ops per second
+
+    def dp_roofline(kk, LL, elem_bytes, solve_ms_):
+        bytes_ = 2 * n_states(kk, LL) * elem_bytes
+        ops_ = 2 * n_relax(kk, LL) + 3 * n_states(kk, LL)
+        t_mem = bytes_ / (peaks["hbm_gbs"] * 1e9) * 1e3
+        t_mem_nom = bytes_ / (NOMINAL_HBM_GBS * 1e9) * 1e3
+        t_alu = ops_ / alu_peak * 1e3
+        return {"algorithmic_bytes": bytes_, "algorithmic_ops": ops_, "t_mem_ms": t_mem, "t_alu_ms": t_alu,
+                "t_mem_ms_at_8TBps": t_mem_nom, "bound": "hbm" if t_mem >= t_alu else "alu",
+                "solve_ms": solve_ms_, "frac": max(t_mem, t_alu) / solve_ms_,
+                "frac_at_8TBps": max(t_mem_nom, t_alu) / solve_ms_}
+
     elem = prof.state_bytes
-    sweep_t = statistics.median(sweep_ms) * 1e-3
-    alg_bytes = 2 * n_states(k, L) * elem  # every state written once and read once
-    achieved = alg_bytes / sweep_t / 1e9
+    sweep_t = med(sweep_ms) * 1e-3
+    whole = dp_roofline(k, L, elem, med(solve_ms))
+    alg_bytes = whole["algorithmic_bytes"]
+    alu_ops = whole["algorithmic_ops"]
     n_launch = prof.sweep_launches
-    # the same sweep against the plain-ALU bound: 2 element-ops per relaxation + 3 per state, at
-    # the measured packed min/max rate and the maximum SM clock
-    alu_ops = 2 * relax_large + 3 * n_states(k, L)
-    alu_peak = PACKED_MINMAX_LANES_PER_CLK_SM * 2 * 148 * peaks.get("sm_max_mhz", 1965.0) * 1e6
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"],
+    if whole["bound"] == "hbm":
+        achieved, peak, unit = alg_bytes / sweep_t / 1e9, peaks["hbm_gbs"], "GB/s"
+    else:
+        achieved, peak, unit = alu_ops / sweep_t / 1e12, alu_peak / 1e12, "Tops/s"
+    roofline = {"bound": whole["bound"], "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak,
                 "traffic": SWEEP_DRAM_BYTES_PER_LAUNCH if prof.fast_path else None,
-                "peak_source": which + " (burst copy figure; the sweep is timed alone)",
-                "kernel": "k_sweep_pair + k_sweep_fast + k_base (%d launches per solve)" % n_launch,
+                "peak_source": (which + " (burst copy figure; the sweep is timed alone)") if whole["bound"] == "hbm"
+                               else "measured in this run (packed min/max issue rate x max SM clock)",
+                "kernel": "k_sweep_pair + k_sweep_fast (%d launches per solve, one per popcount level)" % n_launch,
                 "algorithmic_bytes_per_launch": alg_bytes / n_launch,
                 "ms_per_launch": sweep_t * 1e3 / n_launch,
                 "algorithmic_bytes_per_solve": alg_bytes, "sweep_ms": sweep_t * 1e3,
+                "hbm": {"achieved_GBps": alg_bytes / sweep_t / 1e9, "peak_GBps": peaks["hbm_gbs"],
+                        "frac": alg_bytes / sweep_t / 1e9 / peaks["hbm_gbs"], "peak_source": which},
                 "alu": {"ops_per_solve": alu_ops, "achieved_ops_per_s": alu_ops / sweep_t,
-                        "peak_ops_per_s": alu_peak, "frac": alu_ops / sweep_t / alu_peak}}
+                        "peak_ops_per_s": alu_peak, "frac": alu_ops / sweep_t / alu_peak,
+                        "warp_instr_per_clk_per_sm": rates, "lanes_per_clk_per_sm": minmax_rate * 32,
+                        "peak_source": "measured in this run"},
+                "whole_solve": whole,
+                "sustained": sustained}
+    # the other parts of the step against their own bounds
+    c3 = W.config_deeper_cnn()
+    o3 = other["deeper_cnn_k14_L100"]
+    unl = other["large_unequal_layer_memory_k18_L200"]
+    # per plan: nseg, its offset, nseg - 1 cuts of 2 bytes, nseg nodes of 1 byte in; beta and flags out
+    plan_bytes = 5 * N_PLANS + 3 * n_entries - 2 * int((np.diff(p_off.astype(np.int64)) > 0).sum()) + 9 * N_PLANS
+    ev_cold = med(eval_cold_ms) * 1e-3
+    batch_ops = N_BATCH * (2 * n_relax(BATCH_K, BATCH_L) + 3 * n_states(BATCH_K, BATCH_L))
+    part_rooflines = {
+        "deeper_cnn_k14_L100": dp_roofline(c3.k, c3.L, o3["state_bytes"], o3["solve_ms"]),
+        "large_unequal_layer_memory_k18_L200": dp_roofline(k, L, unl["state_bytes"], unl["solve_ms"]),
+        "evaluator": {"bound": "hbm", "algorithmic_bytes": plan_bytes, "bytes_per_plan": plan_bytes / N_PLANS,
+                      "ms_cold": ev_cold * 1e3, "achieved_GBps": plan_bytes / ev_cold / 1e9,
+                      "frac": plan_bytes / ev_cold / 1e9 / peaks["hbm_gbs"],
+                      "note": "inputs evicted from L2 before each timed launch; eval_ms in the breakdown is "
+                              "the launch inside the step, whose inputs may still be L2-resident"},
+        "batch": {"bound": "alu", "algorithmic_ops": batch_ops, "t_alu_ms": batch_ops / alu_peak * 1e3,
+                  "batch_ms": med(batch_ms), "frac": batch_ops / alu_peak * 1e3 / med(batch_ms)},
+    }
 
-    med = statistics.median
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -396,7 +496,10 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "gpu_launches": launches_per_step * args.steps,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-                "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_s * 1e3},
+                "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_s * 1e3,
+                "workspace": "the %.2f GB search scratch is allocated once by the caller and handed to every "
+                             "step's problem (pp_problem_set_workspace); it is not part of the timed copies"
+                             % (prob.workspace_bytes() / 1e9)},
         "clocks": clk,
         "roofline": roofline,
         "breakdown": {
@@ -405,6 +508,10 @@ def run_ours(args):
             "large_relaxations_per_s": relax_large / (med(solve_ms) * 1e-3),
             "batch_ms": med(batch_ms), "instances_per_s": N_BATCH / (med(batch_ms) * 1e-3),
             "eval_ms": med(eval_ms), "plans_per_s": N_PLANS / (med(eval_ms) * 1e-3),
+            "eval_cold_ms": med(eval_cold_ms), "plans_per_s_cold": N_PLANS / (med(eval_cold_ms) * 1e-3),
+            "eval_int32_rows_cold_ms": med(eval32_cold_ms),
+            "batch_roofline": part_rooflines["batch"],
+            "part_rooflines": part_rooflines,
             "fast_path": prof.fast_path, "beta_ms": sol_rec.beta_ms, "segments": sol_rec.m,
             "greedy_baseline_batched": greedy,
             "random_baseline_large": random_base,

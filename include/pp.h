@@ -160,6 +160,26 @@ pp_status pp_eval_plans_dev(pp_problem *p, int64_t B, const uint8_t *nseg, const
                             const int32_t *nodes, double *beta_ms, uint8_t *plan_status);
 
 /*
+ * The same evaluator (Eq. 3 per cut, Eq. 2 per plan, same validity rules and flags) for plans in
+ * compressed rows: a third of the bytes of the int32 layout, for callers that score plans in bulk.
+ *   nseg      [B]      number of segments of each plan
+ *   plan_off  [B + 1]  plan b owns entries plan_off[b] .. plan_off[b + 1] - 1 of `ends` and `nodes`
+ *                      (non-decreasing; normally the running sum of nseg)
+ *   ends      [total]  16-bit cuts: the first nseg - 1 entries of a plan's row are read
+ *   nodes     [total]  8-bit node ids: the first nseg entries of a plan's row are read
+ *   beta_ms [B], plan_status [B]   out, as for pp_eval_plans; a row that holds fewer than nseg
+ *                      entries, or reaches beyond `total`, is flagged PP_PLAN_BAD_NSEG
+ * Host variant: host pointers, synchronous.  _dev variant: device pointers, asynchronous on the
+ * problem's stream.  B == 0 is a no-op.
+ */
+pp_status pp_eval_plans_packed(pp_problem *p, int64_t B, int64_t total, const uint8_t *nseg,
+                               const uint32_t *plan_off, const uint16_t *ends, const uint8_t *nodes,
+                               double *beta_ms, uint8_t *plan_status);
+pp_status pp_eval_plans_packed_dev(pp_problem *p, int64_t B, int64_t total, const uint8_t *nseg,
+                                   const uint32_t *plan_off, const uint16_t *ends, const uint8_t *nodes,
+                                   double *beta_ms, uint8_t *plan_status);
+
+/*
  * Many independent instances of the same shape (L, k) in one call; each instance is the
  * exact search above, done by one thread block with its whole state table in shared memory.
  *   out_bits [B*L], mem [B*L], node_mem [B*k], bw [B*k*k]   inputs, instance-major
@@ -249,8 +269,8 @@ pp_status pp_debug_mask_order(int32_t k, uint32_t *masks_out, uint32_t *level_of
 /* Measurement hook: issue rate of the packed 16-bit min/max instructions the sweep consists of, on
  * the current device.  One block of 1024 threads per SM runs `iters` trips of 64 dependent-chain
  * instructions per thread on registers only, timed with the SM's own cycle counter; the median over
- * the SMs gives *warp_instr_per_clk_per_sm (host).  op: 0 = two-input packed minimum, 1 = two-input
- * packed maximum, 2 = three-input packed minimum.  The ALU bound of the search's roofline is this
+ * the SMs gives *warp_instr_per_clk_per_sm (host).  op: 0 = two-input packed minimum and maximum in
+ * turn, 1 = three-input packed minimum, 2 = three-input packed maximum.  The ALU bound of the search's roofline is this
  * rate x 32 lanes x 2 elements x SMs x clock.  Synchronous, legacy default stream; allocates and
  * frees a few hundred bytes of device memory. */
 pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm);

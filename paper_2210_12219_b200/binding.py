@@ -27,7 +27,7 @@ EXPORTS = (
     "pp_solve_exact_batch_dev", "pp_last_solve_profile", "pp_debug_read_state_row", "pp_debug_mask_order",
     "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str", "pp_greedy_batch",
     "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev", "pp_debug_minmax_rate",
-    "pp_problem_set_profiling",
+    "pp_problem_set_profiling", "pp_eval_plans_packed", "pp_eval_plans_packed_dev",
 )
 
 
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.pp_solve_exact_dev.argtypes = [vp, vp]
         L.pp_eval_plans.argtypes = [vp, i64, vp, vp, vp, vp, vp]
         L.pp_eval_plans_dev.argtypes = [vp, i64, vp, vp, vp, vp, vp]
+        L.pp_eval_plans_packed.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp]
+        L.pp_eval_plans_packed_dev.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp]
         L.pp_solve_exact_batch.argtypes = [i64, i32, i32] + [vp] * 9
         L.pp_solve_exact_batch_dev.argtypes = [i64, i32, i32] + [vp] * 10
         L.pp_greedy_batch.argtypes = [i64, i32, i32] + [vp] * 9
@@ -223,6 +225,26 @@ class Problem:
         _check(lib().pp_eval_plans_dev(self._h, int(B), *(ctypes.c_void_p(x) for x in
                                        (nseg_ptr, ends_ptr, nodes_ptr, beta_ptr, status_ptr))),
                "pp_eval_plans_dev")
+
+    def eval_plans_packed(self, nseg, plan_off, ends, nodes):
+        """pp_eval_plans_packed: uint8 [B], uint32 [B + 1], uint16 [total], uint8 [total] (host) ->
+        (beta_ms float64 [B], plan_status uint8 [B])."""
+        nseg, p0 = _host(nseg, np.uint8)
+        B = nseg.shape[0]
+        plan_off, p1 = _host(plan_off, np.uint32)
+        ends, p2 = _host(ends, np.uint16)
+        nodes, p3 = _host(nodes, np.uint8)
+        assert plan_off.size == B + 1 and ends.size == nodes.size
+        beta = np.empty(B, dtype=np.float64)
+        status = np.empty(B, dtype=np.uint8)
+        _check(lib().pp_eval_plans_packed(self._h, B, ends.size, p0, p1, p2, p3, ctypes.c_void_p(beta.ctypes.data),
+                                          ctypes.c_void_p(status.ctypes.data)), "pp_eval_plans_packed")
+        return beta, status
+
+    def eval_plans_packed_dev(self, B, total, nseg_ptr, off_ptr, ends_ptr, nodes_ptr, beta_ptr, status_ptr):
+        _check(lib().pp_eval_plans_packed_dev(self._h, int(B), int(total), *(ctypes.c_void_p(x) for x in
+                                              (nseg_ptr, off_ptr, ends_ptr, nodes_ptr, beta_ptr, status_ptr))),
+               "pp_eval_plans_packed_dev")
 
     # -- random comparison baseline -------------------------------------------------------
     def random_plans(self, draws):

@@ -566,6 +566,47 @@ pp_status pp_eval_plans(pp_problem *p, int64_t B, const uint8_t *nseg, const int
     return from_cuda(e2);
 }
 
+pp_status pp_eval_plans_packed_dev(pp_problem *p, int64_t B, int64_t total, const uint8_t *nseg,
+                                   const uint32_t *plan_off, const uint16_t *ends, const uint8_t *nodes,
+                                   double *beta_ms, uint8_t *plan_status)
+{
+    if (!p || B < 0 || total < 0) return PP_ERR_ARG;
+    if (B == 0) return PP_OK;
+    if (!nseg || !plan_off || !beta_ms || !plan_status || ((!ends || !nodes) && total > 0)) return PP_ERR_ARG;
+    PP_CUDA(launch_eval_packed(p->d, B, total, nseg, plan_off, ends, nodes, beta_ms, plan_status, p->stream));
+    return PP_OK;
+}
+
+pp_status pp_eval_plans_packed(pp_problem *p, int64_t B, int64_t total, const uint8_t *nseg,
+                               const uint32_t *plan_off, const uint16_t *ends, const uint8_t *nodes,
+                               double *beta_ms, uint8_t *plan_status)
+{
+    if (!p || B < 0 || total < 0) return PP_ERR_ARG;
+    if (B == 0) return PP_OK;
+    if (!nseg || !plan_off || !beta_ms || !plan_status || ((!ends || !nodes) && total > 0)) return PP_ERR_ARG;
+    const size_t nB = (size_t)B, nT = (size_t)total;
+    const size_t o_off = align_up(nB, 256), o_ends = align_up(o_off + (nB + 1) * 4, 256);
+    const size_t o_nodes = align_up(o_ends + nT * 2, 256), o_beta = align_up(o_nodes + nT, 256);
+    const size_t o_st = align_up(o_beta + nB * 8, 256), bytes = o_st + nB;
+    unsigned char *buf = nullptr;
+    cudaStream_t s = p->stream;
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), bytes, s));
+    cudaError_t e = cudaMemcpyAsync(buf, nseg, nB, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(buf + o_off, plan_off, (nB + 1) * 4, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && nT) e = cudaMemcpyAsync(buf + o_ends, ends, nT * 2, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && nT) e = cudaMemcpyAsync(buf + o_nodes, nodes, nT, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+        e = launch_eval_packed(p->d, B, total, buf, reinterpret_cast<uint32_t *>(buf + o_off),
+                               reinterpret_cast<uint16_t *>(buf + o_ends), buf + o_nodes,
+                               reinterpret_cast<double *>(buf + o_beta), buf + o_st, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(beta_ms, buf + o_beta, nB * 8, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(plan_status, buf + o_st, nB, cudaMemcpyDeviceToHost, s);
+    cudaFreeAsync(buf, s);
+    cudaError_t e2 = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return from_cuda(e);
+    return from_cuda(e2);
+}
+
 pp_status pp_random_plans_dev(pp_problem *p, int64_t P, const uint32_t *draws, uint8_t *nseg, int32_t *ends,
                               int32_t *nodes)
 {

@@ -67,6 +67,9 @@ cudaError_t launch_sweep_pair(const Dev &d, int level, cudaStream_t s, bool firs
 cudaError_t launch_finalize(const Dev &d, pp_solution *out, cudaStream_t s, bool dependent);
 cudaError_t launch_eval(const Dev &d, int64_t B, const uint8_t *nseg, const int32_t *ends,
                         const int32_t *nodes, double *beta, uint8_t *status, cudaStream_t s);
+cudaError_t launch_eval_packed(const Dev &d, int64_t B, int64_t total, const uint8_t *nseg, const uint32_t *off,
+                               const uint16_t *ends, const uint8_t *nodes, double *beta, uint8_t *status,
+                               cudaStream_t s);
 size_t batch_smem_bytes(int L, int k);
 cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
                          const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,

@@ -12,13 +12,21 @@ constexpr int kProbeThreads = 1024;
 constexpr int kProbeChains = 8;    // independent accumulators per thread
 constexpr int kProbeUnroll = 8;    // instructions per accumulator per loop trip
 
+// OP 0: two-input forms, minimum and maximum in turn (a chain of minima alone could be merged into
+// three-input instructions by the assembler and would then count double); OP 1 / OP 2: the
+// three-input minimum / maximum, one instruction each on this architecture.
 template <int OP>
-__device__ __forceinline__ uint32_t probe_op(uint32_t a, uint32_t b, uint32_t c)
+__device__ __forceinline__ uint32_t probe_op(uint32_t a, uint32_t b, uint32_t c, int u)
 {
     uint32_t r;
-    if (OP == 0) asm volatile("min.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    else if (OP == 1) asm volatile("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    else r = __vimin3_u16x2(a, b, c);  // three-input form: one instruction on this architecture
+    if (OP == 0) {
+        if (u & 1) asm volatile("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        else asm volatile("min.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(c));
+    } else if (OP == 1) {
+        r = __vimin3_u16x2(a, b, c);
+    } else {
+        r = __vimax3_u16x2(a, b, c);
+    }
     return r;
 }
 
@@ -37,7 +45,7 @@ k_probe(int iters, uint32_t seed, long long *cycles, uint32_t *sink)
 #pragma unroll
         for (int u = 0; u < kProbeUnroll; ++u)
 #pragma unroll
-            for (int i = 0; i < kProbeChains; ++i) acc[i] = probe_op<OP>(acc[i], bi + u, c + i);
+            for (int i = 0; i < kProbeChains; ++i) acc[i] = probe_op<OP>(acc[i], bi + u, c + i, u);
     }
     __syncthreads();
     const long long t1 = clock64();

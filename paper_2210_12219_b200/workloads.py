@@ -273,3 +273,20 @@ def random_plans(inst: Instance, count: int, seed: int, invalid_fraction: float 
         else:
             nodes[b, 0] = k + int(rng.integers(0, 3))
     return nseg, ends, nodes
+
+
+def pack_plans(nseg: np.ndarray, ends: np.ndarray, nodes: np.ndarray):
+    """Compressed rows for the packed evaluator entry point: plan b keeps its first nseg[b] entries
+    (none when nseg is outside [1, k]).  Values that 16 / 8 bits cannot hold are mapped to the
+    largest code, which is out of range as well.  Returns (plan_off uint32 [B + 1], ends uint16
+    [total], nodes uint8 [total])."""
+    B, k = ends.shape
+    keep = np.where((nseg >= 1) & (nseg <= k), nseg, 0).astype(np.int64)
+    plan_off = np.zeros(B + 1, dtype=np.uint32)
+    plan_off[1:] = np.cumsum(keep)
+    sel = np.arange(k)[None, :] < keep[:, None]
+    e = ends[sel].astype(np.int64)
+    n = nodes[sel].astype(np.int64)
+    e = np.where((e < 0) | (e > 0xFFFF), 0xFFFF, e).astype(np.uint16)
+    n = np.where((n < 0) | (n > 0xFF), 0xFF, n).astype(np.uint8)
+    return plan_off, e, n

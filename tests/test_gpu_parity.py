@@ -310,6 +310,67 @@ def test_evaluator_against_oracle():
                                 np.zeros((0, inst.k), np.int32))[0].shape == (0,)
 
 
+def test_packed_evaluator_against_oracle():
+    # compressed rows (16-bit cuts, 8-bit nodes, offsets) score like the int32 rows
+    for inst, B in ((W.config_tiny(), 3000), (W.config_resnet50_shaped(), 3000), (W.config_large(), 6000),
+                    (W.random_small(50001, 300, 9, dead_links=0.2), 2000)):
+        nseg, ends, nodes = W.random_plans(inst, B, seed=B + 3 * inst.k, invalid_fraction=0.15)
+        want_beta, want_status = oracle.eval_plans(inst, nseg, ends, nodes)
+        off, e16, n8 = W.pack_plans(nseg, ends, nodes)
+        with pp.Problem.from_instance(inst) as p:
+            beta, status = p.eval_plans_packed(nseg, off, e16, n8)
+            assert np.array_equal(status, want_status)
+            assert np.array_equal(beta, want_beta)
+            assert (status != 0).sum() > 10 and len(set(status.tolist())) >= 4
+            assert inst.L > 200 or (status == 0).sum() > 10  # the long chain's random plans rarely fit
+            # a row shorter than its nseg, and a row that reaches beyond the arrays, are refused
+            bad_off = off.copy()
+            victim = int(np.flatnonzero(nseg > 2)[0])
+            bad_off[victim + 1:] -= 1
+            b2, s2 = p.eval_plans_packed(nseg, bad_off, e16, n8)
+            assert s2[victim] == pp.PP_PLAN_BAD_NSEG and np.isinf(b2[victim])
+            b3, s3 = p.eval_plans_packed(nseg[:5], off[:6], e16[:int(off[5]) - 1], n8[:int(off[5]) - 1])
+            last = max(b for b in range(5) if off[b + 1] > off[b])  # the last plan with entries loses one
+            assert s3[last] == pp.PP_PLAN_BAD_NSEG
+            assert p.eval_plans_packed(np.zeros(0, np.uint8), np.zeros(1, np.uint32), np.zeros(0, np.uint16),
+                                       np.zeros(0, np.uint8))[0].shape == (0,)
+
+
+def test_evaluator_beyond_one_pass_of_the_grid():
+    # more plans than one pass of the evaluator's grid covers (148 * 16 blocks of 256): the later
+    # passes of the grid-stride loop are compared with the oracle too (the plans repeat with period
+    # 5003, the oracle scores one period)
+    inst = W.config_resnet50_shaped()
+    period, B = 5003, 700_001
+    nseg, ends, nodes = W.random_plans(inst, period, seed=99, invalid_fraction=0.1)
+    want_beta, want_status = oracle.eval_plans(inst, nseg, ends, nodes)
+    idx = np.arange(B) % period
+    with pp.Problem.from_instance(inst) as p:
+        beta, status = p.eval_plans(nseg[idx], ends[idx], nodes[idx])
+        assert np.array_equal(status, want_status[idx]) and np.array_equal(beta, want_beta[idx])
+        off, e16, n8 = W.pack_plans(nseg[idx], ends[idx], nodes[idx])
+        beta, status = p.eval_plans_packed(nseg[idx], off, e16, n8)
+        assert np.array_equal(status, want_status[idx]) and np.array_equal(beta, want_beta[idx])
+
+
+def test_minmax_rate_hook_and_phase_profile():
+    # the issue-rate hook returns plausible rates (one to four warp instructions per clock per SM),
+    # and the phase times are reported only when asked for
+    for op in range(3):
+        rate = pp.debug_minmax_rate(op, 512)
+        assert 0.5 < rate < 4.5, (op, rate)
+    inst = W.config_resnet50_shaped()
+    with pp.Problem.from_instance(inst) as p:
+        p.solve_exact()
+        prof = p.last_solve_profile()
+        assert prof.ms_total > 0 and prof.ms_sweep == 0 and prof.ms_rank == 0
+        p.set_profiling(True)
+        p.solve_exact()
+        prof = p.last_solve_profile()
+        assert prof.ms_sweep > 0 and prof.ms_rank > 0 and prof.ms_finalize > 0
+        assert prof.sweep_launches == min(inst.k, inst.L) - 1
+
+
 def _stack(insts):
     return (np.stack([i.layer_out_bits for i in insts]), np.stack([i.layer_mem_bytes for i in insts]),
             np.stack([i.node_mem_bytes for i in insts]), np.stack([i.bw_kbps for i in insts]))
