@@ -247,6 +247,32 @@ pp_status pp_greedy_batch_dev(int64_t B, int32_t L, int32_t k, const uint64_t *o
                               double *beta_ms, int32_t *m, int32_t *cuts, int32_t *placement,
                               int8_t *status, void *cuda_stream);
 
+/*
+ * Partition stage of the paper's two-stage heuristic (Section 3.2.1: the partition graph of Eq. 6
+ * and Eq. 7, Algorithm 1), for B independent chains of the same length: cut the chain into
+ * contiguous partitions that each fit one node's memory kappa (the paper's homogeneous capacity),
+ * so that the sum of the weights of the cuts is smallest.  A cut after point c weighs
+ * cut_weight[c]: the paper uses the transfer-size class of the point, pass raw sizes or class
+ * numbers.  Of several plans with the same sum the one with fewer partitions is returned, then the
+ * one whose cuts come earlier (the paper leaves ties open).
+ *   cut_weight [B*L], mem [B*L], kappa [B]     inputs, chain-major; weights below PP_MAX_BITS
+ *   cap_seg    rows of `cuts` / `sizes` have this many entries (cuts beyond it are not written)
+ *   cost [B]   sum of the weights of the chosen cuts;  m [B] number of partitions
+ *   cuts [B*cap_seg]   Q: last point of every partition but the final one, rest -1
+ *   sizes [B*cap_seg]  S: cut_weight at those points, rest 0 (may be NULL)
+ *   status [B] PP_OK; PP_INFEASIBLE (some point exceeds kappa: cost 0, m 0); PP_ERR_LIMIT (a weight
+ *              above the limit or a wrapping memory sum, or m - 1 > cap_seg: cost and m are still set)
+ * The cuts feed pp_eval_plans as `ends` once nodes are chosen for the partitions.  Host variant:
+ * host pointers, synchronous, legacy default stream.  _dev variant: device pointers, asynchronous
+ * on `cuda_stream`.  B == 0 is a no-op.
+ */
+pp_status pp_partition_minsum_batch(int64_t B, int32_t L, const uint64_t *cut_weight, const uint64_t *mem,
+                                    const uint64_t *kappa, int32_t cap_seg, uint64_t *cost, int32_t *m,
+                                    int32_t *cuts, uint64_t *sizes, int8_t *status);
+pp_status pp_partition_minsum_batch_dev(int64_t B, int32_t L, const uint64_t *cut_weight, const uint64_t *mem,
+                                        const uint64_t *kappa, int32_t cap_seg, uint64_t *cost, int32_t *m,
+                                        int32_t *cuts, uint64_t *sizes, int8_t *status, void *cuda_stream);
+
 /* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream.
  * ms_total is always measured.  ms_rank, ms_sweep and ms_finalize need events between the
  * phases, which keep one phase's kernels from being launched under the tail of the previous

@@ -28,6 +28,7 @@ EXPORTS = (
     "pp_problem_force_generic", "pp_solve_exact_static", "pp_status_str", "pp_greedy_batch",
     "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev", "pp_debug_minmax_rate",
     "pp_problem_set_profiling", "pp_eval_plans_packed", "pp_eval_plans_packed_dev",
+    "pp_partition_minsum_batch", "pp_partition_minsum_batch_dev",
 )
 
 
@@ -87,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.pp_problem_set_profiling.argtypes = [vp, i32]
         L.pp_solve_exact_static.argtypes = [i32, vp, vp, i32, vp, vp, vp, vp]
         L.pp_debug_minmax_rate.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
+        L.pp_partition_minsum_batch.argtypes = [i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp]
+        L.pp_partition_minsum_batch_dev.argtypes = [i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.pp_status_str.argtypes = [ctypes.c_int]
         L.pp_status_str.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -313,6 +316,41 @@ def debug_mask_order(k: int):
     _check(lib().pp_debug_mask_order(int(k), ctypes.c_void_p(masks.ctypes.data),
                                      ctypes.c_void_p(level_off.ctypes.data)), "pp_debug_mask_order")
     return masks, level_off
+
+
+@dataclass
+class PartitionBatch:
+    cost: np.ndarray    # uint64 [B]
+    m: np.ndarray       # int32 [B]
+    cuts: np.ndarray    # int32 [B, cap_seg]
+    sizes: np.ndarray   # uint64 [B, cap_seg]
+    status: np.ndarray  # int8 [B]
+
+
+def partition_minsum_batch(cut_weight, mem, kappa, cap_seg: int) -> PartitionBatch:
+    """pp_partition_minsum_batch: host arrays [B, L], [B, L], [B] -> PartitionBatch (synchronous)."""
+    cut_weight, p0 = _host(cut_weight, np.uint64)
+    B, L = cut_weight.shape
+    mem, p1 = _host(mem, np.uint64)
+    kappa, p2 = _host(kappa, np.uint64)
+    assert mem.shape == (B, L) and kappa.shape == (B,)
+    cost = np.empty(B, dtype=np.uint64)
+    m = np.empty(B, dtype=np.int32)
+    cuts = np.full((B, max(cap_seg, 1)), -1, dtype=np.int32)
+    sizes = np.zeros((B, max(cap_seg, 1)), dtype=np.uint64)
+    status = np.empty(B, dtype=np.int8)
+    st = lib().pp_partition_minsum_batch(B, L, p0, p1, p2, int(cap_seg), *(ctypes.c_void_p(a.ctypes.data) for a in
+                                         (cost, m, cuts, sizes, status)))
+    _check(st, "pp_partition_minsum_batch")
+    return PartitionBatch(cost, m, cuts[:, :cap_seg], sizes[:, :cap_seg], status)
+
+
+def partition_minsum_batch_dev(B, L, weight_ptr, mem_ptr, kappa_ptr, cap_seg, cost_ptr, m_ptr, cuts_ptr, sizes_ptr,
+                               status_ptr, cuda_stream: int = 0):
+    st = lib().pp_partition_minsum_batch_dev(int(B), int(L), *(ctypes.c_void_p(x) for x in (weight_ptr, mem_ptr, kappa_ptr)),
+                                             int(cap_seg), *(ctypes.c_void_p(x) for x in
+                                             (cost_ptr, m_ptr, cuts_ptr, sizes_ptr, status_ptr, cuda_stream)))
+    _check(st, "pp_partition_minsum_batch_dev")
 
 
 def debug_minmax_rate(op: int, iters: int = 2048) -> float:

@@ -749,6 +749,57 @@ pp_status pp_greedy_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_b
                            placement, status);
 }
 
+pp_status pp_partition_minsum_batch_dev(int64_t B, int32_t L, const uint64_t *cut_weight, const uint64_t *mem,
+                                        const uint64_t *kappa, int32_t cap_seg, uint64_t *cost, int32_t *m,
+                                        int32_t *cuts, uint64_t *sizes, int8_t *status, void *cuda_stream)
+{
+    if (B < 0 || L < 1 || cap_seg < 0) return PP_ERR_ARG;
+    if (L > PP_MAX_L) return PP_ERR_LIMIT;
+    if (B == 0) return PP_OK;
+    if (!cut_weight || !mem || !kappa || !cost || !m || !status || (!cuts && cap_seg > 0)) return PP_ERR_ARG;
+    PP_CUDA(launch_partition_minsum(B, L, cap_seg, cut_weight, mem, kappa, cost, m, cuts, sizes, status,
+                                    static_cast<cudaStream_t>(cuda_stream)));
+    return PP_OK;
+}
+
+pp_status pp_partition_minsum_batch(int64_t B, int32_t L, const uint64_t *cut_weight, const uint64_t *mem,
+                                    const uint64_t *kappa, int32_t cap_seg, uint64_t *cost, int32_t *m,
+                                    int32_t *cuts, uint64_t *sizes, int8_t *status)
+{
+    if (B < 0 || L < 1 || cap_seg < 0) return PP_ERR_ARG;
+    if (L > PP_MAX_L) return PP_ERR_LIMIT;
+    if (B == 0) return PP_OK;
+    if (!cut_weight || !mem || !kappa || !cost || !m || !status || (!cuts && cap_seg > 0)) return PP_ERR_ARG;
+    const size_t nB = (size_t)B, rows = nB * (size_t)std::max(cap_seg, 1);
+    const size_t sz[8] = {nB * L * 8, nB * L * 8, nB * 8, nB * 8, nB * 4, rows * 4, rows * 8, nB};
+    size_t off[9];
+    off[0] = 0;
+    for (int i = 0; i < 8; ++i) off[i + 1] = align_up(off[i] + sz[i], 256);
+    unsigned char *buf = nullptr;
+    cudaStream_t s = nullptr;
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), off[8], s));
+    const void *src[3] = {cut_weight, mem, kappa};
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i)
+        e = cudaMemcpyAsync(buf + off[i], src[i], sz[i], cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+        e = launch_partition_minsum(B, L, cap_seg, reinterpret_cast<uint64_t *>(buf + off[0]),
+                                    reinterpret_cast<uint64_t *>(buf + off[1]), reinterpret_cast<uint64_t *>(buf + off[2]),
+                                    reinterpret_cast<uint64_t *>(buf + off[3]), reinterpret_cast<int32_t *>(buf + off[4]),
+                                    reinterpret_cast<int32_t *>(buf + off[5]), reinterpret_cast<uint64_t *>(buf + off[6]),
+                                    reinterpret_cast<int8_t *>(buf + off[7]), s);
+    if (e == cudaSuccess) {
+        void *dst[5] = {cost, m, cuts, sizes, status};
+        const size_t n[5] = {sz[3], sz[4], nB * (size_t)cap_seg * 4, nB * (size_t)cap_seg * 8, sz[7]};
+        for (int i = 0; i < 5 && e == cudaSuccess; ++i)
+            if (dst[i] && n[i]) e = cudaMemcpyAsync(dst[i], buf + off[3 + i], n[i], cudaMemcpyDeviceToHost, s);
+    }
+    cudaFreeAsync(buf, s);
+    cudaError_t e2 = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return from_cuda(e);
+    return from_cuda(e2);
+}
+
 pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm)
 {
     if (!warp_instr_per_clk_per_sm || op < 0 || op > 2 || iters < 1 || iters > (1 << 20)) return PP_ERR_ARG;

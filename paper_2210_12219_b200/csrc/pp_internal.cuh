@@ -82,6 +82,11 @@ cudaError_t launch_greedy(int64_t B, int L, int k, const uint64_t *bits, const u
                           const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m, int32_t *cuts,
                           int32_t *place, int8_t *status, cudaStream_t s);
 
+// Partition stage of the paper's heuristic (Algorithm 1), one warp per chain.
+size_t partition_smem_bytes(int L);
+cudaError_t launch_partition_minsum(int64_t B, int L, int cap_seg, const uint64_t *weight, const uint64_t *mem,
+                                    const uint64_t *kappa, uint64_t *cost, int32_t *m, int32_t *cuts,
+                                    uint64_t *sizes, int8_t *status, cudaStream_t s);
 // Issue-rate probe (pp_probe.cu): `blocks` blocks of 1024 threads, cycles[b] = SM clocks block b took.
 cudaError_t launch_probe(int op, int iters, int blocks, long long *cycles, uint32_t *sink, cudaStream_t s);
 double probe_instr_per_block(int iters);
