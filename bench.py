@@ -362,7 +362,8 @@ def run_ours(args):
         other = {}
         for name, inst in (("tiny_k6_L12", W.config_tiny()), ("resnet50_shaped_k10_L50", W.config_resnet50_shaped()),
                            ("deeper_cnn_k14_L100", W.config_deeper_cnn()),
-                           ("large_unequal_layer_memory_k18_L200", W.large_unequal_layers())):
+                           ("large_unequal_layer_memory_k18_L200", W.large_unequal_layers()),
+                           ("geometric_graph_k14_64MB_L50", W.config_geometric(14, 64, 0))):
             with pp.Problem.from_instance(inst) as q:
                 q.set_stream(stream.cuda_stream)
                 if inst.k == k:

@@ -202,6 +202,50 @@ def large_unequal_layers(k: int = 18) -> Instance:
                     np.ascontiguousarray(base.bw_kbps[:k, :k]), "large_unequal_layers")
 
 
+SHANNON_A = 283230.0  # Section 4: chosen so that a device 80 m from the router gets 5.5 Mbps
+
+
+def shannon_mbps(x: float, y: float) -> float:
+    """Eq. 12: rate in Mbps of a device at (x, y) metres from the router at the origin."""
+    return float(np.log2(1.0 + SHANNON_A / (x * x + y * y)))
+
+
+def geometric_bandwidths(k: int, seed: int, link: str = "router") -> tuple[np.ndarray, np.ndarray]:
+    """The random communication graph of the paper's evaluation (Section 4): k devices at positions
+    drawn uniformly from ((-150, -1) u (1, 150))^2 around a WiFi router at the origin, link rates from
+    Shannon's capacity with an SNR that falls with the square of the distance (Eq. 12).
+    link = "router": the rate of a device is that of its own link to the router, and a transfer
+    between two devices passes through the router, so the pair gets the smaller of the two rates.
+    link = "pairwise": Eq. 12 applied to the distance between the two devices (never below 1 m).
+    Returns (bw_kbps uint32 [k, k] symmetric with zero diagonal, positions float64 [k, 2])."""
+    u = stream(6, seed, F_AUX).uniform01(4 * k)
+    mag = 1.0 + 149.0 * u[: 2 * k]
+    sign = np.where(u[2 * k:] < 0.5, -1.0, 1.0)
+    pos = (mag * sign).reshape(k, 2)
+    bw = np.zeros((k, k), dtype=np.uint32)
+    rate = [shannon_mbps(px, py) for px, py in pos]
+    for v in range(k):
+        for w in range(v + 1, k):
+            if link == "router":
+                r = min(rate[v], rate[w])
+            else:
+                dx, dy = pos[v, 0] - pos[w, 0], pos[v, 1] - pos[w, 1]
+                r = float(np.log2(1.0 + SHANNON_A / max(dx * dx + dy * dy, 1.0)))
+            bw[v, w] = bw[w, v] = max(1, int(round(1000.0 * r)))
+    return bw, pos
+
+
+def config_geometric(k: int = 14, cap_mb: int = 64, seed: int = 0, link: str = "router") -> Instance:
+    """The paper's evaluation setting on a synthetic chain: the ResNet50-shaped chain (config 2) on k
+    devices of equal memory (64, 128, 256 or 512 MB in the paper) joined by the random geometric
+    graph of Section 4."""
+    base = config_resnet50_shaped()
+    bw, _ = geometric_bandwidths(k, seed, link)
+    cap = np.full(k, cap_mb * 1_000_000, dtype=np.uint64)
+    return Instance(base.L, k, base.layer_out_bits, base.layer_mem_bytes, cap, bw,
+                    "geometric_k%d_%dMB%s" % (k, cap_mb, "" if link == "router" else "_pairwise"))
+
+
 def random_small(seed: int, L: int, k: int, *, tight: bool = False, dead_links: float = 0.0,
                  ties: bool = False) -> Instance:
     """Small random instance for parity sweeps.  tight=True shrinks capacities so that some

@@ -21,6 +21,7 @@ def main():
     lines = ["# name checksum beta_hex m | cuts | nodes   (written by make_golden.py from oracle.dp_fact)"]
     cases = [W.config_tiny(), W.config_resnet50_shaped(), W.config_deeper_cnn(), W.config_large()]
     cases += W.config_batched(8)
+    cases += [W.config_geometric(14, 64, 0), W.config_geometric(10, 64, 1, link="pairwise")]
     for inst in cases:
         sol = oracle.dp_fact(inst, oracle.max_threads())
         m, cuts, nodes = sol.plan()

@@ -207,6 +207,25 @@ def test_named_configs_2_and_3():
         assert oracle.eval_plan(inst, *got.plan()) == (got.beta_ms, 0)
 
 
+def test_geometric_workload_of_section_4():
+    # the paper's evaluation graph (random positions, Shannon-capacity links, equal node memory), both
+    # readings of how a pair's bandwidth follows from Eq. 12; state rows compared on the k = 14 one
+    for inst in (W.config_geometric(14, 64, 0), W.config_geometric(10, 64, 1, link="pairwise"),
+                 W.config_geometric(12, 128, 2), W.config_geometric(9, 512, 3)):
+        want = oracle.dp_fact(inst, 8)
+        assert_same(inst, gpu_solve(inst), want)
+        assert_same(inst, gpu_solve(inst, generic=True), want)
+    inst = W.config_geometric(14, 64, 0)
+    rng = np.random.default_rng(14)
+    with pp.Problem.from_instance(inst) as p:
+        p.solve_exact()
+        rows = []
+        while len(rows) < 60:
+            S = int(rng.integers(1, 1 << inst.k))
+            rows.append((S, int(rng.choice([v for v in range(inst.k) if S >> v & 1]))))
+        _compare_rows(inst, p, rows)
+
+
 def _sub_instance(inst, nodes):
     idx = np.array(nodes)
     return make_instance(inst.layer_out_bits, inst.layer_mem_bytes, inst.node_mem_bytes[idx],

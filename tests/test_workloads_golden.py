@@ -29,6 +29,7 @@ def named_instances():
     cases = {i.name: i for i in (W.config_tiny(), W.config_resnet50_shaped(), W.config_deeper_cnn(),
                                  W.config_large())}
     cases.update({i.name: i for i in W.config_batched(8)})
+    cases.update({i.name: i for i in (W.config_geometric(14, 64, 0), W.config_geometric(10, 64, 1, link="pairwise"))})
     return cases
 
 
@@ -39,6 +40,27 @@ def test_generators_are_reproducible():
     a, b = W.config_large(), W.config_large()
     assert np.array_equal(a.bw_kbps, b.bw_kbps) and np.array_equal(a.bw_kbps, a.bw_kbps.T)
     assert (np.diag(a.bw_kbps) == 0).all()
+
+
+def test_geometric_workload_follows_section_4():
+    # Eq. 12 with a = 283230 gives 5.5 Mbps at 80 m from the router (the paper's calibration)
+    assert abs(W.shannon_mbps(80.0, 0.0) - 5.5) < 1e-5 and abs(W.shannon_mbps(0.0, -80.0) - 5.499995) < 1e-5
+    assert abs(W.shannon_mbps(48.0, 64.0) - W.shannon_mbps(80.0, 0.0)) < 1e-12  # only the distance counts
+    for seed in range(20):
+        bw, pos = W.geometric_bandwidths(12, seed)
+        assert ((np.abs(pos) > 1.0) & (np.abs(pos) < 150.0)).all()  # no device within 1 m of an axis, none beyond 150 m
+        assert np.array_equal(bw, bw.T) and (np.diag(bw) == 0).all() and (bw[~np.eye(12, dtype=bool)] > 0).all()
+        rate = np.array([W.shannon_mbps(x, y) for x, y in pos])
+        far = int(np.argmin(rate))
+        assert (bw[far][np.arange(12) != far] == int(round(1000 * rate[far]))).all()  # the slower end decides
+        pw, _ = W.geometric_bandwidths(12, seed, link="pairwise")
+        d2 = ((pos[3] - pos[7]) ** 2).sum()
+        assert pw[3, 7] == int(round(1000 * np.log2(1 + 283230.0 / max(d2, 1.0))))
+    g = W.config_geometric(14, 128, 3)
+    assert g.k == 14 and len(set(g.node_mem_bytes.tolist())) == 1 and int(g.node_mem_bytes[0]) == 128_000_000
+    assert np.array_equal(g.layer_out_bits, W.config_resnet50_shaped().layer_out_bits)
+    signs = np.sign(np.concatenate([W.geometric_bandwidths(50, s)[1].ravel() for s in range(4)]))
+    assert 0.35 < (signs < 0).mean() < 0.65  # both half-ranges are used
 
 
 def test_config_shapes_follow_the_recipe():
