@@ -273,6 +273,37 @@ pp_status pp_partition_minsum_batch_dev(int64_t B, int32_t L, const uint64_t *cu
                                         const uint64_t *kappa, int32_t cap_seg, uint64_t *cost, int32_t *m,
                                         int32_t *cuts, uint64_t *sizes, int8_t *status, void *cuda_stream);
 
+/*
+ * Inner step of the paper's placement stage (Section 3.2.2): the threshold classifier of Eq. 8 and
+ * the K-PATH call of Algorithm 2, i.e. the colour-coding search for a simple path of kk vertices in
+ * the subgraph of class-X links, for Q queries on one communication graph.
+ *   n, bw_kbps [n*n]   the communication graph, as for pp_problem_create (row = sender), n <= 64
+ *   kk                 vertices of the path looked for (the paper's k), kk <= 13, same for all queries
+ *   threshold [Q]      Eq. 8: a link is class X, and part of the searched subgraph, when its bandwidth
+ *                      is >= threshold (0 kbps is never a link); Algorithm 2's binary search over the
+ *                      sorted bandwidths is a sequence of such queries
+ *   start, end [Q]     first / last vertex of the path, -1 = any (Algorithm 2's s and u); a walk that
+ *                      reaches `end` before it has kk vertices is not continued
+ *   alive [Q]          bit v set = node v is still available (Algorithm 2 deletes placed nodes)
+ *   colours [Q*n]      colour of every node, below kk (a node with a colour >= kk is not used); the
+ *                      random colouring of the method is the caller's draw, repeated over queries
+ *   found [Q]          out: 1 when a path of kk vertices with kk different colours exists
+ *   path [Q*kk]        out: one such path (any valid one), -1 when none
+ * The paper calls the classifier twice in a row in Algorithm 2 (once with the median edge, once
+ * with `threshold`); here one threshold per query is taken, the median edge's bandwidth.
+ * Host variant: host pointers, synchronous, legacy default stream.  _dev variant: device pointers,
+ * asynchronous on `cuda_stream`.  Q == 0 is a no-op.
+ */
+#define PP_KPATH_MAX_N 64
+#define PP_KPATH_MAX_K 13
+pp_status pp_kpath_colour_batch(int32_t n, const uint32_t *bw_kbps, int64_t Q, int32_t kk, const uint32_t *threshold,
+                                const int32_t *start, const int32_t *end, const uint64_t *alive,
+                                const uint8_t *colours, uint8_t *found, int32_t *path);
+pp_status pp_kpath_colour_batch_dev(int32_t n, const uint32_t *bw_kbps, int64_t Q, int32_t kk,
+                                    const uint32_t *threshold, const int32_t *start, const int32_t *end,
+                                    const uint64_t *alive, const uint8_t *colours, uint8_t *found, int32_t *path,
+                                    void *cuda_stream);
+
 /* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream.
  * ms_total is always measured.  ms_rank, ms_sweep and ms_finalize need events between the
  * phases, which keep one phase's kernels from being launched under the tail of the previous

@@ -29,6 +29,7 @@ EXPORTS = (
     "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev", "pp_debug_minmax_rate",
     "pp_problem_set_profiling", "pp_eval_plans_packed", "pp_eval_plans_packed_dev",
     "pp_partition_minsum_batch", "pp_partition_minsum_batch_dev",
+    "pp_kpath_colour_batch", "pp_kpath_colour_batch_dev",
 )
 
 
@@ -90,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.pp_debug_minmax_rate.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
         L.pp_partition_minsum_batch.argtypes = [i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp]
         L.pp_partition_minsum_batch_dev.argtypes = [i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+        L.pp_kpath_colour_batch.argtypes = [i32, vp, i64, i32] + [vp] * 7
+        L.pp_kpath_colour_batch_dev.argtypes = [i32, vp, i64, i32] + [vp] * 8
         L.pp_status_str.argtypes = [ctypes.c_int]
         L.pp_status_str.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -351,6 +354,26 @@ def partition_minsum_batch_dev(B, L, weight_ptr, mem_ptr, kappa_ptr, cap_seg, co
                                              int(cap_seg), *(ctypes.c_void_p(x) for x in
                                              (cost_ptr, m_ptr, cuts_ptr, sizes_ptr, status_ptr, cuda_stream)))
     _check(st, "pp_partition_minsum_batch_dev")
+
+
+def kpath_colour_batch(bw, kk: int, threshold, start, end, alive, colours):
+    """pp_kpath_colour_batch: bw uint32 [n, n]; per query threshold uint32, start / end int32 (-1 = any),
+    alive uint64 bit masks, colours uint8 [Q, n] -> (found uint8 [Q], path int32 [Q, kk])."""
+    bw, p0 = _host(bw, np.uint32)
+    n = bw.shape[0]
+    threshold, p1 = _host(threshold, np.uint32)
+    Q = threshold.shape[0]
+    start, p2 = _host(start, np.int32)
+    end, p3 = _host(end, np.int32)
+    alive, p4 = _host(alive, np.uint64)
+    colours, p5 = _host(colours, np.uint8)
+    assert colours.size == Q * n and start.size == Q and end.size == Q and alive.size == Q
+    found = np.zeros(Q, dtype=np.uint8)
+    path = np.full((Q, kk), -1, dtype=np.int32)
+    st = lib().pp_kpath_colour_batch(n, p0, Q, int(kk), p1, p2, p3, p4, p5, ctypes.c_void_p(found.ctypes.data),
+                                     ctypes.c_void_p(path.ctypes.data))
+    _check(st, "pp_kpath_colour_batch")
+    return found, path
 
 
 def debug_minmax_rate(op: int, iters: int = 2048) -> float:

@@ -800,6 +800,53 @@ pp_status pp_partition_minsum_batch(int64_t B, int32_t L, const uint64_t *cut_we
     return from_cuda(e2);
 }
 
+pp_status pp_kpath_colour_batch_dev(int32_t n, const uint32_t *bw_kbps, int64_t Q, int32_t kk,
+                                    const uint32_t *threshold, const int32_t *start, const int32_t *end,
+                                    const uint64_t *alive, const uint8_t *colours, uint8_t *found, int32_t *path,
+                                    void *cuda_stream)
+{
+    if (n < 1 || kk < 1 || Q < 0) return PP_ERR_ARG;
+    if (n > PP_KPATH_MAX_N || kk > PP_KPATH_MAX_K) return PP_ERR_LIMIT;
+    if (Q == 0) return PP_OK;
+    if (!bw_kbps || !threshold || !start || !end || !alive || !colours || !found || !path) return PP_ERR_ARG;
+    PP_CUDA(launch_kpath(n, kk, Q, bw_kbps, threshold, start, end, reinterpret_cast<const unsigned long long *>(alive),
+                         colours, found, path, static_cast<cudaStream_t>(cuda_stream)));
+    return PP_OK;
+}
+
+pp_status pp_kpath_colour_batch(int32_t n, const uint32_t *bw_kbps, int64_t Q, int32_t kk, const uint32_t *threshold,
+                                const int32_t *start, const int32_t *end, const uint64_t *alive,
+                                const uint8_t *colours, uint8_t *found, int32_t *path)
+{
+    if (n < 1 || kk < 1 || Q < 0) return PP_ERR_ARG;
+    if (n > PP_KPATH_MAX_N || kk > PP_KPATH_MAX_K) return PP_ERR_LIMIT;
+    if (Q == 0) return PP_OK;
+    if (!bw_kbps || !threshold || !start || !end || !alive || !colours || !found || !path) return PP_ERR_ARG;
+    const size_t nQ = (size_t)Q;
+    const size_t sz[9] = {(size_t)n * n * 4, nQ * 4, nQ * 4, nQ * 4, nQ * 8, nQ * n, nQ, nQ * kk * 4, 0};
+    size_t off[9];
+    off[0] = 0;
+    for (int i = 0; i < 8; ++i) off[i + 1] = align_up(off[i] + sz[i], 256);
+    unsigned char *buf = nullptr;
+    cudaStream_t s = nullptr;
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), off[8], s));
+    const void *src[6] = {bw_kbps, threshold, start, end, alive, colours};
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i < 6 && e == cudaSuccess; ++i)
+        e = cudaMemcpyAsync(buf + off[i], src[i], sz[i], cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess)
+        e = launch_kpath(n, kk, Q, reinterpret_cast<uint32_t *>(buf + off[0]), reinterpret_cast<uint32_t *>(buf + off[1]),
+                         reinterpret_cast<int32_t *>(buf + off[2]), reinterpret_cast<int32_t *>(buf + off[3]),
+                         reinterpret_cast<unsigned long long *>(buf + off[4]), buf + off[5], buf + off[6],
+                         reinterpret_cast<int32_t *>(buf + off[7]), s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(found, buf + off[6], sz[6], cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(path, buf + off[7], sz[7], cudaMemcpyDeviceToHost, s);
+    cudaFreeAsync(buf, s);
+    cudaError_t e2 = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return from_cuda(e);
+    return from_cuda(e2);
+}
+
 pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm)
 {
     if (!warp_instr_per_clk_per_sm || op < 0 || op > 2 || iters < 1 || iters > (1 << 20)) return PP_ERR_ARG;

@@ -87,6 +87,11 @@ size_t partition_smem_bytes(int L);
 cudaError_t launch_partition_minsum(int64_t B, int L, int cap_seg, const uint64_t *weight, const uint64_t *mem,
                                     const uint64_t *kappa, uint64_t *cost, int32_t *m, int32_t *cuts,
                                     uint64_t *sizes, int8_t *status, cudaStream_t s);
+// Colour-coding k-path search of the placement stage (Algorithm 2's K-PATH), one block per query.
+size_t kpath_smem_bytes(int kk);
+cudaError_t launch_kpath(int n, int kk, int64_t Q, const uint32_t *bw, const uint32_t *threshold, const int32_t *start,
+                         const int32_t *end, const unsigned long long *alive, const uint8_t *colours, uint8_t *found,
+                         int32_t *path, cudaStream_t s);
 // Issue-rate probe (pp_probe.cu): `blocks` blocks of 1024 threads, cycles[b] = SM clocks block b took.
 cudaError_t launch_probe(int op, int iters, int blocks, long long *cycles, uint32_t *sink, cudaStream_t s);
 double probe_instr_per_block(int iters);
