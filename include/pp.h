@@ -332,6 +332,12 @@ pp_status pp_debug_mask_order(int32_t k, uint32_t *masks_out, uint32_t *level_of
  * frees a few hundred bytes of device memory. */
 pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm);
 
+/* Test hook: make the nth device allocation the library attempts from now on (1 = the next one)
+ * report "out of memory" without asking the driver; 0 clears a pending request.  Lets a test see
+ * PP_ERR_NOMEM come back from pp_problem_create, pp_solve_exact and the host-pointer entry points on
+ * a device that has memory to spare. */
+pp_status pp_debug_fail_alloc(int32_t nth);
+
 /* Force (1) or forbid (0) the generic sweep kernel; 2 = automatic choice among the kernels that
  * take one source mask per warp (the two-mask kernel is left out); 3 = the two-mask kernel on every
  * level it can run, however small; -1 restores the automatic choice.  Meant for tests that want

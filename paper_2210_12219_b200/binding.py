@@ -29,7 +29,7 @@ EXPORTS = (
     "pp_greedy_batch_dev", "pp_random_plans", "pp_random_plans_dev", "pp_debug_minmax_rate",
     "pp_problem_set_profiling", "pp_eval_plans_packed", "pp_eval_plans_packed_dev",
     "pp_partition_minsum_batch", "pp_partition_minsum_batch_dev",
-    "pp_kpath_colour_batch", "pp_kpath_colour_batch_dev",
+    "pp_kpath_colour_batch", "pp_kpath_colour_batch_dev", "pp_debug_fail_alloc",
 )
 
 
@@ -93,6 +93,7 @@ def lib() -> ctypes.CDLL:
         L.pp_partition_minsum_batch_dev.argtypes = [i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.pp_kpath_colour_batch.argtypes = [i32, vp, i64, i32] + [vp] * 7
         L.pp_kpath_colour_batch_dev.argtypes = [i32, vp, i64, i32] + [vp] * 8
+        L.pp_debug_fail_alloc.argtypes = [i32]
         L.pp_status_str.argtypes = [ctypes.c_int]
         L.pp_status_str.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -374,6 +375,11 @@ def kpath_colour_batch(bw, kk: int, threshold, start, end, alive, colours):
                                      ctypes.c_void_p(path.ctypes.data))
     _check(st, "pp_kpath_colour_batch")
     return found, path
+
+
+def debug_fail_alloc(nth: int):
+    """pp_debug_fail_alloc: the nth device allocation from now on reports out of memory (0 clears)."""
+    _check(lib().pp_debug_fail_alloc(int(nth)), "pp_debug_fail_alloc")
 
 
 def debug_minmax_rate(op: int, iters: int = 2048) -> float:

@@ -1,6 +1,7 @@
 // C-ABI of libpp (see include/pp.h) and the host orchestration behind it: validation,
 // memory prefix sums, window table, mask lists, launch sequence, result download.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
@@ -83,6 +84,16 @@ const MaskList &mask_list(int k)
     return cache.emplace(k, std::move(ml)).first->second;
 }
 
+// Test hook (pp_debug_fail_alloc): the n-th device allocation from now on reports out of memory
+// without asking the driver, so that the out-of-memory paths can be exercised on a healthy device.
+std::atomic<int> g_fail_alloc_countdown{0};
+bool alloc_should_fail()
+{
+    int c = g_fail_alloc_countdown.load();
+    while (c > 0 && !g_fail_alloc_countdown.compare_exchange_weak(c, c - 1)) {}
+    return c == 1;
+}
+
 // Device copy of a mask list, uploaded once per (device, k) and kept for the life of the process:
 // masks [2^k - 1] followed (256-byte aligned) by level_off [k + 2].
 struct DeviceMasks {
@@ -100,7 +111,7 @@ cudaError_t device_masks(int k, const MaskList &ml, DeviceMasks *out)
     if (it == cache.end()) {
         const size_t mb = (ml.masks.size() * 4 + 255) / 256 * 256, lb = ml.level_off.size() * 4;
         unsigned char *buf = nullptr;
-        e = cudaMalloc(reinterpret_cast<void **>(&buf), mb + lb);
+        e = alloc_should_fail() ? cudaErrorMemoryAllocation : cudaMalloc(reinterpret_cast<void **>(&buf), mb + lb);
         if (e != cudaSuccess) return e;
         e = cudaMemcpy(buf, ml.masks.data(), ml.masks.size() * 4, cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemcpy(buf + mb, ml.level_off.data(), lb, cudaMemcpyHostToDevice);
@@ -123,6 +134,7 @@ cudaError_t staging_alloc(void **ptr, size_t bytes, cudaStream_t s)
 {
     static std::mutex mu;
     static cudaMemPool_t pools[64] = {};
+    if (alloc_should_fail()) return cudaErrorMemoryAllocation;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -210,6 +222,8 @@ void bind_work(pp_problem *p)
     p->d.inv = reinterpret_cast<uint32_t *>(b + w.inv);
     p->d.rank = b + w.rank;
     p->d.table = b + w.table;
+    p->d.rank_elems = (uint64_t)p->k * p->k * p->Lpad;
+    p->d.table_elems = ((uint64_t)p->k << p->k) * p->Lpad;
 }
 
 pp_status ensure_work(pp_problem *p)
@@ -217,6 +231,7 @@ pp_status ensure_work(pp_problem *p)
     if (p->d_work) return PP_OK;
     WorkLayout w = work_layout(p->L, p->k, p->Lpad, p->U, p->elem);
     void *ptr = nullptr;
+    if (alloc_should_fail()) return PP_ERR_NOMEM;
     PP_CUDA(cudaMalloc(&ptr, w.total));
     p->d_work = static_cast<unsigned char *>(ptr);
     p->work_bytes = w.total;
@@ -873,6 +888,13 @@ pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per
     const long long med = h[sms / 2];
     if (med <= 0) return PP_ERR_CUDA;
     *warp_instr_per_clk_per_sm = probe_instr_per_block(iters) / (double)med;
+    return PP_OK;
+}
+
+pp_status pp_debug_fail_alloc(int32_t nth)
+{
+    if (nth < 0) return PP_ERR_ARG;
+    g_fail_alloc_countdown.store(nth);
     return PP_OK;
 }
 

@@ -34,6 +34,8 @@ struct Dev {
     uint32_t *inv;             // [U*L+2] inv[r] = some entry e with rk[e] == r (equal ranks hold equal doubles)
     void *rank;                // [k*k*Lpad] rank[(w*k+v)*Lpad + c] of gamma[c][v][w], element type
     void *table;               // [2^k * k * Lpad] state rows, row (S, v) at (S*k+v)*Lpad
+    uint64_t table_elems;      // elements of the state table / of the rank table: what an index
+    uint64_t rank_elems;       //        may reach (checked only in the bounds-checking build)
     unsigned long long *best;  // packed (rank, popcount, mask, v) of the best final state
     int32_t *err;              // device error word (0 = fine, kErrBacktrack)
     const void *fast_meta;     // per-node window constants of the register-tiled sweep, or null
@@ -44,6 +46,18 @@ struct Dev {
 
 static constexpr unsigned long long kNoBest = ~0ull;
 static constexpr int32_t kErrBacktrack = 1;  // the backtrack found no predecessor (inconsistent table)
+static constexpr int32_t kErrBounds = 3;     // bounds-checking build: an index left its table
+
+// Bounds-checking build (-DPP_DEBUG_BOUNDS, libpp_dbg.so): every access to the state table and to
+// the rank table in global memory goes through PP_IN_BOUNDS, which records kErrBounds in the
+// device error word and makes the caller skip the access when the index is outside the table.
+// Nothing traps; the solve then returns PP_ERR_CUDA.  In the normal build the check is `true`.
+#ifdef PP_DEBUG_BOUNDS
+#define PP_IN_BOUNDS(d, index, limit) \
+    ((uint64_t)(index) < (uint64_t)(limit) ? true : (atomicCAS((d).err, 0, kErrBounds), false))
+#else
+#define PP_IN_BOUNDS(d, index, limit) true
+#endif
 
 // final-state key: smaller is better; rank in the high bits, then popcount, mask, node
 __host__ __device__ inline unsigned long long pack_best(uint32_t rank, int popc, uint32_t mask, int v)

@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(128) k_expand_base(Dev d)
         for (int c = threadIdx.x; c < Lpad; c += blockDim.x) {
             T x = kInf;
             if (u >= 0 && c < L) x = (T)(1u + d.cnt[(size_t)u * L + d.pos[c]]);
-            rank[(size_t)r * Lpad + c] = x;
+            if (PP_IN_BOUNDS(d, (size_t)r * Lpad + c, d.rank_elems)) rank[(size_t)r * Lpad + c] = x;
         }
     } else {
         const int v = blockIdx.x - rows;
@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(128) k_expand_base(Dev d)
         const uint64_t cap = d.cap[v];
         for (int c = threadIdx.x; c < Lpad; c += blockDim.x) {
             const T x = (c < L && d.M[c + 1] <= cap) ? (T)0 : kInf;
-            row[c] = x;
+            if (PP_IN_BOUNDS(d, ((size_t)S * k + v) * Lpad + c, d.table_elems)) row[c] = x;
             if (c == L - 1 && x != kInf) atomicMin(d.best, pack_best(0u, 1, S, v));
         }
     }

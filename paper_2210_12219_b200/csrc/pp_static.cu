@@ -168,6 +168,8 @@ extern "C" pp_status pp_solve_exact_static(int32_t L, const uint64_t *layer_out_
     d.inv = reinterpret_cast<uint32_t *>(b + o_inv);
     d.rank = b + o_rank;
     d.table = b + o_table;
+    d.rank_elems = (uint64_t)k * k * Lpad;
+    d.table_elems = ((uint64_t)k << k) * Lpad;
 
     int launches = 0;
     e = launch_rank_base(d, s, &launches);

@@ -47,8 +47,10 @@ __global__ void k_sweep_generic(Dev d, int level)
         T g = kInf;
         for (uint32_t rem = S; rem; rem &= rem - 1) {
             int v = __ffs(rem) - 1;
-            T a = table[((size_t)S * k + v) * Lpad + c];
-            T b = rank[((size_t)w * k + v) * Lpad + c];
+            const size_t ia = ((size_t)S * k + v) * Lpad + c, ib = ((size_t)w * k + v) * Lpad + c;
+            if (!PP_IN_BOUNDS(d, ia, d.table_elems) || !PP_IN_BOUNDS(d, ib, d.rank_elems)) continue;
+            T a = table[ia];
+            T b = rank[ib];
             T m = a > b ? a : b;
             g = m < g ? m : g;
         }
@@ -68,7 +70,8 @@ __global__ void k_sweep_generic(Dev d, int level)
             }
         }
         uint32_t S2 = S | (1u << w);
-        table_w[((size_t)S2 * k + w) * Lpad + c2] = best;
+        const size_t io = ((size_t)S2 * k + w) * Lpad + c2;
+        if (PP_IN_BOUNDS(d, io, d.table_elems)) table_w[io] = best;
         if (c2 == L - 1) offer_best<T>(d, best, S2, w);
     }
 }
@@ -155,7 +158,8 @@ __global__ void __launch_bounds__(1024) k_finalize(Dev d, pp_solution *out)
             for (int c0 = lo; c0 < c2; c0 += 32) {
                 const int c = c0 + lane;
                 bool hit = false;
-                if (c < c2) {
+                if (c < c2 && PP_IN_BOUNDS(d, ((size_t)P * k + v) * Lpad + c, d.table_elems) &&
+                    PP_IN_BOUNDS(d, ((size_t)w * k + v) * Lpad + c, d.rank_elems)) {
                     const T a = trow[c];
                     const T b = rrow[c];
                     const T mx = a > b ? a : b;

@@ -281,7 +281,8 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split, i
         const uint16_t *src = table + (size_t)Sx * k * Lpad + 8 * lane;
 #pragma unroll
         for (int vi = 0; vi < NV; ++vi)
-            dp[vi] = active ? __ldg(reinterpret_cast<const uint4 *>(src + voff[vi]))
+            dp[vi] = active && PP_IN_BOUNDS(d, (size_t)Sx * k * Lpad + 8 * lane + voff[vi], d.table_elems)
+                         ? __ldg(reinterpret_cast<const uint4 *>(src + voff[vi]))
                             : make_uint4(kInf2, kInf2, kInf2, kInf2);
         best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
     };
@@ -357,7 +358,8 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split, i
 #pragma unroll
             for (int t = 0; t < NT; ++t) {
                 const uint32_t S2 = S_cur | (1u << w[t]);
-                if (active)  // row (S2, w) lies ((k << w) + w) rows after row (S_cur, 0)
+                if (active && PP_IN_BOUNDS(d, (size_t)S_cur * k * Lpad + 8 * lane + (size_t)((k << w[t]) + w[t]) * Lpad,
+                                           d.table_elems))  // row (S2, w) lies ((k << w) + w) rows after row (S_cur, 0)
                     *reinterpret_cast<uint4 *>(row_base + (uint32_t)(((k << w[t]) + w[t]) * Lpad)) =
                         make_uint4(o[t][0], o[t][1], o[t][2], o[t][3]);
                 const uint32_t reg = last_reg == 0 ? o[t][0] : (last_reg == 1 ? o[t][1] : (last_reg == 2 ? o[t][2] : o[t][3]));

@@ -207,14 +207,16 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g, int first_le
     auto load_rows1 = [&](uint32_t A) {
         const uint32_t i1 = A * mask_rows + lane;
 #pragma unroll
-        for (int vi = 0; vi < NV; ++vi) dp1[vi] = active ? __ldg(table + (i1 + wo[vi])) : inf4;
+        for (int vi = 0; vi < NV; ++vi)
+            dp1[vi] = active && PP_IN_BOUNDS(d, (uint64_t)(i1 + wo[vi]) * 8, d.table_elems) ? __ldg(table + (i1 + wo[vi])) : inf4;
     };
     auto load_rows2 = [&](uint32_t B) {
         const uint32_t i2 = B * mask_rows + lane;
 #pragma unroll
         for (int vi = 0; vi < NV; ++vi) {
             voff[vi] = wo[vi] * 8;
-            dp2[vi] = active ? __ldg(table + (i2 + wo[vi == NC ? NV : vi])) : inf4;
+            const uint32_t at = i2 + wo[vi == NC ? NV : vi];
+            dp2[vi] = active && PP_IN_BOUNDS(d, (uint64_t)at * 8, d.table_elems) ? __ldg(table + at) : inf4;
         }
         voffb = wo[NV] * 8;
         best_next = *reinterpret_cast<volatile unsigned long long *>(d.best);
@@ -348,12 +350,12 @@ k_sweep_pair(Dev d, int level, const PairMeta *__restrict__ meta_g, int first_le
                 st_if(table_w + (base1 + mb.w),
                       make_uint4(__byte_perm(out[0], out[1], 0x5410), __byte_perm(out[2], out[3], 0x5410),
                                  __byte_perm(out[4], out[5], 0x5410), __byte_perm(out[6], out[7], 0x5410)),
-                      active);
+                      active && PP_IN_BOUNDS(d, (uint64_t)(base1 + mb.w) * 8, d.table_elems));
             if (ok2)
                 st_if(table_w + (base2 + mb.w),
                       make_uint4(__byte_perm(out[0], out[1], 0x7632), __byte_perm(out[2], out[3], 0x7632),
                                  __byte_perm(out[4], out[5], 0x7632), __byte_perm(out[6], out[7], 0x7632)),
-                      active);
+                      active && PP_IN_BOUNDS(d, (uint64_t)(base2 + mb.w) * 8, d.table_elems));
             // final states: ranks at or below the best rank seen so far are rare
             uint32_t x = out[7];
             if (!L8) {

@@ -29,6 +29,12 @@ def test_every_declared_symbol_is_exported(lib):
         assert hasattr(lib, name), name
 
 
+def test_bounds_checking_build_exports_the_same_symbols():
+    dbg = ctypes.CDLL(build.build_debug())
+    for name in binding.EXPORTS:
+        assert hasattr(dbg, name), name
+
+
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(binding.pp_solution) == 8 + 4 + 4 + 4 * 20 + 4 * 20
     assert ctypes.sizeof(binding.pp_profile) == 36
