@@ -55,8 +55,15 @@ struct FastMeta {
 };
 
 constexpr int NT = 1;  // target nodes processed together
-// per-warp strip of the general window step (u16): the levels of the sparse table, then +inf
-__host__ __device__ constexpr int gen_strip_elems(int levels, int Lpad) { return levels * Lpad + 8; }
+// Per-warp strip of the general window step: the levels of the sparse table, then one word of +inf.
+// A level is four planes of 32 words: plane i holds, for every lane, the lane's register i (cut
+// positions 8 lane + 2 i and + 2 i + 1).  Position c of level s is therefore the halfword at
+// gen_strip_byte(s, c): lanes that look up neighbouring positions hit neighbouring banks.
+__host__ __device__ constexpr int gen_strip_elems(int levels, int /*Lpad*/) { return (levels * 128 + 4) * 2; }
+__host__ __device__ constexpr uint32_t gen_strip_byte(int s, int c)
+{
+    return (uint32_t)((((s * 4 + ((c & 7) >> 1)) * 32 + (c >> 3)) << 2) + ((c & 1) << 1));
+}
 constexpr int kTailWords = 128 + 128;           // per-warp suffix strip of the constant-window step: +inf pad, data
 
 // Window minimum of NT rows held as r[t][0..3]; result in o[t][0..3].  tl points at this lane's four
@@ -152,37 +159,43 @@ __device__ __forceinline__ void window_min_general(const uint32_t (&r)[4], const
                                                    int lane, bool active, int nlev, int Lpad, uint32_t (&o)[4])
 {
     uint32_t t[4] = {r[0], r[1], r[2], r[3]};
-    uint16_t *mine = T + 8 * lane;
+    uint32_t *mine = reinterpret_cast<uint32_t *>(T) + lane;  // this lane's word of plane 0, level 0
+    auto park = [&](int s) {
+        if (active) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) mine[(s * 4 + i) * 32] = t[i];
+        }
+    };
     __syncwarp();  // the previous row's readers are done with the strip
-    if (active) *reinterpret_cast<uint4 *>(mine) = make_uint4(t[0], t[1], t[2], t[3]);
+    park(0);
     if (nlev > 1) {  // shift by one position
         const uint32_t below = __shfl_up_sync(0xFFFFFFFFu, t[3], 1);
         const uint32_t y0 = __byte_perm(below, t[0], 0x5432), y1 = __byte_perm(t[0], t[1], 0x5432);
         const uint32_t y2 = __byte_perm(t[1], t[2], 0x5432), y3 = __byte_perm(t[2], t[3], 0x5432);
         t[0] = vmin2(t[0], y0); t[1] = vmin2(t[1], y1); t[2] = vmin2(t[2], y2); t[3] = vmin2(t[3], y3);
-        if (active) *reinterpret_cast<uint4 *>(mine + Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+        park(1);
     }
     if (nlev > 2) {  // by two positions: one register
         const uint32_t below = __shfl_up_sync(0xFFFFFFFFu, t[3], 1);
         const uint32_t a0 = vmin2(t[0], below), a1 = vmin2(t[1], t[0]), a2 = vmin2(t[2], t[1]), a3 = vmin2(t[3], t[2]);
         t[0] = a0; t[1] = a1; t[2] = a2; t[3] = a3;
-        if (active) *reinterpret_cast<uint4 *>(mine + 2 * Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+        park(2);
     }
     if (nlev > 3) {  // by four positions: two registers
         const uint32_t b2 = __shfl_up_sync(0xFFFFFFFFu, t[2], 1), b3 = __shfl_up_sync(0xFFFFFFFFu, t[3], 1);
         const uint32_t a0 = vmin2(t[0], b2), a1 = vmin2(t[1], b3), a2 = vmin2(t[2], t[0]), a3 = vmin2(t[3], t[1]);
         t[0] = a0; t[1] = a1; t[2] = a2; t[3] = a3;
-        if (active) *reinterpret_cast<uint4 *>(mine + 3 * Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+        park(3);
     }
     for (int s = 4; s < nlev; ++s) {  // by 8 * 2^(s-4) positions: whole lanes
         const int dl = 1 << (s - 4);
 #pragma unroll
         for (int j = 0; j < 4; ++j) t[j] = vmin2(t[j], __shfl_up_sync(0xFFFFFFFFu, t[j], dl));
-        if (active) *reinterpret_cast<uint4 *>(mine + s * Lpad) = make_uint4(t[0], t[1], t[2], t[3]);
+        park(s);
     }
     __syncwarp();
     // lanes beyond the row take empty windows
-    const uint32_t none = (uint32_t)(nlev * Lpad * 2) * 0x10001u;
+    const uint32_t none = (uint32_t)(nlev * 128 * 4) * 0x10001u;
     const uint4 ma = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane) : make_uint4(none, none, none, none);
     const uint4 mb = active ? *reinterpret_cast<const uint4 *>(meta_row + 8 * lane + 4) : make_uint4(none, none, none, none);
     const uint32_t mw[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
@@ -241,7 +254,8 @@ k_sweep_fast(Dev d, int level, const FastMeta *__restrict__ meta_g, int split, i
                        (threadIdx.x >> 5) * gen_strip_elems(d.gen_levels, Lpad);
     if (GEN) {
         for (int i = threadIdx.x; i < k * Lpad; i += kFastThreads) gm_s[i] = d.gen_meta[i];
-        if ((threadIdx.x & 31) == 0) strips[d.gen_levels * Lpad] = 0xFFFFu;  // the constant +inf behind the table
+        if ((threadIdx.x & 31) == 0)  // the constant +inf behind the table
+            *reinterpret_cast<uint32_t *>(strips + d.gen_levels * 256) = kInf2;
     }
     __syncthreads();
     if (!first_level) asm volatile("griddepcontrol.wait;" ::: "memory");  // previous level complete and visible
@@ -475,7 +489,7 @@ int gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out)
         for (int c2 = 0; c2 < L; ++c2) maxlen = std::max(maxlen, c2 - (int)lo[w * L + c2]);
     int levels = 1;
     while ((1 << levels) <= maxlen) ++levels;  // floor(log2(maxlen)) + 1
-    const uint32_t inf_off = (uint32_t)(levels * Lpad * 2);
+    const uint32_t inf_off = (uint32_t)(levels * 128 * 4);
     for (int w = 0; w < k; ++w)
         for (int c2 = 0; c2 < Lpad; ++c2) {
             const int a = c2 < L ? lo[w * L + c2] : c2;  // pads: empty window
@@ -484,8 +498,8 @@ int gen_meta_build(int L, int k, int Lpad, const int16_t *lo, uint32_t *out)
             if (len > 0) {
                 int s = 0;
                 while ((2 << s) <= len) ++s;
-                o1 = (uint32_t)((s * Lpad + c2 - 1) * 2);
-                o2 = (uint32_t)((s * Lpad + a + (1 << s) - 1) * 2);
+                o1 = gen_strip_byte(s, c2 - 1);
+                o2 = gen_strip_byte(s, a + (1 << s) - 1);
             }
             out[w * Lpad + c2] = o1 | (o2 << 16);
         }
