@@ -241,6 +241,13 @@ def run_ours(args):
         clk = clocks.summary()
         prof = prob.last_solve_profile()
         launches_per_step = prof.total_launches + 2
+        if args.step_only:  # for a profiler's launch list: the warm-up and the timed steps, nothing else
+            if rank == 0:
+                print("step only: %d steps, %.4f ms per step, %d launches per step"
+                      % (args.steps, max_over_ranks(ms_local) / args.steps, launches_per_step))
+            if dist is not None:
+                dist.destroy_process_group()
+            return
 
         # per-part device times (same launch configuration, measured after the timed region): the
         # whole solve as the timed step runs it, then its phases with events between them (which
@@ -635,6 +642,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    ap.add_argument("--step-only", action="store_true",
+                    help="run the warm-up and the timed steps and exit (for a profiler's launch list)")
     ap.add_argument("--only", choices=["sweep", "unequal", "batch", "greedy", "random"],
                     help="profiler helper: run one part a few times and exit (see run_only)")
     ap.add_argument("--k", type=int, default=16, help="--only sweep/unequal/random: nodes kept of the Large instance")
