@@ -39,7 +39,7 @@ METRIC = "exact-plan DP relaxations/s"
 UNIT = "relaxations/s"
 # DRAM bytes (read + write) per sweep launch of the Large solve from an ncu capture of the sweep
 # kernels as they stand; None whenever those kernels have changed since the counters were taken.
-SWEEP_DRAM_BYTES_PER_LAUNCH = None
+SWEEP_DRAM_BYTES_PER_LAUNCH = 100.40e6
 NOMINAL_HBM_GBS = 8000.0  # the "about 8 TB/s" the roofline is also quoted against
 N_PLANS = 262144
 N_BATCH = 4096
