@@ -304,6 +304,33 @@ pp_status pp_kpath_colour_batch_dev(int32_t n, const uint32_t *bw_kbps, int64_t 
                                     const uint64_t *alive, const uint8_t *colours, uint8_t *found, int32_t *path,
                                     void *cuda_stream);
 
+/*
+ * Placement stage of the paper's two-stage heuristic (Section 3.2.2, Algorithm 2 SUBGRAPH-K-PATH and
+ * Algorithm 3 K-PATH-MATCHING): nodes for the n_cuts + 1 partitions that the partition stage left,
+ * cut j joining node j and node j + 1.  The cut sizes are put into n_classes classes by their rank
+ * among the distinct sizes; classes are served from the highest down, within a class the maximal
+ * runs of consecutive cuts longest first (equal lengths by first cut); a run of l cuts gets a path
+ * of l + 1 unused nodes between its already placed neighbours, at the largest link-bandwidth
+ * threshold (Eq. 8) for which the colour-coding search of pp_kpath_colour_batch finds one: the
+ * bisection of Algorithm 2 over the sorted bandwidths, each probe a batch of `trials` colourings,
+ * the first colouring that finds a path decides.
+ *   n, bw_kbps [n*n]   host: the communication graph (row = sender), n <= 64
+ *   n_cuts, sizes [n_cuts]   host: transfer sizes S of the cuts, in chain order
+ *   n_classes          number of transfer-size (= bandwidth) classes, >= 1
+ *   trials, draws [trials*n]  host: 32-bit random numbers of the caller; node v gets colour
+ *                      floor(draw * k / 2^32) in a search for a path of k vertices
+ *   nodes [n_cuts+1]   host out: N, all different; -1 when the stage fails
+ *   cut_threshold [n_cuts]   host out, may be NULL: the threshold found for the run of each cut
+ * Returns PP_OK; PP_INFEASIBLE when some run finds no path at any threshold (the paper then runs the
+ * stage again with fewer classes: the caller's loop); PP_ERR_LIMIT for n > 64 or a run of more than
+ * 12 cuts.  Where the paper's listings are inconsistent (the classifier called twice, the path length
+ * taken from the list of runs, the end vertex read one past the run) the readings are those of the
+ * description above.  Synchronous; the device work runs on `cuda_stream`.
+ */
+pp_status pp_kpath_matching(int32_t n, const uint32_t *bw_kbps, int32_t n_cuts, const uint64_t *sizes,
+                            int32_t n_classes, int32_t trials, const uint32_t *draws, int32_t *nodes,
+                            uint32_t *cut_threshold, void *cuda_stream);
+
 /* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream.
  * ms_total is always measured.  ms_rank, ms_sweep and ms_finalize need events between the
  * phases, which keep one phase's kernels from being launched under the tail of the previous

@@ -30,6 +30,7 @@ EXPORTS = (
     "pp_problem_set_profiling", "pp_eval_plans_packed", "pp_eval_plans_packed_dev",
     "pp_partition_minsum_batch", "pp_partition_minsum_batch_dev",
     "pp_kpath_colour_batch", "pp_kpath_colour_batch_dev", "pp_debug_fail_alloc",
+    "pp_kpath_matching",
 )
 
 
@@ -94,6 +95,7 @@ def lib() -> ctypes.CDLL:
         L.pp_kpath_colour_batch.argtypes = [i32, vp, i64, i32] + [vp] * 7
         L.pp_kpath_colour_batch_dev.argtypes = [i32, vp, i64, i32] + [vp] * 8
         L.pp_debug_fail_alloc.argtypes = [i32]
+        L.pp_kpath_matching.argtypes = [i32, vp, i32, vp, i32, i32, vp, vp, vp, vp]
         L.pp_status_str.argtypes = [ctypes.c_int]
         L.pp_status_str.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -375,6 +377,23 @@ def kpath_colour_batch(bw, kk: int, threshold, start, end, alive, colours):
                                      ctypes.c_void_p(path.ctypes.data))
     _check(st, "pp_kpath_colour_batch")
     return found, path
+
+
+def kpath_matching(bw, sizes, n_classes: int, draws, cuda_stream: int = 0):
+    """pp_kpath_matching: bw uint32 [n, n], sizes uint64 [n_cuts], draws uint32 [trials, n] ->
+    (status, nodes int32 [n_cuts + 1], cut_threshold uint32 [n_cuts])."""
+    bw, p0 = _host(bw, np.uint32)
+    n = bw.shape[0]
+    sizes, p1 = _host(sizes, np.uint64)
+    draws, p2 = _host(draws, np.uint32)
+    assert draws.ndim == 2 and draws.shape[1] == n
+    nodes = np.full(sizes.size + 1, -1, dtype=np.int32)
+    thr = np.zeros(max(sizes.size, 1), dtype=np.uint32)
+    st = lib().pp_kpath_matching(n, p0, int(sizes.size), p1, int(n_classes), int(draws.shape[0]), p2,
+                                 ctypes.c_void_p(nodes.ctypes.data), ctypes.c_void_p(thr.ctypes.data),
+                                 ctypes.c_void_p(cuda_stream))
+    _check(st, "pp_kpath_matching", ok=(PP_OK, PP_INFEASIBLE))
+    return st, nodes, thr[: sizes.size]
 
 
 def debug_fail_alloc(nth: int):

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
 #include <limits>
 #include <map>
 #include <mutex>
@@ -860,6 +861,134 @@ pp_status pp_kpath_colour_batch(int32_t n, const uint32_t *bw_kbps, int64_t Q, i
     cudaError_t e2 = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return from_cuda(e);
     return from_cuda(e2);
+}
+
+// Placement stage of the paper's heuristic (Section 3.2.2, Algorithms 2 and 3), orchestrated on the
+// host: classes of the cut sizes, runs of cuts per class, and for every run a bisection over the
+// sorted link bandwidths whose probes are batches of colour-coding k-path queries on the device (one
+// query per trial colouring).
+pp_status pp_kpath_matching(int32_t n, const uint32_t *bw_kbps, int32_t n_cuts, const uint64_t *sizes,
+                            int32_t n_classes, int32_t trials, const uint32_t *draws, int32_t *nodes,
+                            uint32_t *cut_threshold, void *cuda_stream)
+{
+    if (n < 1 || n_cuts < 0 || n_classes < 1 || trials < 1) return PP_ERR_ARG;
+    if (!bw_kbps || !draws || !nodes || (!sizes && n_cuts > 0)) return PP_ERR_ARG;
+    if (n > PP_KPATH_MAX_N) return PP_ERR_LIMIT;
+    const int m = n_cuts + 1;
+    for (int j = 0; j < m; ++j) nodes[j] = -1;
+    if (cut_threshold)
+        for (int j = 0; j < n_cuts; ++j) cut_threshold[j] = 0;
+    if (n_cuts == 0) {
+        nodes[0] = 0;
+        return PP_OK;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    try {
+        // classes of the sizes by rank among the distinct values, highest class served first
+        std::vector<uint64_t> distinct(sizes, sizes + n_cuts);
+        std::sort(distinct.begin(), distinct.end());
+        distinct.erase(std::unique(distinct.begin(), distinct.end()), distinct.end());
+        std::vector<int> cls(n_cuts);
+        for (int j = 0; j < n_cuts; ++j) {
+            const size_t rank = std::lower_bound(distinct.begin(), distinct.end(), sizes[j]) - distinct.begin();
+            cls[j] = (int)(rank * (size_t)n_classes / distinct.size());
+        }
+        // link bandwidths in descending order: the thresholds Algorithm 2 bisects over
+        std::vector<uint32_t> edge_list;
+        for (int v = 0; v < n; ++v)
+            for (int w = 0; w < n; ++w)
+                if (v != w && bw_kbps[v * n + w] > 0) edge_list.push_back(bw_kbps[v * n + w]);
+        std::sort(edge_list.begin(), edge_list.end(), std::greater<uint32_t>());
+        // device buffers for one batch of queries (the longest path decides their size)
+        const size_t T = (size_t)trials;
+        const size_t sz[8] = {(size_t)n * n * 4, T * 4, T * 4, T * 4, T * 8, T * n, T, T * PP_KPATH_MAX_K * 4};
+        size_t off[9];
+        off[0] = 0;
+        for (int i = 0; i < 8; ++i) off[i + 1] = align_up(off[i] + sz[i], 256);
+        unsigned char *buf = nullptr;
+        PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), off[8], s));
+        struct Release {
+            unsigned char *b; cudaStream_t st;
+            ~Release() { cudaFreeAsync(b, st); cudaStreamSynchronize(st); }
+        } release{buf, s};
+        PP_CUDA(cudaMemcpyAsync(buf + off[0], bw_kbps, sz[0], cudaMemcpyHostToDevice, s));
+        std::vector<uint32_t> h_thr(T);
+        std::vector<int32_t> h_start(T), h_end(T), h_path(T * PP_KPATH_MAX_K);
+        std::vector<uint64_t> h_alive(T);
+        std::vector<uint8_t> h_col(T * n), h_found(T);
+        uint64_t used = 0;
+        for (int X = n_classes - 1; X >= 0; --X) {
+            // maximal runs of cuts of class X, longest first, equal lengths by first cut
+            std::vector<std::pair<int, int>> runs;  // (first cut, cuts)
+            for (int i = 0; i < n_cuts;) {
+                if (cls[i] != X) { ++i; continue; }
+                int j = i;
+                while (j < n_cuts && cls[j] == X) ++j;
+                runs.emplace_back(i, j - i);
+                i = j;
+            }
+            std::stable_sort(runs.begin(), runs.end(),
+                             [](const std::pair<int, int> &a, const std::pair<int, int> &b) { return a.second > b.second; });
+            for (const auto &run : runs) {
+                const int first = run.first, cuts = run.second, kk = cuts + 1;
+                if (kk > PP_KPATH_MAX_K) return PP_ERR_LIMIT;
+                const int sv = nodes[first], uv = nodes[first + cuts];
+                uint64_t alive = ~used;
+                if (sv >= 0) alive |= 1ull << sv;
+                if (uv >= 0) alive |= 1ull << uv;
+                for (size_t t = 0; t < T; ++t) {
+                    h_start[t] = sv;
+                    h_end[t] = uv;
+                    h_alive[t] = alive;
+                    for (int v = 0; v < n; ++v)
+                        h_col[t * n + v] = (uint8_t)(((uint64_t)draws[t * n + v] * (uint64_t)kk) >> 32);
+                }
+                PP_CUDA(cudaMemcpyAsync(buf + off[2], h_start.data(), sz[2], cudaMemcpyHostToDevice, s));
+                PP_CUDA(cudaMemcpyAsync(buf + off[3], h_end.data(), sz[3], cudaMemcpyHostToDevice, s));
+                PP_CUDA(cudaMemcpyAsync(buf + off[4], h_alive.data(), sz[4], cudaMemcpyHostToDevice, s));
+                PP_CUDA(cudaMemcpyAsync(buf + off[5], h_col.data(), sz[5], cudaMemcpyHostToDevice, s));
+                size_t low = 0, high = edge_list.size();
+                std::vector<int32_t> best_path;
+                uint32_t best_t = 0;
+                while (low < high) {
+                    const size_t median = (low + high) / 2;
+                    std::fill(h_thr.begin(), h_thr.end(), edge_list[median]);
+                    PP_CUDA(cudaMemcpyAsync(buf + off[1], h_thr.data(), sz[1], cudaMemcpyHostToDevice, s));
+                    PP_CUDA(launch_kpath(n, kk, (int64_t)T, reinterpret_cast<uint32_t *>(buf + off[0]),
+                                         reinterpret_cast<uint32_t *>(buf + off[1]), reinterpret_cast<int32_t *>(buf + off[2]),
+                                         reinterpret_cast<int32_t *>(buf + off[3]),
+                                         reinterpret_cast<unsigned long long *>(buf + off[4]), buf + off[5], buf + off[6],
+                                         reinterpret_cast<int32_t *>(buf + off[7]), s));
+                    PP_CUDA(cudaMemcpyAsync(h_found.data(), buf + off[6], T, cudaMemcpyDeviceToHost, s));
+                    PP_CUDA(cudaMemcpyAsync(h_path.data(), buf + off[7], T * kk * 4, cudaMemcpyDeviceToHost, s));
+                    PP_CUDA(cudaStreamSynchronize(s));
+                    size_t hit = T;
+                    for (size_t t = 0; t < T && hit == T; ++t)
+                        if (h_found[t]) hit = t;  // the first colouring that finds a path
+                    if (hit == T) {
+                        low = median + 1;
+                    } else {
+                        high = median;
+                        best_path.assign(h_path.begin() + hit * kk, h_path.begin() + (hit + 1) * kk);
+                        best_t = edge_list[median];
+                    }
+                }
+                if (best_path.empty()) {
+                    for (int j = 0; j < m; ++j) nodes[j] = -1;
+                    return PP_INFEASIBLE;
+                }
+                for (int i = 0; i < kk; ++i) {
+                    nodes[first + i] = best_path[i];
+                    used |= 1ull << best_path[i];
+                }
+                if (cut_threshold)
+                    for (int i = 0; i < cuts; ++i) cut_threshold[first + i] = best_t;
+            }
+        }
+    } catch (const std::bad_alloc &) {
+        return PP_ERR_NOMEM;
+    }
+    return PP_OK;
 }
 
 pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm)
