@@ -383,6 +383,41 @@ def run_ours(args):
                 other[name] = {"solve_ms": min(ts[2:]), "relaxations_per_s": n_relax(inst.k, inst.L) / (min(ts[2:]) * 1e-3),
                                "state_bytes": qp.state_bytes, "fast_path": qp.fast_path, "pair_levels": qp.pair_levels}
 
+        # the paper's own two-stage heuristic (Algorithm 1, then Algorithms 2 and 3) against the exact
+        # optimum on the evaluation setting of its Section 4: 14 devices of 32 MB on a random geometric
+        # graph, the ResNet50-shaped chain; not part of the timed step
+        h_ratios, h_failed = [], 0
+        draws_rng = np.random.default_rng(777)
+        for seed in range(8):
+            gi = W.config_geometric(14, 32, seed, link="pairwise")
+            part = pp.partition_minsum_batch(gi.layer_out_bits[None, :], gi.layer_mem_bytes[None, :],
+                                             gi.node_mem_bytes[:1].copy(), gi.L)
+            gm = int(part.m[0])
+            if part.status[0] != 0 or gm > gi.k:
+                h_failed += 1
+                continue
+            h_draws = draws_rng.integers(0, 2**32, size=(24, gi.k), dtype=np.uint64).astype(np.uint32)
+            st, h_nodes, _ = pp.kpath_matching(gi.bw_kbps, part.sizes[0, :gm - 1], 3, h_draws, stream.cuda_stream)
+            if st != 0:
+                h_failed += 1
+                continue
+            g_ends = np.full((1, gi.k), -1, np.int32)
+            g_nd = np.full((1, gi.k), -1, np.int32)
+            g_ends[0, :gm - 1] = part.cuts[0, :gm - 1]
+            g_nd[0, :gm] = h_nodes
+            with pp.Problem.from_instance(gi) as q:
+                q.set_stream(stream.cuda_stream)
+                hb, hf = q.eval_plans(np.array([gm], np.uint8), g_ends, g_nd)
+                ex = q.solve_exact()
+            if hf[0] == 0 and ex.status == 0 and ex.beta_ms > 0:
+                h_ratios.append(float(hb[0] / ex.beta_ms))
+        heuristic = {"instances": 8, "no_plan": h_failed,
+                     "beta_over_optimum_median": float(np.median(h_ratios)) if h_ratios else None,
+                     "beta_over_optimum_mean": float(np.mean(h_ratios)) if h_ratios else None,
+                     "beta_over_optimum_max": float(np.max(h_ratios)) if h_ratios else None,
+                     "setting": "ResNet50-shaped chain, 14 devices of 32 MB, geometric graph (pairwise Eq. 12), "
+                                "3 classes, 24 colourings per probe"}
+
     sol_rec = pp.pp_solution.from_buffer_copy(d_sol.cpu().numpy().tobytes())
     ms_per_step = ms_total / args.steps
     value, _ = aggregate_over_ranks(relax_step * args.steps, ms_local * 1e-3, dist, dev)
@@ -523,6 +558,7 @@ def run_ours(args):
             "fast_path": prof.fast_path, "beta_ms": sol_rec.beta_ms, "segments": sol_rec.m,
             "greedy_baseline_batched": greedy,
             "random_baseline_large": random_base,
+            "paper_heuristic_geometric": heuristic,
             "other_configs": other,
         },
     }
