@@ -331,6 +331,27 @@ pp_status pp_kpath_matching(int32_t n, const uint32_t *bw_kbps, int32_t n_cuts, 
                             int32_t n_classes, int32_t trials, const uint32_t *draws, int32_t *nodes,
                             uint32_t *cut_threshold, void *cuda_stream);
 
+/*
+ * Exact search under the paper's full objective, Eq. 1: beta = max over the plan's partitions and
+ * cuts of { c_k, gamma_k }, the compute time of every partition counted as well (Eq. 2, which
+ * pp_solve_exact minimises, drops it: the paper argues that transfers dominate on its hardware).
+ *   layer_work  host [L]  computation of each layer in work units (below PP_MAX_BITS)
+ *   node_speed  host [k]  work units per millisecond of each node; 0 = the node cannot compute
+ * c_k = (exact integer sum of the partition's work) / (speed of its node): one IEEE-754 binary64
+ * division, in milliseconds, like gamma.  All other arguments, the constraints, the canonical plan
+ * and the outputs are those of pp_problem_create + pp_solve_exact.  One call does everything
+ * (allocates its tables, runs, frees); synchronous, legacy default stream.  The state table holds
+ * doubles (k * 2^k * L * 8 bytes) and every compute time has its own table entry (k * L * L * 8
+ * bytes): PP_ERR_LIMIT beyond k = 16 or L = 256, PP_ERR_NOMEM when the device cannot hold them.
+ * With layer_work all zero the result is that of pp_solve_exact.
+ */
+#define PP_COMPUTE_MAX_K 16
+#define PP_COMPUTE_MAX_L 256
+pp_status pp_solve_exact_compute(int32_t L, const uint64_t *layer_out_bits, const uint64_t *layer_mem_bytes,
+                                 const uint64_t *layer_work, int32_t k, const uint64_t *node_mem_bytes,
+                                 const uint32_t *bw_kbps, const uint32_t *node_speed, double *beta_ms, int32_t *m,
+                                 int32_t *cuts, int32_t *placement);
+
 /* Device-time breakdown of the last exact solve of `p`; synchronises the problem's stream.
  * ms_total is always measured.  ms_rank, ms_sweep and ms_finalize need events between the
  * phases, which keep one phase's kernels from being launched under the tail of the previous

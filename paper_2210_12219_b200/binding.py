@@ -30,7 +30,7 @@ EXPORTS = (
     "pp_problem_set_profiling", "pp_eval_plans_packed", "pp_eval_plans_packed_dev",
     "pp_partition_minsum_batch", "pp_partition_minsum_batch_dev",
     "pp_kpath_colour_batch", "pp_kpath_colour_batch_dev", "pp_debug_fail_alloc",
-    "pp_kpath_matching",
+    "pp_kpath_matching", "pp_solve_exact_compute",
 )
 
 
@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
         L.pp_kpath_colour_batch_dev.argtypes = [i32, vp, i64, i32] + [vp] * 8
         L.pp_debug_fail_alloc.argtypes = [i32]
         L.pp_kpath_matching.argtypes = [i32, vp, i32, vp, i32, i32, vp, vp, vp, vp]
+        L.pp_solve_exact_compute.argtypes = [i32, vp, vp, vp, i32, vp, vp, vp, ctypes.POINTER(ctypes.c_double),
+                                             ctypes.POINTER(i32), vp, vp]
         L.pp_status_str.argtypes = [ctypes.c_int]
         L.pp_status_str.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -394,6 +396,22 @@ def kpath_matching(bw, sizes, n_classes: int, draws, cuda_stream: int = 0):
                                  ctypes.c_void_p(cuda_stream))
     _check(st, "pp_kpath_matching", ok=(PP_OK, PP_INFEASIBLE))
     return st, nodes, thr[: sizes.size]
+
+
+def solve_exact_compute(inst, layer_work, node_speed) -> Solution:
+    """pp_solve_exact_compute: the exact search under Eq. 1 for a workloads.Instance plus per-layer work
+    (uint64 [L]) and per-node speed (uint32 [k])."""
+    keep = [_host(inst.layer_out_bits, np.uint64), _host(inst.layer_mem_bytes, np.uint64), _host(layer_work, np.uint64),
+            _host(inst.node_mem_bytes, np.uint64), _host(inst.bw_kbps, np.uint32), _host(node_speed, np.uint32)]
+    k = int(inst.k)
+    beta, m = ctypes.c_double(), ctypes.c_int32()
+    cuts = np.full(max(k - 1, 1), -1, dtype=np.int32)
+    placement = np.full(k, -1, dtype=np.int32)
+    st = lib().pp_solve_exact_compute(int(inst.L), keep[0][1], keep[1][1], keep[2][1], k, keep[3][1], keep[4][1],
+                                      keep[5][1], ctypes.byref(beta), ctypes.byref(m),
+                                      ctypes.c_void_p(cuts.ctypes.data), ctypes.c_void_p(placement.ctypes.data))
+    _check(st, "pp_solve_exact_compute", ok=(PP_OK, PP_INFEASIBLE))
+    return Solution(st, beta.value, int(m.value), cuts[: max(k - 1, 0)], placement)
 
 
 def debug_fail_alloc(nth: int):

@@ -991,6 +991,75 @@ pp_status pp_kpath_matching(int32_t n, const uint32_t *bw_kbps, int32_t n_cuts, 
     return PP_OK;
 }
 
+pp_status pp_solve_exact_compute(int32_t L, const uint64_t *layer_out_bits, const uint64_t *layer_mem_bytes,
+                                 const uint64_t *layer_work, int32_t k, const uint64_t *node_mem_bytes,
+                                 const uint32_t *bw_kbps, const uint32_t *node_speed, double *beta_ms, int32_t *m,
+                                 int32_t *cuts, int32_t *placement)
+{
+    if (!beta_ms || !m || !placement || (!cuts && k > 1) || !layer_work || !node_speed) return PP_ERR_ARG;
+    pp_status st = validate(L, layer_out_bits, layer_mem_bytes, k, node_mem_bytes, bw_kbps);
+    if (st != PP_OK) return st;
+    if (L > PP_COMPUTE_MAX_L || k > PP_COMPUTE_MAX_K) return PP_ERR_LIMIT;
+    for (int i = 0; i < L; ++i)
+        if (layer_work[i] >= PP_MAX_BITS) return PP_ERR_LIMIT;
+    try {
+        std::vector<uint64_t> M(L + 1, 0), Wp(L + 1, 0);
+        for (int i = 0; i < L; ++i) {
+            M[i + 1] = M[i] + layer_mem_bytes[i];
+            Wp[i + 1] = Wp[i] + layer_work[i];
+        }
+        DeviceMasks dmasks;
+        PP_CUDA(device_masks(k, mask_list(k), &dmasks));
+        struct Part { const void *src; size_t bytes; size_t off; };
+        std::vector<Part> parts = {
+            {layer_out_bits, (size_t)L * 8, 0}, {M.data(), (size_t)(L + 1) * 8, 0}, {Wp.data(), (size_t)(L + 1) * 8, 0},
+            {node_mem_bytes, (size_t)k * 8, 0}, {bw_kbps, (size_t)k * k * 4, 0}, {node_speed, (size_t)k * 4, 0},
+            {nullptr, 16, 0} /* best value, best key */, {nullptr, sizeof(pp_solution), 0},
+            {nullptr, (size_t)k * k * L * 8, 0} /* gamma */, {nullptr, (size_t)k * L * L * 8, 0} /* compute times */,
+            {nullptr, ((size_t)k << k) * L * 8, 0} /* state table */};
+        size_t total = 0;
+        for (auto &q : parts) { q.off = total; total = align_up(total + q.bytes, 256); }
+        unsigned char *buf = nullptr;
+        if (alloc_should_fail()) return PP_ERR_NOMEM;
+        PP_CUDA(cudaMalloc(reinterpret_cast<void **>(&buf), total));
+        struct Release {
+            unsigned char *b;
+            ~Release() { cudaFree(b); }
+        } release{buf};
+        cudaStream_t s = nullptr;
+        for (int i = 0; i < 6; ++i)
+            PP_CUDA(cudaMemcpyAsync(buf + parts[i].off, parts[i].src, parts[i].bytes, cudaMemcpyHostToDevice, s));
+        CtDev d{};
+        d.L = L; d.k = k;
+        d.bits = reinterpret_cast<uint64_t *>(buf + parts[0].off);
+        d.M = reinterpret_cast<uint64_t *>(buf + parts[1].off);
+        d.Wp = reinterpret_cast<uint64_t *>(buf + parts[2].off);
+        d.cap = reinterpret_cast<uint64_t *>(buf + parts[3].off);
+        d.bw = reinterpret_cast<uint32_t *>(buf + parts[4].off);
+        d.speed = reinterpret_cast<uint32_t *>(buf + parts[5].off);
+        d.masks = dmasks.masks;
+        d.level_off = dmasks.level_off;
+        d.best_val = reinterpret_cast<unsigned long long *>(buf + parts[6].off);
+        d.best_key = d.best_val + 1;
+        pp_solution *d_sol = reinterpret_cast<pp_solution *>(buf + parts[7].off);
+        d.gam = reinterpret_cast<double *>(buf + parts[8].off);
+        d.seg = reinterpret_cast<double *>(buf + parts[9].off);
+        d.table = reinterpret_cast<double *>(buf + parts[10].off);
+        PP_CUDA(launch_compute_search(d, d_sol, s));
+        pp_solution h{};
+        PP_CUDA(cudaMemcpyAsync(&h, d_sol, sizeof h, cudaMemcpyDeviceToHost, s));
+        PP_CUDA(cudaStreamSynchronize(s));
+        if (h.status != PP_OK && h.status != PP_INFEASIBLE) return PP_ERR_CUDA;
+        *beta_ms = h.beta_ms;
+        *m = h.m;
+        for (int j = 0; j < k - 1; ++j) cuts[j] = h.cuts[j];
+        for (int j = 0; j < k; ++j) placement[j] = h.placement[j];
+        return static_cast<pp_status>(h.status);
+    } catch (const std::bad_alloc &) {
+        return PP_ERR_NOMEM;
+    }
+}
+
 pp_status pp_debug_minmax_rate(int32_t op, int32_t iters, double *warp_instr_per_clk_per_sm)
 {
     if (!warp_instr_per_clk_per_sm || op < 0 || op > 2 || iters < 1 || iters > (1 << 20)) return PP_ERR_ARG;

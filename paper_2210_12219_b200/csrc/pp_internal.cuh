@@ -106,6 +106,16 @@ size_t kpath_smem_bytes(int kk);
 cudaError_t launch_kpath(int n, int kk, int64_t Q, const uint32_t *bw, const uint32_t *threshold, const int32_t *start,
                          const int32_t *end, const unsigned long long *alive, const uint8_t *colours, uint8_t *found,
                          int32_t *path, cudaStream_t s);
+// Exact search under Eq. 1 (compute times in the bottleneck), pp_compute.cu.
+struct CtDev {
+    int L, k;
+    const uint64_t *bits, *M, *Wp, *cap;   // [L], [L+1] memory prefix sums, [L+1] work prefix sums, [k]
+    const uint32_t *bw, *speed;            // [k*k], [k]
+    const uint32_t *masks, *level_off;     // node sets by popcount (any order within a level)
+    double *gam, *seg, *table;             // [k*k*L], [k*L*L], [2^k * k * L]
+    unsigned long long *best_val, *best_key;  // adjacent 64-bit words
+};
+cudaError_t launch_compute_search(const CtDev &d, pp_solution *out, cudaStream_t s);
 // Issue-rate probe (pp_probe.cu): `blocks` blocks of 1024 threads, cycles[b] = SM clocks block b took.
 cudaError_t launch_probe(int op, int iters, int blocks, long long *cycles, uint32_t *sink, cudaStream_t s);
 double probe_instr_per_block(int iters);
