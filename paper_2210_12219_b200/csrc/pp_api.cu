@@ -129,6 +129,54 @@ cudaError_t device_masks(int k, const MaskList &ml, DeviceMasks *out)
     return cudaSuccess;
 }
 
+// Row numbering of the instance-per-lane batch path, per (device, k): rows ordered by (popcount,
+// mask, node), the masks listed by (popcount, value).
+struct LaneTables {
+    uint32_t *rowoff = nullptr, *mlist = nullptr, *moff = nullptr;
+};
+cudaError_t lane_tables(int k, LaneTables *out)
+{
+    static std::mutex mu;
+    static std::map<std::pair<int, int>, LaneTables> cache;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = cache.find({dev, k});
+    if (it == cache.end()) {
+        const uint32_t nm = 1u << k;
+        std::vector<uint32_t> host(2 * (size_t)nm + (size_t)k + 2);
+        uint32_t *rowoff = host.data(), *mlist = rowoff + nm, *moff = mlist + nm;
+        uint32_t rows = 0, masks = 0;
+        for (int pc = 0; pc <= k; ++pc) {
+            moff[pc] = masks;
+            for (uint32_t S = 0; S < nm; ++S)
+                if (__builtin_popcount(S) == pc) {
+                    rowoff[S] = rows;
+                    rows += (uint32_t)pc;
+                    mlist[masks++] = S;
+                }
+        }
+        moff[k + 1] = masks;
+        uint32_t *buf = nullptr;
+        e = alloc_should_fail() ? cudaErrorMemoryAllocation
+                                : cudaMalloc(reinterpret_cast<void **>(&buf), host.size() * 4);
+        if (e != cudaSuccess) return e;
+        e = cudaMemcpy(buf, host.data(), host.size() * 4, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            cudaFree(buf);
+            return e;
+        }
+        LaneTables lt;
+        lt.rowoff = buf;
+        lt.mlist = buf + nm;
+        lt.moff = buf + 2 * (size_t)nm;
+        it = cache.emplace(std::make_pair(dev, k), lt).first;
+    }
+    *out = it->second;
+    return cudaSuccess;
+}
+
 // Staging buffers of the host-pointer entry points come from a pool of the library's own that
 // keeps its memory between calls (the default pool would hand it back at every synchronisation).
 cudaError_t staging_alloc(void **ptr, size_t bytes, cudaStream_t s)
@@ -172,6 +220,9 @@ pp_status from_cuda(cudaError_t e)
     } while (0)
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// instances whose tables share the scratch memory of the instance-per-lane batch path at a time
+constexpr int64_t kBatchLanesChunk = 4096;
 
 struct WorkLayout {
     size_t pos, order, gu, cnt, rk, inv, rank, table, total;
@@ -675,8 +726,43 @@ pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64
     PP_CUDA(cudaGetDevice(&dev));
     PP_CUDA(cudaDeviceGetAttribute(&max_sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     if (batch_smem_bytes(L, k) + 1024 > (size_t)max_sm) return PP_ERR_LIMIT;
-    PP_CUDA(launch_batch(B, L, k, out_bits, mem, node_mem, bw, beta_ms, m, cuts, placement, status,
-                         static_cast<cudaStream_t>(cuda_stream)));
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (!batch_lanes_takes(B, L, k)) {
+        PP_CUDA(launch_batch(B, L, k, out_bits, mem, node_mem, bw, beta_ms, m, cuts, placement, status, s));
+        return PP_OK;
+    }
+    // Instance-per-lane path: the tables of a chunk of instances live in scratch memory from the
+    // library's pool, ordered on the caller's stream; chunks follow one another on that stream.
+    LaneTables lt;
+    PP_CUDA(lane_tables(k, &lt));
+    const int64_t chunk = std::min<int64_t>(B, kBatchLanesChunk);
+    const size_t G = (size_t)((chunk + 31) / 32);
+    BatchLanes t;
+    t.LH = batch_lanes_words(L);
+    t.rows = (uint32_t)k << (k - 1);
+    t.rowoff = lt.rowoff;
+    t.mlist = lt.mlist;
+    t.moff = lt.moff;
+    const size_t line = (size_t)t.LH * 32 * sizeof(uint32_t);
+    const size_t b_table = G * t.rows * line, b_rank = G * (size_t)(k * k) * line, b_len = G * (size_t)k * line;
+    const size_t b_key = G * 32 * sizeof(unsigned long long), b_flag = align_up(G * 32, 256);
+    unsigned char *buf = nullptr;
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), b_table + b_rank + b_len + b_key + b_flag, s));
+    t.table = reinterpret_cast<uint32_t *>(buf);
+    t.rank = reinterpret_cast<uint32_t *>(buf + b_table);
+    t.len = reinterpret_cast<uint32_t *>(buf + b_table + b_rank);
+    t.key = reinterpret_cast<unsigned long long *>(buf + b_table + b_rank + b_len);
+    t.flag = reinterpret_cast<int8_t *>(buf + b_table + b_rank + b_len + b_key);
+    cudaError_t e = cudaSuccess;
+    for (int64_t b0 = 0; b0 < B && e == cudaSuccess; b0 += chunk) {
+        const int64_t n = std::min<int64_t>(chunk, B - b0);
+        e = launch_batch_prep(n, L, k, out_bits + b0 * L, mem + b0 * L, node_mem + b0 * k, bw + b0 * k * k, t, s);
+        if (e == cudaSuccess)
+            e = launch_batch_lanes(n, L, k, out_bits + b0 * L, bw + b0 * k * k, t, beta_ms + b0, m + b0,
+                                   cuts ? cuts + b0 * (k - 1) : nullptr, placement + b0 * k, status + b0, s);
+    }
+    cudaFreeAsync(buf, s);
+    PP_CUDA(e);
     return PP_OK;
 }
 

@@ -30,21 +30,10 @@ constexpr int kBatchWarps = kBatchThreads / 32;
 constexpr uint16_t kInf16 = 0xFFFFu;
 
 struct BatchLayout {
-    size_t dp, g, rank, rk, cnt, skey, sval, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, mlist, moff, total;
+    size_t dp, g, rank, rk, cnt, skey, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, mlist, moff, total;
 };
 
-// Sort slots that one list of L quotients takes.  A list is ascending as it is computed, so for
-// L <= 32 it is laid out as a sorted run of the next power of two (padded with +inf keys) and the
-// sorting network starts at twice that size; longer lists are sorted from single keys.
-__host__ __device__ inline int batch_run_slots(int L)
-{
-    if (L > 32) return L;
-    int R = 1;
-    while (R < L) R <<= 1;
-    return R;
-}
-
-__host__ __device__ inline BatchLayout batch_layout(int L, int k)
+__host__ __device__ inline BatchLayout batch_layout(int L, int k, bool prep = false)
 {
     BatchLayout b;
     const size_t rows = (size_t)k << (k - 1);
@@ -59,8 +48,6 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
                                                      // two neighbouring cut positions form one word
     size_t o = 0;
     auto take = [&o](size_t bytes) { size_t at = o; o = (o + bytes + 15) & ~(size_t)15; return at; };
-    size_t npad = 1;
-    while (npad < U * batch_run_slots(L)) npad <<= 1;
     b.M = take((size_t)(L + 1) * sizeof(uint64_t));
     b.cap = take((size_t)k * sizeof(uint64_t));
     b.bits = take((size_t)L * sizeof(uint64_t));
@@ -73,22 +60,20 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k)
     b.rowinfo = take(rows * sizeof(uint32_t));
     b.mlist = take(((size_t)1 << k) * sizeof(uint16_t));
     b.moff = take((size_t)(k + 2) * sizeof(uint32_t));
-    // The sort scratch and the per-entry ranks are dead before the first state is
-    // written: they share the bytes of the state table.
+    // The quotient matrix and the per-entry ranks are dead before the first state is written: they
+    // share the bytes of the state table.
     {
         auto up16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
-        const size_t scratch = up16(npad * sizeof(unsigned long long)) +
-                               up16(npad * sizeof(uint16_t)) + up16(U * L * sizeof(uint16_t)) +
-                               up16(U * L * sizeof(uint32_t));
-        const size_t table = rows * Ls * sizeof(uint16_t);
+        const size_t keys = ((U + 1) * L + 1) * sizeof(unsigned long long);  // a row of +inf and a pad in front
+        const size_t scratch = up16(keys) + up16(U * L * sizeof(uint16_t)) + up16(U * L * sizeof(uint32_t));
+        const size_t table = prep ? 0 : rows * Ls * sizeof(uint16_t);  // the preparing kernel keeps no states
         b.dp = take(table > scratch ? table : scratch);
         size_t q = b.dp;
-        b.skey = q; q += up16(npad * sizeof(unsigned long long));
-        b.sval = q; q += up16(npad * sizeof(uint16_t));
+        b.skey = q; q += up16(keys);
         b.rk = q;   q += up16(U * L * sizeof(uint16_t));
         b.cnt = q;
     }
-    b.g = take(best * Ls * sizeof(uint16_t));
+    b.g = take(prep ? 0 : best * Ls * sizeof(uint16_t));
     b.rank = take((size_t)k * k * Ls * sizeof(uint16_t));
     b.pair_u = take((size_t)k * k * sizeof(int16_t));
     b.pos = take((size_t)L * sizeof(int16_t));
@@ -109,46 +94,6 @@ size_t batch_smem_bytes(int L, int k)
 __device__ __forceinline__ uint32_t info_pack(uint32_t P, int w, uint32_t src0)
 {
     return P | ((uint32_t)w << 12) | (src0 << 16);
-}
-
-// (key, payload) pairs in lexicographic order; payloads are distinct, so the order is total
-__device__ __forceinline__ bool pair_gt(unsigned long long ka, uint32_t va, unsigned long long kb, uint32_t vb)
-{
-    return ka > kb || (ka == kb && va > vb);
-}
-
-// Bitonic steps of the size levels size_lo..size_hi whose stride is at most 32, on the 64-key tile
-// that starts at `base` (a multiple of 64): lane l holds keys base+l and base+l+32 in registers.
-__device__ __forceinline__ void sort_tile(unsigned long long *skey, uint16_t *sval, int base, int lane,
-                                          int size_lo, int size_hi)
-{
-    unsigned long long ka = skey[base + lane], kb = skey[base + lane + 32];
-    uint32_t va = sval[base + lane], vb = sval[base + lane + 32];
-    for (int size = size_lo; size <= size_hi; size <<= 1) {
-        const bool upa = ((base + lane) & size) == 0, upb = ((base + lane + 32) & size) == 0;
-        int stride = size >> 1;
-        if (stride >= 32) {  // the two keys of a lane are partners
-            if (pair_gt(ka, va, kb, vb) == upa) {
-                const unsigned long long tk = ka; ka = kb; kb = tk;
-                const uint32_t tv = va; va = vb; vb = tv;
-            }
-            stride = 16;
-        }
-        for (; stride > 0; stride >>= 1) {
-            const bool lower = (lane & stride) == 0;
-            const unsigned long long oka = __shfl_xor_sync(0xFFFFFFFFu, ka, stride);
-            const uint32_t ova = __shfl_xor_sync(0xFFFFFFFFu, va, stride);
-            const unsigned long long okb = __shfl_xor_sync(0xFFFFFFFFu, kb, stride);
-            const uint32_t ovb = __shfl_xor_sync(0xFFFFFFFFu, vb, stride);
-            // the lower partner keeps the smaller pair when the run ascends
-            if (pair_gt(ka, va, oka, ova) == (lower == upa)) { ka = oka; va = ova; }
-            if (pair_gt(kb, vb, okb, ovb) == (lower == upb)) { kb = okb; vb = ovb; }
-        }
-    }
-    skey[base + lane] = ka;
-    skey[base + lane + 32] = kb;
-    sval[base + lane] = (uint16_t)va;
-    sval[base + lane + 32] = (uint16_t)vb;
 }
 
 // Phase A of one level for the sources masks of NV nodes: g[(P + w, w)][c] = min over v in P of
@@ -207,10 +152,11 @@ __global__ void __launch_bounds__(kBatchThreads, kBatchBlocksPerSm)
 k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
         const uint32_t *__restrict__ g_bw, double *__restrict__ o_beta, int32_t *__restrict__ o_m,
-        int32_t *__restrict__ o_cuts, int32_t *__restrict__ o_place, int8_t *__restrict__ o_status)
+        int32_t *__restrict__ o_cuts, int32_t *__restrict__ o_place, int8_t *__restrict__ o_status,
+        const BatchLanes lanes, const int prep)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    const BatchLayout lay = batch_layout(L, k);
+    const BatchLayout lay = batch_layout(L, k, prep != 0);
     uint64_t *M = reinterpret_cast<uint64_t *>(smem + lay.M);
     uint64_t *cap = reinterpret_cast<uint64_t *>(smem + lay.cap);
     uint64_t *s_bits = reinterpret_cast<uint64_t *>(smem + lay.bits);
@@ -228,8 +174,7 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     uint16_t *rank = reinterpret_cast<uint16_t *>(smem + lay.rank);    // [v][w][c]
     uint16_t *rk = reinterpret_cast<uint16_t *>(smem + lay.rk);        // [U][L]
     uint32_t *cnt = reinterpret_cast<uint32_t *>(smem + lay.cnt);      // [U][L]
-    unsigned long long *skey = reinterpret_cast<unsigned long long *>(smem + lay.skey);  // sort keys
-    uint16_t *sval = reinterpret_cast<uint16_t *>(smem + lay.sval);    // sort payload: entry index
+    unsigned long long *skey = reinterpret_cast<unsigned long long *>(smem + lay.skey);  // quotient matrix
     int16_t *pair_u = reinterpret_cast<int16_t *>(smem + lay.pair_u);
     int16_t *pos = reinterpret_cast<int16_t *>(smem + lay.pos);
     int16_t *lo = reinterpret_cast<int16_t *>(smem + lay.lo);
@@ -359,88 +304,38 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             lo[e] = (int16_t)c;  // the pad of an odd L keeps c2: an empty window
         }
         // ---- 2. quotients and their ranks ----
-        // Rank = 1 + number of quotients strictly below: bitonic sort of the bit patterns (positive
-        // doubles order like unsigned integers) with the entry index as payload, then every run of
-        // equal keys takes the position of its first element.
+        // Rank = 1 + number of quotients strictly below.  The quotients form a matrix whose rows (one
+        // per distinct bandwidth, widest link first) and columns (layers by ascending bits) both
+        // ascend, so the count for one entry is a staircase walk: in every row step left while the
+        // element is not below the entry, add the column reached, go down a row.  A walk takes
+        // exactly U + L steps (row U is a row of +inf that empties the column counter), each one
+        // shared-memory load and a few selects, and needs no barrier.  Positive doubles order like
+        // their bit patterns.
         {
-            // Entry e = u * L + i is bits[order[i]] / ubw[u], ascending in i.  With runs, list u takes
-            // the R slots from u * R, in descending order when u is odd: the network then starts
-            // from bitonic blocks of 2 R keys.  Pads carry the largest key and end up behind the
-            // n real entries; they all compare equal, which a compare-exchange leaves alone.
             const int n = U * L;
-            const int R = batch_run_slots(L);
-            const bool runs = L <= 32;
-            const int rshift = 31 - __clz(R);
-            int npad = 1;
-            while (npad < U * R) npad <<= 1;
-            for (int i = tid; i < npad; i += kBatchThreads) {
-                int u, ii;
-                if (runs) {
-                    u = i >> rshift;
-                    ii = i & (R - 1);
-                    if (u & 1) ii = R - 1 - ii;
-                } else {
-                    u = i / L;
-                    ii = i - u * L;
-                }
-                const bool real = u < U && ii < L;
-                skey[i] = real ? (unsigned long long)__double_as_longlong(
-                                     __ddiv_rn((double)s_sorted[ii], (double)ubw[u]))
-                               : ~0ull;
-                sval[i] = real ? (uint16_t)(u * L + ii) : kInf16;
+            unsigned long long *K = skey;  // K[1 + r * L + i]; K[0] is only read behind the j > 0 test
+            __syncthreads();               // uord is complete
+            for (int e = tid; e < (U + 1) * L; e += kBatchThreads) {
+                const int r = e / L, i = e - r * L;
+                K[1 + e] = r < U ? (unsigned long long)__double_as_longlong(__ddiv_rn(
+                                       (double)s_sorted[i], (double)ubw[uord[U - 1 - r]]))
+                                 : ~0ull;
             }
+            if (tid == 0) K[0] = 0ull;
             __syncthreads();
-            if (npad >= 64) {
-                // Tiles of 64 keys, two per lane, stay in a warp's registers for every run of steps
-                // with stride <= 32 (shuffles, no block barrier); only strides >= 64 go through
-                // shared memory with a barrier each.
-                const int tiles = npad >> 6;
-                for (int t = wid; t < tiles; t += kBatchWarps) sort_tile(skey, sval, t << 6, lane, runs ? 2 * R : 2, 64);
-                __syncthreads();
-                for (int size = 128; size <= npad; size <<= 1) {
-                    for (int stride = size >> 1; stride >= 64; stride >>= 1) {
-                        for (int t = tid; t < (npad >> 1); t += kBatchThreads) {
-                            const int lo_i = 2 * t - (t & (stride - 1));  // index with the stride bit clear
-                            const int hi_i = lo_i + stride;
-                            const bool up = (lo_i & size) == 0;
-                            const unsigned long long a = skey[lo_i], b = skey[hi_i];
-                            const uint16_t va = sval[lo_i], vb = sval[hi_i];
-                            if (pair_gt(a, va, b, vb) == up) {
-                                skey[lo_i] = b;
-                                skey[hi_i] = a;
-                                sval[lo_i] = vb;
-                                sval[hi_i] = va;
-                            }
-                        }
-                        __syncthreads();
-                    }
-                    for (int t = wid; t < tiles; t += kBatchWarps) sort_tile(skey, sval, t << 6, lane, size, size);
-                    __syncthreads();
+            const int steps = U + L;
+            for (int e = tid; e < n; e += kBatchThreads) {
+                const int r0 = e / L, i = e - r0 * L;
+                const unsigned long long x = K[1 + e];
+                int j = L, p = L, acc = 0;  // p = r * L + j: the element left of column j in row r
+#pragma unroll 4
+                for (int st = 0; st < steps; ++st) {
+                    const bool ge = j > 0 && K[p] >= x;
+                    acc += ge ? 0 : j;
+                    p += ge ? -1 : L;
+                    j -= ge ? 1 : 0;
                 }
-            } else {
-                for (int size = 2; size <= npad; size <<= 1)
-                    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-                        for (int t = tid; t < (npad >> 1); t += kBatchThreads) {
-                            const int lo_i = 2 * t - (t & (stride - 1));  // index with the stride bit clear
-                            const int hi_i = lo_i + stride;
-                            const bool up = (lo_i & size) == 0;
-                            const unsigned long long a = skey[lo_i], b = skey[hi_i];
-                            if ((a > b) == up) {
-                                skey[lo_i] = b;
-                                skey[hi_i] = a;
-                                const uint16_t va = sval[lo_i];
-                                sval[lo_i] = sval[hi_i];
-                                sval[hi_i] = va;
-                            }
-                        }
-                        __syncthreads();
-                    }
-            }
-            for (int i = tid; i < n; i += kBatchThreads) {
-                int first = i;  // runs of equal quotients are short except in degenerate inputs
-                const unsigned long long key = skey[i];
-                while (first > 0 && skey[first - 1] == key) --first;
-                rk[sval[i]] = (uint16_t)(1 + first);
+                rk[uord[U - 1 - r0] * L + i] = (uint16_t)(1 + acc);
             }
         }
         __syncthreads();
@@ -450,6 +345,41 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             rank[e] = (u < 0 || c >= L) ? kInf16 : rk[u * L + pos[c]];
         }
         __syncthreads();  // the per-entry ranks share their bytes with the state table
+        if (prep) {
+            // Preparing for the instance-per-lane sweep: this instance's column of the rank table, the
+            // window lengths, the base frontier, the best single-node plan and the limit flag.
+            const int LH = lanes.LH;
+            const size_t g = (size_t)(inst >> 5);
+            const int ln = (int)(inst & 31);
+            const uint32_t *rank32 = reinterpret_cast<const uint32_t *>(rank);
+            uint32_t *rT = lanes.rank + g * (size_t)(k * k * LH) * 32 + ln;
+            for (int e = tid; e < k * k * LH; e += kBatchThreads) {
+                const int r = e / LH, wd = e - r * LH;
+                rT[(size_t)e * 32] = wd < Lh ? rank32[r * Lh + wd] : 0xFFFFFFFFu;
+            }
+            uint32_t *lT = lanes.len + g * (size_t)(k * LH) * 32 + ln;
+            uint32_t *tT = lanes.table + g * (size_t)lanes.rows * LH * 32 + ln;
+            for (int e = tid; e < k * LH; e += kBatchThreads) {
+                const int w = e / LH, wd = e - w * LH;
+                uint32_t len = 0, base = 0xFFFFFFFFu;
+                for (int h = 0; h < 2; ++h) {
+                    const int c = 2 * wd + h;
+                    if (c >= L) continue;
+                    len |= (uint32_t)(c - lo[w * Ls + c]) << (16 * h);
+                    if (M[c + 1] <= cap[w]) base &= ~(0xFFFFu << (16 * h));
+                }
+                lT[(size_t)e * 32] = len;
+                tT[((size_t)rowoff[1u << w] * LH + wd) * 32] = base;
+            }
+            if (tid == 0) {
+                unsigned long long best = kNoBest;
+                for (int v = k - 1; v >= 0; --v)
+                    if (M[L] <= cap[v]) best = pack_best(0u, 1, 1u << v, v);
+                lanes.key[inst] = best;
+                lanes.flag[inst] = (int8_t)s_bad;
+            }
+            continue;
+        }
         // base frontier
         for (int e = tid; e < k * Ls; e += kBatchThreads) {
             const int v = e / Ls, c = e - v * Ls;
@@ -602,12 +532,13 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     }
 }
 
-cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
-                         const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
-                         int32_t *cuts, int32_t *placement, int8_t *status, cudaStream_t s)
+static cudaError_t launch_batch_kernel(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                                       const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
+                                       int32_t *cuts, int32_t *placement, int8_t *status,
+                                       const BatchLanes *lanes, cudaStream_t s)
 {
     if (B <= 0) return cudaSuccess;
-    size_t sm = batch_smem_bytes(L, k);
+    const size_t sm = batch_layout(L, k, lanes != nullptr).total;
     cudaError_t e = cudaFuncSetAttribute(k_batch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 148, per_sm = 1;
@@ -618,9 +549,22 @@ cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const ui
     if (per_sm < 1) per_sm = 1;
     int64_t grid = (int64_t)sms * per_sm;
     if (grid > B) grid = B;
-    k_batch<<<(unsigned)grid, kBatchThreads, sm, s>>>(B, L, k, bits, mem, cap, bw, beta, m, cuts,
-                                                      placement, status);
+    k_batch<<<(unsigned)grid, kBatchThreads, sm, s>>>(B, L, k, bits, mem, cap, bw, beta, m, cuts, placement,
+                                                      status, lanes ? *lanes : BatchLanes{}, lanes ? 1 : 0);
     return cudaGetLastError();
+}
+
+cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                         const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
+                         int32_t *cuts, int32_t *placement, int8_t *status, cudaStream_t s)
+{
+    return launch_batch_kernel(B, L, k, bits, mem, cap, bw, beta, m, cuts, placement, status, nullptr, s);
+}
+
+cudaError_t launch_batch_prep(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                              const uint64_t *cap, const uint32_t *bw, const BatchLanes &t, cudaStream_t s)
+{
+    return launch_batch_kernel(B, L, k, bits, mem, cap, bw, nullptr, nullptr, nullptr, nullptr, nullptr, &t, s);
 }
 
 }  // namespace pp

@@ -88,6 +88,30 @@ size_t batch_smem_bytes(int L, int k);
 cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
                          const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
                          int32_t *cuts, int32_t *placement, int8_t *status, cudaStream_t s);
+// Many-instance search with one instance per lane (pp_batch_lanes.cu): tables of a chunk of
+// instances in global memory, instance-minor, so that the 32 lanes of a warp read 32 neighbouring
+// words.  Group g holds instances 32 g .. 32 g + 31 of the chunk.
+struct BatchLanes {
+    uint32_t *table;          // [group][compact row][LH][32]: states, two cut positions per word
+    uint32_t *rank;           // [group][v * k + w][LH][32]: gamma ranks, same packing
+    uint32_t *len;            // [group][w][LH][32]: window lengths c' - lo_w(c'), same packing
+    unsigned long long *key;  // [group][32]: smallest final state so far (value, popcount, mask, node)
+    int8_t *flag;             // [group][32]: 1 = an input beyond the limits
+    const uint32_t *rowoff;   // [2^k]: compact row of (S, lowest node of S), rows ordered by (popcount, mask, node)
+    const uint32_t *mlist;    // masks by (popcount, value)
+    const uint32_t *moff;     // [k + 2]: first entry of each popcount in mlist
+    uint32_t rows;            // k * 2^(k-1)
+    int LH;                   // words per row in these tables: 4, 8, 12 or 16
+};
+bool batch_lanes_takes(int64_t B, int L, int k);
+int batch_lanes_words(int L);
+// prep: one block per instance ranks gamma and writes the instance's column of the tables
+cudaError_t launch_batch_prep(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                              const uint64_t *cap, const uint32_t *bw, const BatchLanes &t, cudaStream_t s);
+// the levels and the backtrack over a prepared chunk; *launches counts the kernels queued
+cudaError_t launch_batch_lanes(int64_t B, int L, int k, const uint64_t *bits, const uint32_t *bw,
+                               const BatchLanes &t, double *beta, int32_t *m, int32_t *cuts,
+                               int32_t *placement, int8_t *status, cudaStream_t s);
 // Random comparison baseline (Section 4): P plans of problem d from 2 k draws each.
 cudaError_t launch_random_plans(const Dev &d, int64_t P, const uint32_t *draws, uint8_t *nseg, int32_t *ends,
                                 int32_t *nodes, cudaStream_t s);

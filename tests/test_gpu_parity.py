@@ -430,6 +430,31 @@ def test_batched_solve_odd_shapes():
     assert ei.value.status == pp.PP_ERR_LIMIT
 
 
+def test_batched_solve_instance_per_lane_shapes():
+    # from 64 instances on, chains of up to 32 layers on up to 8 nodes are solved 32 instances to a
+    # warp: every row width of that path (4, 8, 12, 16 words), batches that end inside a group of 32,
+    # more nodes than layers, and the degenerate inputs
+    for L, k, n in ((2, 3, 64), (5, 2, 97), (7, 8, 65), (13, 5, 130), (16, 3, 96), (17, 6, 71), (24, 8, 100),
+                    (25, 4, 64), (30, 7, 70), (32, 4, 89)):
+        insts = [W.random_small(61000 + 100 * L + i, L, k, tight=(i % 3 == 1), ties=(i % 3 == 2),
+                                dead_links=0.25 if i % 4 == 3 else 0.0) for i in range(n)]
+        got = pp.solve_exact_batch(L, k, *_stack(insts))
+        for b, inst in enumerate(insts):
+            want = oracle.dp_naive(inst)
+            assert got.status[b] == want.status, (L, k, b)
+            assert got.plan(b) == want.plan(), (L, k, b)
+            assert got.beta_ms[b] == want.beta_ms or np.isinf(want.beta_ms)
+            assert (got.cuts[b, max(want.m - 1, 0):] == -1).all() and (got.placement[b, want.m:] == -1).all()
+    # an instance beyond the limits is flagged on its own, its neighbours are solved
+    insts = [W.random_small(62000 + i, 12, 4) for i in range(80)]
+    bits, mem, cap, bw = _stack(insts)
+    bits[17, 3] = np.uint64(1) << np.uint64(41)
+    got = pp.solve_exact_batch(12, 4, bits, mem, cap, bw)
+    assert got.status[17] == pp.PP_ERR_LIMIT and got.m[17] == 0 and np.isinf(got.beta_ms[17])
+    for b in (16, 18, 79):
+        assert got.plan(b) == oracle.dp_naive(insts[b]).plan()
+
+
 def test_workspace_and_stream_from_torch():
     import torch
     inst = W.config_resnet50_shaped()
