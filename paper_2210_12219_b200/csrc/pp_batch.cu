@@ -1,5 +1,5 @@
 // Many-instance exact search: one thread block per instance, the whole state table in shared
-// memory as 16-bit ranks (the sort scratch and the per-entry ranks of the ranking live in the same bytes
+// memory as 16-bit ranks (the quotient matrix and the per-entry ranks of the ranking live in the same bytes
 // before the table is written).  Same recurrence, final choice and backtrack rule as the
 // single-instance path (see pp_sweep.cu); global memory sees the inputs once and the result
 // record once.
@@ -7,9 +7,8 @@
 // Per instance the block
 //   1. stages the inputs, builds the memory prefix sums and the window table lo[w][c'];
 //   2. rank-compresses gamma (Eq. 3): layers sorted by bits, distinct bandwidths listed, one fp64
-//      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, obtained by
-//      a bitonic sort of all quotients (64-key tiles in registers, the wide strides in shared memory;
-//      chains of up to 32 layers enter as the sorted runs they already are);
+//      division per (distinct bandwidth, layer), rank = 1 + number of quotients below, counted by a
+//      staircase walk over the matrix of quotients, which ascends along rows and columns;
 //   3. sweeps the popcount levels with a flat thread <-> (target row, position) mapping:
 //      phase A forms g[c] = min_v max(dp[S'\{w}][v][c], rank[v][w][c]) for every row of the level,
 //      two neighbouring positions per thread as one packed u16x2 word, thread <-> (source mask,
@@ -33,7 +32,7 @@ struct BatchLayout {
     size_t dp, g, rank, rk, cnt, skey, M, cap, bits, sbits, bw, ubw, uord, pair_u, pos, lo, rowoff, loff, rowinfo, mlist, moff, total;
 };
 
-__host__ __device__ inline BatchLayout batch_layout(int L, int k, bool prep = false)
+__host__ __device__ inline BatchLayout batch_layout(int L, int k)
 {
     BatchLayout b;
     const size_t rows = (size_t)k << (k - 1);
@@ -66,14 +65,14 @@ __host__ __device__ inline BatchLayout batch_layout(int L, int k, bool prep = fa
         auto up16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
         const size_t keys = ((U + 1) * L + 1) * sizeof(unsigned long long);  // a row of +inf and a pad in front
         const size_t scratch = up16(keys) + up16(U * L * sizeof(uint16_t)) + up16(U * L * sizeof(uint32_t));
-        const size_t table = prep ? 0 : rows * Ls * sizeof(uint16_t);  // the preparing kernel keeps no states
+        const size_t table = rows * Ls * sizeof(uint16_t);
         b.dp = take(table > scratch ? table : scratch);
         size_t q = b.dp;
         b.skey = q; q += up16(keys);
         b.rk = q;   q += up16(U * L * sizeof(uint16_t));
         b.cnt = q;
     }
-    b.g = take(prep ? 0 : best * Ls * sizeof(uint16_t));
+    b.g = take(best * Ls * sizeof(uint16_t));
     b.rank = take((size_t)k * k * Ls * sizeof(uint16_t));
     b.pair_u = take((size_t)k * k * sizeof(int16_t));
     b.pos = take((size_t)L * sizeof(int16_t));
@@ -152,11 +151,10 @@ __global__ void __launch_bounds__(kBatchThreads, kBatchBlocksPerSm)
 k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
         const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
         const uint32_t *__restrict__ g_bw, double *__restrict__ o_beta, int32_t *__restrict__ o_m,
-        int32_t *__restrict__ o_cuts, int32_t *__restrict__ o_place, int8_t *__restrict__ o_status,
-        const BatchLanes lanes, const int prep)
+        int32_t *__restrict__ o_cuts, int32_t *__restrict__ o_place, int8_t *__restrict__ o_status)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    const BatchLayout lay = batch_layout(L, k, prep != 0);
+    const BatchLayout lay = batch_layout(L, k);
     uint64_t *M = reinterpret_cast<uint64_t *>(smem + lay.M);
     uint64_t *cap = reinterpret_cast<uint64_t *>(smem + lay.cap);
     uint64_t *s_bits = reinterpret_cast<uint64_t *>(smem + lay.bits);
@@ -345,41 +343,6 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
             rank[e] = (u < 0 || c >= L) ? kInf16 : rk[u * L + pos[c]];
         }
         __syncthreads();  // the per-entry ranks share their bytes with the state table
-        if (prep) {
-            // Preparing for the instance-per-lane sweep: this instance's column of the rank table, the
-            // window lengths, the base frontier, the best single-node plan and the limit flag.
-            const int LH = lanes.LH;
-            const size_t g = (size_t)(inst >> 5);
-            const int ln = (int)(inst & 31);
-            const uint32_t *rank32 = reinterpret_cast<const uint32_t *>(rank);
-            uint32_t *rT = lanes.rank + g * (size_t)(k * k * LH) * 32 + ln;
-            for (int e = tid; e < k * k * LH; e += kBatchThreads) {
-                const int r = e / LH, wd = e - r * LH;
-                rT[(size_t)e * 32] = wd < Lh ? rank32[r * Lh + wd] : 0xFFFFFFFFu;
-            }
-            uint32_t *lT = lanes.len + g * (size_t)(k * LH) * 32 + ln;
-            uint32_t *tT = lanes.table + g * (size_t)lanes.rows * LH * 32 + ln;
-            for (int e = tid; e < k * LH; e += kBatchThreads) {
-                const int w = e / LH, wd = e - w * LH;
-                uint32_t len = 0, base = 0xFFFFFFFFu;
-                for (int h = 0; h < 2; ++h) {
-                    const int c = 2 * wd + h;
-                    if (c >= L) continue;
-                    len |= (uint32_t)(c - lo[w * Ls + c]) << (16 * h);
-                    if (M[c + 1] <= cap[w]) base &= ~(0xFFFFu << (16 * h));
-                }
-                lT[(size_t)e * 32] = len;
-                tT[((size_t)rowoff[1u << w] * LH + wd) * 32] = base;
-            }
-            if (tid == 0) {
-                unsigned long long best = kNoBest;
-                for (int v = k - 1; v >= 0; --v)
-                    if (M[L] <= cap[v]) best = pack_best(0u, 1, 1u << v, v);
-                lanes.key[inst] = best;
-                lanes.flag[inst] = (int8_t)s_bad;
-            }
-            continue;
-        }
         // base frontier
         for (int e = tid; e < k * Ls; e += kBatchThreads) {
             const int v = e / Ls, c = e - v * Ls;
@@ -532,13 +495,12 @@ k_batch(int64_t B, int L, int k, const uint64_t *__restrict__ g_bits,
     }
 }
 
-static cudaError_t launch_batch_kernel(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
-                                       const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
-                                       int32_t *cuts, int32_t *placement, int8_t *status,
-                                       const BatchLanes *lanes, cudaStream_t s)
+cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                         const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
+                         int32_t *cuts, int32_t *placement, int8_t *status, cudaStream_t s)
 {
     if (B <= 0) return cudaSuccess;
-    const size_t sm = batch_layout(L, k, lanes != nullptr).total;
+    size_t sm = batch_smem_bytes(L, k);
     cudaError_t e = cudaFuncSetAttribute(k_batch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
     int dev = 0, sms = 148, per_sm = 1;
@@ -549,22 +511,9 @@ static cudaError_t launch_batch_kernel(int64_t B, int L, int k, const uint64_t *
     if (per_sm < 1) per_sm = 1;
     int64_t grid = (int64_t)sms * per_sm;
     if (grid > B) grid = B;
-    k_batch<<<(unsigned)grid, kBatchThreads, sm, s>>>(B, L, k, bits, mem, cap, bw, beta, m, cuts, placement,
-                                                      status, lanes ? *lanes : BatchLanes{}, lanes ? 1 : 0);
+    k_batch<<<(unsigned)grid, kBatchThreads, sm, s>>>(B, L, k, bits, mem, cap, bw, beta, m, cuts,
+                                                      placement, status);
     return cudaGetLastError();
-}
-
-cudaError_t launch_batch(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
-                         const uint64_t *cap, const uint32_t *bw, double *beta, int32_t *m,
-                         int32_t *cuts, int32_t *placement, int8_t *status, cudaStream_t s)
-{
-    return launch_batch_kernel(B, L, k, bits, mem, cap, bw, beta, m, cuts, placement, status, nullptr, s);
-}
-
-cudaError_t launch_batch_prep(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
-                              const uint64_t *cap, const uint32_t *bw, const BatchLanes &t, cudaStream_t s)
-{
-    return launch_batch_kernel(B, L, k, bits, mem, cap, bw, nullptr, nullptr, nullptr, nullptr, nullptr, &t, s);
 }
 
 }  // namespace pp

@@ -8,9 +8,9 @@
 // few thousand instances), instance-minor: the 32 lanes of a warp read 32 neighbouring words.
 //
 // Per chunk of instances:
-//   1. k_batch in its preparing mode (pp_batch.cu), one block per instance: staging, windows, the
-//      ranking of gamma (Eq. 3); writes the instance's column of the rank table, the window lengths,
-//      the base frontier and the best single-node plan;
+//   1. k_lanes_prep, one warp per instance: staging, windows, the ranking of gamma (Eq. 3); writes
+//      the instance's column of the rank table, the window lengths, the base frontier and the best
+//      single-node plan;
 //   2. one launch per popcount level, k_lanes_level<NV, LH>: a warp takes (group of 32 instances,
 //      source mask P of NV nodes), keeps the NV rows of P in registers (two cut positions per 32-bit
 //      word, LH words per row), and for every node w outside P forms
@@ -28,12 +28,241 @@ namespace pp {
 namespace {
 
 constexpr int kLevelWarps = 4;
+constexpr int kPrepWarps = 4;
 constexpr int kBackWarps = 8;
 constexpr int kLanesMinB = 64;  // below this the block-per-instance kernel keeps more of the GPU busy
 constexpr int kLanesMaxK = 8;   // NV <= 7 rows of a source mask in registers
 constexpr int kLanesMaxL = 32;  // LH <= 16 words per row
 constexpr uint32_t kMagic = 0x4B000000u;     // bit pattern of 2^23: kMagic | r is the float 2^23 + r for r < 2^23
 constexpr uint32_t kMagicInf = 0x4B00FFFFu;  // the rank of +inf in that form; also caps a masked candidate
+
+// Shared memory of one warp of the preparing kernel (byte offsets; every part 16-byte aligned).
+struct PrepLayout {
+    size_t K, M, bits, sorted, cap, bw, ubw, rk, pair_u, rowu, pos, total;
+    int Ks;  // row stride of the quotient matrix in keys: a sentinel in front of the L quotients
+};
+
+__host__ __device__ inline PrepLayout prep_layout(int L, int k)
+{
+    PrepLayout p;
+    const size_t U = (size_t)k * (k - 1);
+    size_t o = 0;
+    auto take = [&o](size_t bytes) { size_t at = o; o = (o + bytes + 15) & ~(size_t)15; return at; };
+    p.Ks = L + 1;
+    p.K = take((U + 1) * (size_t)p.Ks * 8);
+    p.M = take(33 * 8);
+    p.bits = take(32 * 8);
+    p.sorted = take(32 * 8);
+    p.cap = take(8 * 8);
+    p.bw = take(64 * 4);
+    p.ubw = take(64 * 4);
+    p.rk = take((U * L + 1) * 2);
+    p.pair_u = take(64);
+    p.rowu = take(64);
+    p.pos = take(32);
+    p.total = o;
+    return p;
+}
+
+// One warp per instance, lane <-> layer (L <= 32) or node pair (k * k <= 64, two per lane): staging,
+// the windows, the ranking of gamma (Eq. 3), and the instance's column of the tables of BatchLanes.
+//   * layers ordered by bits (ties by index), distinct usable bandwidths listed in order of first
+//     appearance, as in the block-per-instance kernel;
+//   * window start lo_w(c2) by a branch-free binary search over the memory prefix sums;
+//   * rank = 1 + number of quotients strictly below.  The quotients form a matrix whose rows (one
+//     per distinct bandwidth, widest link first) and columns (layers by ascending bits) both ascend,
+//     so the count for one entry is a staircase walk: in every row step left while the element is
+//     not below the entry, add the column reached, go down a row.  Keys are the bit patterns of the
+//     quotients (positive doubles order like them) plus one, so that a zero in front of every row
+//     stops the walk to the left without a test; row U holds the largest key and empties the column
+//     counter; a walk takes exactly U + L steps.  Two walks per lane run interleaved.
+__global__ void __launch_bounds__(kPrepWarps * 32)
+k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, const uint64_t *__restrict__ g_bits,
+             const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
+             const uint32_t *__restrict__ g_bw)
+{
+    extern __shared__ __align__(16) unsigned char smem_prep[];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const PrepLayout lay = prep_layout(L, k);
+    unsigned char *base = smem_prep + (size_t)wid * lay.total;
+    unsigned long long *K = reinterpret_cast<unsigned long long *>(base + lay.K);
+    unsigned long long *M = reinterpret_cast<unsigned long long *>(base + lay.M);
+    unsigned long long *s_bits = reinterpret_cast<unsigned long long *>(base + lay.bits);
+    unsigned long long *s_sorted = reinterpret_cast<unsigned long long *>(base + lay.sorted);
+    unsigned long long *s_cap = reinterpret_cast<unsigned long long *>(base + lay.cap);
+    uint32_t *s_bw = reinterpret_cast<uint32_t *>(base + lay.bw);
+    uint32_t *ubw = reinterpret_cast<uint32_t *>(base + lay.ubw);
+    uint16_t *rk = reinterpret_cast<uint16_t *>(base + lay.rk);
+    int8_t *pair_u = reinterpret_cast<int8_t *>(base + lay.pair_u);
+    uint8_t *rowu = base + lay.rowu;
+    uint8_t *pos = base + lay.pos;
+    const int Ks = lay.Ks, LH = t.LH, kk = k * k;
+    const uint32_t FULL = 0xFFFFFFFFu;
+    // floor(x / k) for x < 64 and floor(x / L) for x < k (k-1) L <= 1792 by a multiplication
+    const uint32_t recip_k = (65536u + (uint32_t)k - 1u) / (uint32_t)k;
+    const uint32_t recip_L = (65536u + (uint32_t)L - 1u) / (uint32_t)L;
+    for (int64_t inst = (int64_t)blockIdx.x * kPrepWarps + wid; inst < B; inst += (int64_t)gridDim.x * kPrepWarps) {
+        __syncwarp();
+        // ---- staging, prefix sums of the memory ----
+        const unsigned long long b = lane < L ? g_bits[inst * L + lane] : 0ull;
+        const unsigned long long mm = lane < L ? g_mem[inst * L + lane] : 0ull;
+        const uint32_t bw0 = lane < kk ? g_bw[inst * kk + lane] : 0u;
+        const uint32_t bw1 = lane + 32 < kk ? g_bw[inst * kk + lane + 32] : 0u;
+        bool bad = b >= PP_MAX_BITS || bw0 >= PP_MAX_KBPS || bw1 >= PP_MAX_KBPS;
+        unsigned long long x = mm;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long y = __shfl_up_sync(FULL, x, o);
+            if (lane >= o) {
+                if (y > ~0ull - x) bad = true;  // the 64-bit sum would wrap: PP_ERR_LIMIT
+                x += y;
+            }
+        }
+        if (lane == 0) M[0] = 0ull;
+        M[lane + 1] = x;  // beyond L: the total, never read
+        s_bits[lane] = b;
+        s_bw[lane] = bw0;
+        s_bw[lane + 32] = bw1;
+        if (lane < k) s_cap[lane] = g_cap[inst * k + lane];
+        bad = __any_sync(FULL, bad);
+        __syncwarp();
+        // ---- layers in ascending order of bits (ties by index) ----
+        {
+            int p = 0;
+            for (int o = 0; o < L; ++o) {
+                const unsigned long long xo = s_bits[o];
+                p += (xo < b) || (xo == b && o < lane);
+            }
+            if (lane < L) {
+                s_sorted[p] = b;
+                pos[lane] = (uint8_t)p;
+            }
+        }
+        // ---- distinct usable bandwidths in order of first appearance ----
+        int U;
+        {
+            const int p0 = lane, p1 = lane + 32;
+            const int v0 = (int)(((uint32_t)p0 * recip_k) >> 16), v1 = (int)(((uint32_t)p1 * recip_k) >> 16);
+            const bool us0 = p0 < kk && v0 != p0 - v0 * k && bw0 != 0u;
+            const bool us1 = p1 < kk && v1 != p1 - v1 * k && bw1 != 0u;
+            int f0 = us0 ? p0 : -1, f1 = us1 ? p1 : -1;
+            int v2 = 0, w2 = 0;
+            for (int p2 = 0; p2 < kk; ++p2) {  // ascending: the first match stays
+                const uint32_t b2 = s_bw[p2];
+                const bool us2 = v2 != w2 && b2 != 0u;
+                if (us2 && us0 && b2 == bw0 && p2 < f0) f0 = p2;
+                if (us2 && us1 && b2 == bw1 && p2 < f1) f1 = p2;
+                if (++w2 == k) { w2 = 0; ++v2; }
+            }
+            const bool first0 = us0 && f0 == p0, first1 = us1 && f1 == p1;
+            const uint32_t m0 = __ballot_sync(FULL, first0), m1 = __ballot_sync(FULL, first1);
+            const int n0 = __popc(m0);
+            U = n0 + __popc(m1);
+            auto index_of = [&](int f) {
+                return f < 32 ? __popc(m0 & ((1u << f) - 1u)) : n0 + __popc(m1 & ((1u << (f - 32)) - 1u));
+            };
+            const int u0 = f0 >= 0 ? index_of(f0) : -1, u1 = f1 >= 0 ? index_of(f1) : -1;
+            pair_u[p0] = (int8_t)u0;
+            pair_u[p1] = (int8_t)u1;
+            if (first0) ubw[u0] = bw0;
+            if (first1) ubw[u1] = bw1;
+        }
+        __syncwarp();
+        // rows of the quotient matrix: widest link first (the values of a column then ascend)
+        for (int u = lane; u < U; u += 32) {
+            const uint32_t mine = ubw[u];
+            int r = 0;
+            for (int u2 = 0; u2 < U; ++u2) r += ubw[u2] > mine;
+            rowu[r] = (uint8_t)u;
+        }
+        // ---- windows, base frontier ----
+        {
+            uint32_t *lT = t.len + (size_t)(inst >> 5) * (size_t)(k * LH) * 32 + (inst & 31);
+            uint32_t *tT = t.table + (size_t)(inst >> 5) * (size_t)t.rows * LH * 32 + (inst & 31);
+            const unsigned long long Mc = M[lane + 1];  // memory of layers 0..lane
+            for (int w = 0; w < k; ++w) {
+                const unsigned long long capw = s_cap[w];
+                // c* = number of prefix sums M[0..lane+1] below M[lane+1] - cap: the first start layer
+                // from which the segment ending at this layer fits; window start = max(c* - 1, 0)
+                const unsigned long long thr = Mc > capw ? Mc - capw : 0ull;
+                int cs = 0;
+#pragma unroll
+                for (int step = 32; step; step >>= 1)
+                    if (cs + step <= lane + 2 && M[cs + step - 1] < thr) cs += step;
+                const int lo = cs > 0 ? cs - 1 : 0;
+                const uint32_t len = lane < L ? (uint32_t)(lane - lo) : 0u;
+                const uint32_t inf = (lane < L && Mc <= capw) ? 0u : 0xFFFFu;
+                const uint32_t len0 = __shfl_sync(FULL, len, 2 * lane), len1 = __shfl_sync(FULL, len, 2 * lane + 1);
+                const uint32_t inf0 = __shfl_sync(FULL, inf, 2 * lane), inf1 = __shfl_sync(FULL, inf, 2 * lane + 1);
+                if (lane < LH) {
+                    lT[(size_t)(w * LH + lane) * 32] = lane < 16 ? len0 | (len1 << 16) : 0u;
+                    tT[((size_t)t.rowoff[1u << w] * LH + lane) * 32] = lane < 16 ? inf0 | (inf1 << 16) : 0xFFFFFFFFu;
+                }
+            }
+            if (lane == 0) {
+                unsigned long long best = kNoBest;
+                for (int v = k - 1; v >= 0; --v)
+                    if (M[L] <= s_cap[v]) best = pack_best(0u, 1, 1u << v, v);
+                t.key[inst] = best;
+                t.flag[inst] = (int8_t)bad;
+            }
+        }
+        __syncwarp();
+        // ---- quotient matrix ----
+        for (int r = 0; r <= U; ++r) {
+            unsigned long long key = ~0ull;
+            if (r < U)
+                key = 1ull + (unsigned long long)__double_as_longlong(
+                                 __ddiv_rn((double)s_sorted[lane < L ? lane : 0], (double)ubw[rowu[r]]));
+            if (lane < L) K[r * Ks + 1 + lane] = key;
+            if (lane == 0) K[r * Ks] = 0ull;
+        }
+        __syncwarp();
+        // ---- ranks ----
+        {
+            const int n = U * L, steps = U + L;
+            for (int e0 = 0; e0 < n; e0 += 64) {
+                const int eA = e0 + lane, eB = e0 + 32 + lane;
+                const int rA = (int)(((uint32_t)eA * recip_L) >> 16), rB = (int)(((uint32_t)eB * recip_L) >> 16);
+                const int iA = eA - rA * L, iB = eB - rB * L;
+                // an idle lane walks with the smallest key: left along row 0, then down the zeros
+                const unsigned long long xA = eA < n ? K[rA * Ks + 1 + iA] : 1ull;
+                const unsigned long long xB = eB < n ? K[rB * Ks + 1 + iB] : 1ull;
+                int jA = L, jB = L, accA = 0, accB = 0;
+                const unsigned long long *pA = K + L, *pB = K + L;  // the last quotient of row 0
+#pragma unroll 2
+                for (int st = 0; st < steps; ++st) {
+                    const bool geA = *pA >= xA, geB = *pB >= xB;
+                    accA += geA ? 0 : jA;
+                    accB += geB ? 0 : jB;
+                    pA += geA ? -1 : Ks;
+                    pB += geB ? -1 : Ks;
+                    jA -= geA ? 1 : 0;
+                    jB -= geB ? 1 : 0;
+                }
+                if (eA < n) rk[rowu[rA] * L + iA] = (uint16_t)(1 + accA);
+                if (eB < n) rk[rowu[rB] * L + iB] = (uint16_t)(1 + accB);
+            }
+        }
+        __syncwarp();
+        // ---- rank table, two positions per word: rank[v][w][c] = rank of (bandwidth of v -> w, layer c) ----
+        {
+            uint32_t *rT = t.rank + (size_t)(inst >> 5) * (size_t)(kk * LH) * 32 + (inst & 31);
+            const int c0 = 2 * lane, c1 = 2 * lane + 1;
+            const int q0 = c0 < L ? pos[c0] : 0, q1 = c1 < L ? pos[c1] : 0;
+            for (int pr = 0; pr < kk; ++pr) {
+                const int u = pair_u[pr];
+                uint32_t word = 0xFFFFFFFFu;
+                if (u >= 0) {
+                    const uint32_t a = c0 < L ? rk[u * L + q0] : 0xFFFFu;
+                    const uint32_t c = c1 < L ? rk[u * L + q1] : 0xFFFFu;
+                    word = a | (c << 16);
+                }
+                if (lane < LH) rT[(size_t)(pr * LH + lane) * 32] = word;
+            }
+        }
+    }
+}
 
 template <int NV, int LH>
 __global__ void __launch_bounds__(kLevelWarps * 32)
@@ -284,6 +513,22 @@ int batch_lanes_words(int L)
 {
     const int Lh = (L + 1) / 2;
     return Lh <= 4 ? 4 : Lh <= 8 ? 8 : Lh <= 12 ? 12 : 16;
+}
+
+cudaError_t launch_batch_prep(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
+                              const uint64_t *cap, const uint32_t *bw, const BatchLanes &t, cudaStream_t s)
+{
+    if (B <= 0) return cudaSuccess;
+    const size_t sm = prep_layout(L, k).total * kPrepWarps;
+    cudaError_t e = cudaFuncSetAttribute(k_lanes_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int64_t blocks = (B + kPrepWarps - 1) / kPrepWarps;
+    if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
+    k_lanes_prep<<<(unsigned)blocks, kPrepWarps * 32, sm, s>>>(t, B, L, k, bits, mem, cap, bw);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_batch_lanes(int64_t B, int L, int k, const uint64_t *bits, const uint32_t *bw,

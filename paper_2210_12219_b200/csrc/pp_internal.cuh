@@ -105,7 +105,7 @@ struct BatchLanes {
 };
 bool batch_lanes_takes(int64_t B, int L, int k);
 int batch_lanes_words(int L);
-// prep: one block per instance ranks gamma and writes the instance's column of the tables
+// prep: one warp per instance ranks gamma and writes the instance's column of the tables
 cudaError_t launch_batch_prep(int64_t B, int L, int k, const uint64_t *bits, const uint64_t *mem,
                               const uint64_t *cap, const uint32_t *bw, const BatchLanes &t, cudaStream_t s);
 // the levels and the backtrack over a prepared chunk; *launches counts the kernels queued
