@@ -28,7 +28,9 @@ namespace pp {
 namespace {
 
 constexpr int kLevelWarps = 4;
+constexpr int kLevelFourBlocks = 5;  // source masks of up to this many nodes: registers capped for four blocks per SM
 constexpr int kPrepWarps = 4;
+constexpr int kWalks = 2;  // staircase walks a lane runs interleaved: the walk is a chain of dependent loads
 constexpr int kBackWarps = 8;
 constexpr int kLanesMinB = 64;  // below this the block-per-instance kernel keeps more of the GPU busy
 constexpr int kLanesMaxK = 8;   // NV <= 7 rows of a source mask in registers
@@ -75,7 +77,7 @@ __host__ __device__ inline PrepLayout prep_layout(int L, int k)
 //     not below the entry, add the column reached, go down a row.  Keys are the bit patterns of the
 //     quotients (positive doubles order like them) plus one, so that a zero in front of every row
 //     stops the walk to the left without a test; row U holds the largest key and empties the column
-//     counter; a walk takes exactly U + L steps.  Two walks per lane run interleaved.
+//     counter; a walk takes exactly U + L steps.  A lane runs several walks interleaved.
 __global__ void __launch_bounds__(kPrepWarps * 32)
 k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, const uint64_t *__restrict__ g_bits,
              const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
@@ -220,28 +222,38 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
         __syncwarp();
         // ---- ranks ----
         {
+            // The column counter is not kept: a step down from row r at column j leaves from byte
+            // offset 8 (r Ks + j), so the sum of the offsets of the U steps down is
+            // 8 (Ks U (U - 1) / 2 + sum of the columns).
             const int n = U * L, steps = U + L;
-            for (int e0 = 0; e0 < n; e0 += 64) {
-                const int eA = e0 + lane, eB = e0 + 32 + lane;
-                const int rA = (int)(((uint32_t)eA * recip_L) >> 16), rB = (int)(((uint32_t)eB * recip_L) >> 16);
-                const int iA = eA - rA * L, iB = eB - rB * L;
-                // an idle lane walks with the smallest key: left along row 0, then down the zeros
-                const unsigned long long xA = eA < n ? K[rA * Ks + 1 + iA] : 1ull;
-                const unsigned long long xB = eB < n ? K[rB * Ks + 1 + iB] : 1ull;
-                int jA = L, jB = L, accA = 0, accB = 0;
-                const unsigned long long *pA = K + L, *pB = K + L;  // the last quotient of row 0
+            const unsigned char *Kb = reinterpret_cast<const unsigned char *>(K);
+            const int down = Ks * 8, start = L * 8;  // the last quotient of row 0
+            const int rows_part = Ks * (U * (U - 1) / 2);
+            for (int e0 = 0; e0 < n; e0 += 32 * kWalks) {
+                unsigned long long x[kWalks];
+                int p[kWalks], sum[kWalks], cell[kWalks];
+#pragma unroll
+                for (int q = 0; q < kWalks; ++q) {
+                    const int e = e0 + 32 * q + lane;
+                    const int r = (int)(((uint32_t)e * recip_L) >> 16), i = e - r * L;
+                    // an idle lane walks with the smallest key: left along row 0, then down the zeros
+                    x[q] = e < n ? K[r * Ks + 1 + i] : 1ull;
+                    cell[q] = e < n ? rowu[r] * L + i : -1;
+                    p[q] = start;
+                    sum[q] = 0;
+                }
 #pragma unroll 2
                 for (int st = 0; st < steps; ++st) {
-                    const bool geA = *pA >= xA, geB = *pB >= xB;
-                    accA += geA ? 0 : jA;
-                    accB += geB ? 0 : jB;
-                    pA += geA ? -1 : Ks;
-                    pB += geB ? -1 : Ks;
-                    jA -= geA ? 1 : 0;
-                    jB -= geB ? 1 : 0;
+#pragma unroll
+                    for (int q = 0; q < kWalks; ++q) {
+                        const bool ge = *reinterpret_cast<const unsigned long long *>(Kb + p[q]) >= x[q];
+                        sum[q] += ge ? 0 : p[q];
+                        p[q] += ge ? -8 : down;
+                    }
                 }
-                if (eA < n) rk[rowu[rA] * L + iA] = (uint16_t)(1 + accA);
-                if (eB < n) rk[rowu[rB] * L + iB] = (uint16_t)(1 + accB);
+#pragma unroll
+                for (int q = 0; q < kWalks; ++q)
+                    if (cell[q] >= 0) rk[cell[q]] = (uint16_t)(1 + (sum[q] >> 3) - rows_part);
             }
         }
         __syncwarp();
@@ -265,19 +277,26 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
 }
 
 template <int NV, int LH>
-__global__ void __launch_bounds__(kLevelWarps * 32)
-k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L)
+__global__ void __launch_bounds__(kLevelWarps * 32, NV <= kLevelFourBlocks ? 4 : 3)
+k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, const int split)
 {
+    // Launched as a programmatic dependent of the kernel before it: nothing is read before that
+    // kernel is complete, and the next one may be scheduled as soon as this one's blocks retire.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
     const int lane = threadIdx.x & 31;
     const uint32_t nmasks = t.moff[NV + 1] - t.moff[NV];
     const int64_t G = (B + 31) >> 5;
-    const int64_t items = G * nmasks;
+    // a level with few source masks gives the targets of one mask to `split` warps
+    const int64_t items = G * nmasks * split;
     const uint32_t full = (1u << k) - 1u;
     const int wfin = (L - 1) >> 1, sfin = ((L - 1) & 1) * 16;
     for (int64_t item = (int64_t)blockIdx.x * kLevelWarps + (threadIdx.x >> 5); item < items;
          item += (int64_t)gridDim.x * kLevelWarps) {
-        const int64_t g = item / nmasks;
-        const uint32_t P = t.mlist[t.moff[NV] + (uint32_t)(item - g * nmasks)];
+        const int64_t g = item / (nmasks * split);
+        const uint32_t within = (uint32_t)(item - g * (nmasks * split));
+        const uint32_t P = t.mlist[t.moff[NV] + within / (uint32_t)split];
+        const int part = (int)(within % (uint32_t)split);
         // lanes past the end of the batch read the last instance's column and store to their own
         const int64_t left = B - g * 32;
         const int valid = left < 32 ? (int)left : 32;
@@ -300,7 +319,10 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L)
             }
         }
         unsigned long long key = kNoBest;
+        int turn = part;
         for (uint32_t wrem = full & ~P; wrem; wrem &= wrem - 1) {
+            if (turn-- != 0) continue;  // another warp's target
+            turn = split - 1;
             const int w = __ffs(wrem) - 1;
             uint32_t gg[LH];
             {
@@ -399,9 +421,12 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
              const uint32_t *__restrict__ g_bw, double *__restrict__ o_beta, int32_t *__restrict__ o_m,
              int32_t *__restrict__ o_cuts, int32_t *__restrict__ o_place, int8_t *__restrict__ o_status)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const int LH = t.LH;
     const double kInf = __longlong_as_double(0x7FF0000000000000ll);
+    __shared__ uint32_t s_len[kBackWarps][kLanesMaxK * 16];  // the instance's window lengths: one load fewer per step
+    uint32_t *mylen = s_len[threadIdx.x >> 5];
     for (int64_t inst = (int64_t)blockIdx.x * kBackWarps + (threadIdx.x >> 5); inst < B;
          inst += (int64_t)gridDim.x * kBackWarps) {
         const size_t g = (size_t)(inst >> 5);
@@ -415,6 +440,8 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
         int32_t *place = o_place + inst * k;
         if (lane < k) place[lane] = -1;
         if (cuts && lane < k - 1) cuts[lane] = -1;
+        __syncwarp();
+        for (int e = lane; e < k * LH; e += 32) mylen[e] = ln[(size_t)e * 32];
         __syncwarp();
         if (bad || key == kNoBest) {
             if (lane == 0) {
@@ -457,7 +484,7 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
             }
             if (j == 0) break;
             const uint32_t P = S & ~(1u << w);
-            const int l0 = c2 - (int)lanes_elem(ln, (size_t)w, LH, c2);
+            const int l0 = c2 - (int)((mylen[w * LH + (c2 >> 1)] >> ((c2 & 1) * 16)) & 0xFFFFu);
             const uint32_t prow = t.rowoff[P];
             unsigned int pick = 0xFFFFFFFFu;
             for (int base = 0; base < (c2 - l0) * k && pick == 0xFFFFFFFFu; base += 32) {
@@ -489,17 +516,32 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
     }
 }
 
+template <typename... Args, typename... Params>
+cudaError_t launch_dependent(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <int LH>
-cudaError_t launch_level(int nv, const BatchLanes &t, int64_t B, int k, int L, unsigned grid, cudaStream_t s)
+cudaError_t launch_level(int nv, const BatchLanes &t, int64_t B, int k, int L, int split, unsigned grid, cudaStream_t s)
 {
     switch (nv) {
 #define PP_CASE(N) \
-    case N: k_lanes_level<N, LH><<<grid, kLevelWarps * 32, 0, s>>>(t, B, k, L); break;
+    case N: return launch_dependent(k_lanes_level<N, LH>, grid, kLevelWarps * 32, s, t, B, k, L, split);
         PP_CASE(1) PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6) PP_CASE(7)
 #undef PP_CASE
         default: return cudaErrorInvalidValue;
     }
-    return cudaGetLastError();
 }
 
 }  // namespace
@@ -542,17 +584,20 @@ cudaError_t launch_batch_lanes(int64_t B, int L, int k, const uint64_t *bits, co
     const int64_t G = (B + 31) >> 5;
     const int jmax = k < L ? k : L;
     uint64_t binom = (uint64_t)k;  // C(k, j - 1), the source masks of level j
+    const int64_t slots = (int64_t)sms * 16;  // warps the GPU holds at a time, roughly
     for (int j = 2; j <= jmax; ++j) {
-        const int64_t items = G * (int64_t)binom;
+        int split = 1;  // warps per source mask: a level with few masks spreads the k - j + 1 targets
+        while (split < k - j + 1 && G * (int64_t)binom * split < 3 * slots) ++split;
+        const int64_t items = G * (int64_t)binom * split;
         int64_t blocks = (items + kLevelWarps - 1) / kLevelWarps;
         const int64_t cap = (int64_t)sms * 32;
         if (blocks > cap) blocks = cap;
         cudaError_t e;
         switch (t.LH) {
-            case 4: e = launch_level<4>(j - 1, t, B, k, L, (unsigned)blocks, s); break;
-            case 8: e = launch_level<8>(j - 1, t, B, k, L, (unsigned)blocks, s); break;
-            case 12: e = launch_level<12>(j - 1, t, B, k, L, (unsigned)blocks, s); break;
-            case 16: e = launch_level<16>(j - 1, t, B, k, L, (unsigned)blocks, s); break;
+            case 4: e = launch_level<4>(j - 1, t, B, k, L, split, (unsigned)blocks, s); break;
+            case 8: e = launch_level<8>(j - 1, t, B, k, L, split, (unsigned)blocks, s); break;
+            case 12: e = launch_level<12>(j - 1, t, B, k, L, split, (unsigned)blocks, s); break;
+            case 16: e = launch_level<16>(j - 1, t, B, k, L, split, (unsigned)blocks, s); break;
             default: e = cudaErrorInvalidValue;
         }
         if (e != cudaSuccess) return e;
@@ -560,8 +605,8 @@ cudaError_t launch_batch_lanes(int64_t B, int L, int k, const uint64_t *bits, co
     }
     int64_t blocks = (B + kBackWarps - 1) / kBackWarps;
     if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
-    k_lanes_back<<<(unsigned)blocks, kBackWarps * 32, 0, s>>>(t, B, L, k, bits, bw, beta, m, cuts, placement, status);
-    return cudaGetLastError();
+    return launch_dependent(k_lanes_back, (unsigned)blocks, kBackWarps * 32, s, t, B, L, k, bits, bw, beta, m, cuts,
+                            placement, status);
 }
 
 }  // namespace pp
