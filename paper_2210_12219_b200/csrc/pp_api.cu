@@ -745,14 +745,16 @@ pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64
     t.moff = lt.moff;
     const size_t line = (size_t)t.LH * 32 * sizeof(uint32_t);
     const size_t b_table = G * t.rows * line, b_rank = G * (size_t)(k * k) * line, b_len = G * (size_t)k * line;
+    const size_t b_win = 2 * b_len;
     const size_t b_key = G * 32 * sizeof(unsigned long long), b_flag = align_up(G * 32, 256);
     unsigned char *buf = nullptr;
-    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), b_table + b_rank + b_len + b_key + b_flag, s));
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), b_table + b_rank + b_len + b_win + b_key + b_flag, s));
     t.table = reinterpret_cast<uint32_t *>(buf);
     t.rank = reinterpret_cast<uint32_t *>(buf + b_table);
     t.len = reinterpret_cast<uint32_t *>(buf + b_table + b_rank);
-    t.key = reinterpret_cast<unsigned long long *>(buf + b_table + b_rank + b_len);
-    t.flag = reinterpret_cast<int8_t *>(buf + b_table + b_rank + b_len + b_key);
+    t.win = reinterpret_cast<uint32_t *>(buf + b_table + b_rank + b_len);
+    t.key = reinterpret_cast<unsigned long long *>(buf + b_table + b_rank + b_len + b_win);
+    t.flag = reinterpret_cast<int8_t *>(buf + b_table + b_rank + b_len + b_win + b_key);
     cudaError_t e = cudaSuccess;
     for (int64_t b0 = 0; b0 < B && e == cudaSuccess; b0 += chunk) {
         const int64_t n = std::min<int64_t>(chunk, B - b0);

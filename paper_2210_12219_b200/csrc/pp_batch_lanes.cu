@@ -15,8 +15,8 @@
 //      source mask P of NV nodes), keeps the NV rows of P in registers (two cut positions per 32-bit
 //      word, LH words per row), and for every node w outside P forms
 //      g[c] = min_v max(dp[P][v][c], rank[v][w][c]) with packed 16-bit min/max, takes the window
-//      minimum over [lo_w(c'), c'-1] (a fully unrolled scan over the distance, cut short at the
-//      longest window of the warp, a lane's shorter window masked arithmetically), stores the row of (P + w, w), and keeps the smallest final state
+//      minimum over [lo_w(c'), c'-1] from a sparse table of g in the lane's own column of shared
+//      memory (the one place where a lane needs an index of its own), stores the row of (P + w, w), and keeps the smallest final state
 //      (value, popcount, mask, node), merged into the instance's key with one atomic per lane;
 //   3. k_lanes_back, one warp per instance: the value of the winning rank and the backtrack by the
 //      threshold rule, lanes over the candidates.
@@ -30,13 +30,24 @@ namespace {
 constexpr int kLevelWarps = 4;
 constexpr int kLevelFourBlocks = 5;  // source masks of up to this many nodes: registers capped for four blocks per SM
 constexpr int kPrepWarps = 4;
+constexpr int kFlagLimit = 1;     // BatchLanes::flag: an input beyond the limits
+constexpr int kFlagDeferred = 2;  // ... the first preparing pass left the ranking to the second
 constexpr int kWalks = 2;  // staircase walks a lane runs interleaved: the walk is a chain of dependent loads
 constexpr int kBackWarps = 8;
 constexpr int kLanesMinB = 64;  // below this the block-per-instance kernel keeps more of the GPU busy
 constexpr int kLanesMaxK = 8;   // NV <= 7 rows of a source mask in registers
 constexpr int kLanesMaxL = 32;  // LH <= 16 words per row
-constexpr uint32_t kMagic = 0x4B000000u;     // bit pattern of 2^23: kMagic | r is the float 2^23 + r for r < 2^23
-constexpr uint32_t kMagicInf = 0x4B00FFFFu;  // the rank of +inf in that form; also caps a masked candidate
+
+// Sparse table of one row g in a warp's shared memory: level s holds T_s[c] = min g[c - 2^s + 1 .. c],
+// two positions per 32-bit word like the rows, word (s, wd) of lane l at byte ((s LH + wd) 32 + l) 4:
+// every lane reads and writes its own bank.  Word kWinLevels * LH holds +inf.  A cell is named by
+// its byte offset without the lane's part, which fits 16 bits.
+constexpr int kWinLevels = 5;  // windows of up to 31 positions
+__host__ __device__ inline uint32_t win_cell(int s, int pos, int LH)
+{
+    return (uint32_t)((s * LH + (pos >> 1)) * 128 + (pos & 1) * 2);
+}
+__host__ __device__ inline size_t win_bytes_per_warp(int LH) { return (size_t)(kWinLevels * LH + 1) * 128; }
 
 // Shared memory of one warp of the preparing kernel (byte offsets; every part 16-byte aligned).
 struct PrepLayout {
@@ -44,10 +55,10 @@ struct PrepLayout {
     int Ks;  // row stride of the quotient matrix in keys: a sentinel in front of the L quotients
 };
 
-__host__ __device__ inline PrepLayout prep_layout(int L, int k)
+__host__ __device__ inline PrepLayout prep_layout(int L, int ucap)
 {
     PrepLayout p;
-    const size_t U = (size_t)k * (k - 1);
+    const size_t U = (size_t)ucap;  // distinct bandwidths the quotient matrix has room for
     size_t o = 0;
     auto take = [&o](size_t bytes) { size_t at = o; o = (o + bytes + 15) & ~(size_t)15; return at; };
     p.Ks = L + 1;
@@ -78,14 +89,18 @@ __host__ __device__ inline PrepLayout prep_layout(int L, int k)
 //     quotients (positive doubles order like them) plus one, so that a zero in front of every row
 //     stops the walk to the left without a test; row U holds the largest key and empties the column
 //     counter; a walk takes exactly U + L steps.  A lane runs several walks interleaved.
+// The matrix is the bulk of a warp's shared memory, and the walks are chains of dependent loads that
+// want many warps in flight, so the kernel runs twice: the first pass has room for k (k - 1) / 2
+// distinct bandwidths (every symmetric network) and marks an instance that has more; the second pass,
+// with room for k (k - 1), takes only the marked ones and returns at once from all others.
 __global__ void __launch_bounds__(kPrepWarps * 32)
 k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, const uint64_t *__restrict__ g_bits,
              const uint64_t *__restrict__ g_mem, const uint64_t *__restrict__ g_cap,
-             const uint32_t *__restrict__ g_bw)
+             const uint32_t *__restrict__ g_bw, const int ucap, const int second_pass)
 {
     extern __shared__ __align__(16) unsigned char smem_prep[];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const PrepLayout lay = prep_layout(L, k);
+    const PrepLayout lay = prep_layout(L, ucap);
     unsigned char *base = smem_prep + (size_t)wid * lay.total;
     unsigned long long *K = reinterpret_cast<unsigned long long *>(base + lay.K);
     unsigned long long *M = reinterpret_cast<unsigned long long *>(base + lay.M);
@@ -104,6 +119,7 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
     const uint32_t recip_k = (65536u + (uint32_t)k - 1u) / (uint32_t)k;
     const uint32_t recip_L = (65536u + (uint32_t)L - 1u) / (uint32_t)L;
     for (int64_t inst = (int64_t)blockIdx.x * kPrepWarps + wid; inst < B; inst += (int64_t)gridDim.x * kPrepWarps) {
+        if (second_pass && !(t.flag[inst] & kFlagDeferred)) continue;  // ranked by the first pass
         __syncwarp();
         // ---- staging, prefix sums of the memory ----
         const unsigned long long b = lane < L ? g_bits[inst * L + lane] : 0ull;
@@ -181,6 +197,7 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
         {
             uint32_t *lT = t.len + (size_t)(inst >> 5) * (size_t)(k * LH) * 32 + (inst & 31);
             uint32_t *tT = t.table + (size_t)(inst >> 5) * (size_t)t.rows * LH * 32 + (inst & 31);
+            uint32_t *wT = t.win + (size_t)(inst >> 5) * (size_t)(k * 2 * LH) * 32 + (inst & 31);
             const unsigned long long Mc = M[lane + 1];  // memory of layers 0..lane
             for (int w = 0; w < k; ++w) {
                 const unsigned long long capw = s_cap[w];
@@ -196,6 +213,17 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
                 const uint32_t inf = (lane < L && Mc <= capw) ? 0u : 0xFFFFu;
                 const uint32_t len0 = __shfl_sync(FULL, len, 2 * lane), len1 = __shfl_sync(FULL, len, 2 * lane + 1);
                 const uint32_t inf0 = __shfl_sync(FULL, inf, 2 * lane), inf1 = __shfl_sync(FULL, inf, 2 * lane + 1);
+                {
+                    // window [lo, lane - 1] of length len >= 1 = union of the two runs of 2^s positions
+                    // that end at lane - 1 and that start at lo, s = floor(log2 len): their sparse-table
+                    // cells; an empty window reads the cell that holds +inf
+                    uint32_t code = win_cell(kWinLevels, 0, LH) * 0x00010001u;
+                    if (len != 0u) {
+                        const int sl = 31 - __clz((int)len);
+                        code = win_cell(sl, lane - 1, LH) | (win_cell(sl, lo + (1 << sl) - 1, LH) << 16);
+                    }
+                    if (lane < 2 * LH) wT[(size_t)(w * 2 * LH + lane) * 32] = code;
+                }
                 if (lane < LH) {
                     lT[(size_t)(w * LH + lane) * 32] = lane < 16 ? len0 | (len1 << 16) : 0u;
                     tT[((size_t)t.rowoff[1u << w] * LH + lane) * 32] = lane < 16 ? inf0 | (inf1 << 16) : 0xFFFFFFFFu;
@@ -206,9 +234,10 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
                 for (int v = k - 1; v >= 0; --v)
                     if (M[L] <= s_cap[v]) best = pack_best(0u, 1, 1u << v, v);
                 t.key[inst] = best;
-                t.flag[inst] = (int8_t)bad;
+                t.flag[inst] = (int8_t)((bad ? kFlagLimit : 0) | (U > ucap ? kFlagDeferred : 0));
             }
         }
+        if (U > ucap) continue;  // more distinct bandwidths than this pass has room for: left to the second pass
         __syncwarp();
         // ---- quotient matrix ----
         for (int r = 0; r <= U; ++r) {
@@ -276,6 +305,17 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
     }
 }
 
+__device__ __forceinline__ void st_shared_u32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_shared_u16(uint32_t addr)
+{
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
+    return v;
+}
+
 template <int NV, int LH>
 __global__ void __launch_bounds__(kLevelWarps * 32, NV <= kLevelFourBlocks ? 4 : 3)
 k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, const int split)
@@ -285,6 +325,10 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     const int lane = threadIdx.x & 31;
+    extern __shared__ __align__(16) unsigned char smem_level[];
+    const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem_level) +
+                           (uint32_t)((threadIdx.x >> 5) * win_bytes_per_warp(LH)) + (uint32_t)lane * 4u;
+    st_shared_u32(sbase + win_cell(kWinLevels, 0, LH), 0xFFFFFFFFu);
     const uint32_t nmasks = t.moff[NV + 1] - t.moff[NV];
     const int64_t G = (B + 31) >> 5;
     // a level with few source masks gives the targets of one mask to `split` warps
@@ -304,7 +348,7 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
         const uint32_t *tab = t.table + (size_t)g * t.rows * (LH * 32) + col;
         uint32_t *tabw = t.table + (size_t)g * t.rows * (LH * 32) + lane;
         const uint32_t *rk = t.rank + (size_t)g * (size_t)(k * k) * (LH * 32) + col;
-        const uint32_t *ln = t.len + (size_t)g * (size_t)k * (LH * 32) + col;
+        const uint32_t *wn = t.win + (size_t)g * (size_t)(k * 2) * (LH * 32) + col;
         uint32_t d[NV][LH];
         int vs[NV];
         {
@@ -324,6 +368,9 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
             if (turn-- != 0) continue;  // another warp's target
             turn = split - 1;
             const int w = __ffs(wrem) - 1;
+            uint32_t cw[2 * LH];  // the window cells of this node, asked for before anything else
+#pragma unroll
+            for (int c2 = 0; c2 < 2 * LH; ++c2) cw[c2] = wn[(size_t)(w * 2 * LH + c2) * 32];
             uint32_t gg[LH];
             {
                 const uint32_t *r0 = rk + (size_t)((vs[0] * k + w) * LH) * 32;
@@ -344,59 +391,41 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
 #pragma unroll
                 for (int wd = 0; wd < LH; ++wd) gg[wd] = __vminu2(gg[wd], __vmaxu2(d[NV - 1][wd], r1[wd * 32]));
             }
-            // window lengths of this node, and the longest one among the 32 instances
-            uint32_t lw[LH];
-            uint32_t m2 = 0;
+            // Window minimum over [lo_w(c2), c2 - 1] for every c2: the sparse table of g goes to the
+            // lane's column of shared memory, level s from level s - 1 by one packed minimum per word
+            // (level 1 needs the row shifted by one position), and every cut position then reads the
+            // two cells the preparing kernel named for it.
+            {
+                uint32_t cur[LH];
 #pragma unroll
-            for (int wd = 0; wd < LH; ++wd) {
-                lw[wd] = ln[(size_t)(w * LH + wd) * 32];
-                m2 = __vmaxu2(m2, lw[wd]);
-            }
-            const int wmax = (int)__reduce_max_sync(0xFFFFFFFFu, max(m2 & 0xFFFFu, m2 >> 16));
-            // The window minimum runs on floats that hold 2^23 + rank exactly (such floats order like
-            // their bit patterns): out[c2] = min of g over the len(c2) positions before c2.  Every
-            // distance up to the warp's longest window is taken; a lane whose own window is shorter
-            // adds 2^16 to the candidate, t = saturate(distance - len) being 0 inside the window and
-            // 1 outside, so that the masking is two multiply-add-pipe instructions and the 3-input
-            // integer minimum takes two candidates at a time.
-            float uf[2 * LH], lf[2 * LH];
-#pragma unroll
-            for (int wd = 0; wd < LH; ++wd) {
-                uf[2 * wd] = __uint_as_float(__byte_perm(gg[wd], kMagic, 0x7610));
-                uf[2 * wd + 1] = __uint_as_float(__byte_perm(gg[wd], kMagic, 0x7632));
-                lf[2 * wd] = __uint_as_float(__byte_perm(lw[wd], kMagic, 0x7610));
-                lf[2 * wd + 1] = __uint_as_float(__byte_perm(lw[wd], kMagic, 0x7632));
-            }
-            // distances in blocks of four, all positions inside a block: the positions are independent
-            // of one another, and the test against the warp's longest window is made once per block
-            int ob[2 * LH];
-#pragma unroll
-            for (int c2 = 0; c2 < 2 * LH; ++c2) ob[c2] = (int)kMagicInf;
-#pragma unroll
-            for (int d0 = 1; d0 < 2 * LH; d0 += 4) {
-                if (d0 > wmax) break;
-#pragma unroll
-                for (int c2 = d0; c2 < 2 * LH; ++c2) {
-                    int x[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int dd = d0 + q;
-                        x[q] = (int)kMagicInf;
-                        if (dd <= c2) {
-                            const float t = __saturatef((8388608.0f + (float)dd) - lf[c2]);
-                            x[q] = __float_as_int(fmaf(t, 65536.0f, uf[c2 - dd]));
-                        }
-                    }
-                    ob[c2] = __vimin3_s32(ob[c2], x[0], x[1]);
-                    if (d0 + 2 <= c2) ob[c2] = __vimin3_s32(ob[c2], x[2], x[3]);
+                for (int wd = 0; wd < LH; ++wd) {
+                    st_shared_u32(sbase + win_cell(0, 2 * wd, LH), gg[wd]);
+                    const uint32_t prev = wd ? gg[wd - 1] : 0xFFFFFFFFu;
+                    cur[wd] = __vminu2(gg[wd], __byte_perm(prev, gg[wd], 0x5432));  // positions 2wd-1, 2wd
+                    st_shared_u32(sbase + win_cell(1, 2 * wd, LH), cur[wd]);
                 }
+#pragma unroll
+                for (int sl = 2; sl < kWinLevels; ++sl) {
+                    const int shift = 1 << (sl - 2);  // words
+#pragma unroll
+                    for (int wd = LH - 1; wd >= 0; --wd) {  // downwards: cur[wd - shift] is still the level below
+                        if (wd >= shift) cur[wd] = __vminu2(cur[wd], cur[wd - shift]);
+                        st_shared_u32(sbase + win_cell(sl, 2 * wd, LH), cur[wd]);
+                    }
+                }
+            }
+            uint32_t ob[2 * LH];
+#pragma unroll
+            for (int c2 = 0; c2 < 2 * LH; ++c2) {
+                const uint32_t a = ld_shared_u16(sbase + (cw[c2] & 0xFFFFu)), b2 = ld_shared_u16(sbase + (cw[c2] >> 16));
+                ob[c2] = min(a, b2);
             }
             const uint32_t S2 = P | (1u << w);
             const uint32_t row = t.rowoff[S2] + (uint32_t)__popc(S2 & ((1u << w) - 1u));
             uint32_t xw = 0xFFFFFFFFu;
 #pragma unroll
             for (int wd = 0; wd < LH; ++wd) {
-                const uint32_t o = __byte_perm((uint32_t)ob[2 * wd], (uint32_t)ob[2 * wd + 1], 0x5410);
+                const uint32_t o = ob[2 * wd] | (ob[2 * wd + 1] << 16);
                 tabw[((size_t)row * LH + wd) * 32] = o;
                 if (wd == wfin) xw = o;
             }
@@ -435,7 +464,7 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
         const uint32_t *rk = t.rank + g * (size_t)(k * k) * (size_t)(LH * 32) + col;
         const uint32_t *ln = t.len + g * (size_t)k * (size_t)(LH * 32) + col;
         const unsigned long long key = t.key[inst];
-        const int bad = t.flag[inst];
+        const int bad = t.flag[inst] & kFlagLimit;
         int32_t *cuts = o_cuts ? o_cuts + inst * (k - 1) : nullptr;
         int32_t *place = o_place + inst * k;
         if (lane < k) place[lane] = -1;
@@ -517,12 +546,13 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
 }
 
 template <typename... Args, typename... Params>
-cudaError_t launch_dependent(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t s, Args... args)
+cudaError_t launch_dependent(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem, cudaStream_t s,
+                             Args... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -537,7 +567,13 @@ cudaError_t launch_level(int nv, const BatchLanes &t, int64_t B, int k, int L, i
 {
     switch (nv) {
 #define PP_CASE(N) \
-    case N: return launch_dependent(k_lanes_level<N, LH>, grid, kLevelWarps * 32, s, t, B, k, L, split);
+    case N: {                                                                                                  \
+        const size_t sm = win_bytes_per_warp(LH) * kLevelWarps;                                                \
+        cudaError_t e = cudaFuncSetAttribute(k_lanes_level<N, LH>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                             (int)sm);                                                          \
+        if (e != cudaSuccess) return e;                                                                        \
+        return launch_dependent(k_lanes_level<N, LH>, grid, kLevelWarps * 32, sm, s, t, B, k, L, split);       \
+    }
         PP_CASE(1) PP_CASE(2) PP_CASE(3) PP_CASE(4) PP_CASE(5) PP_CASE(6) PP_CASE(7)
 #undef PP_CASE
         default: return cudaErrorInvalidValue;
@@ -561,16 +597,25 @@ cudaError_t launch_batch_prep(int64_t B, int L, int k, const uint64_t *bits, con
                               const uint64_t *cap, const uint32_t *bw, const BatchLanes &t, cudaStream_t s)
 {
     if (B <= 0) return cudaSuccess;
-    const size_t sm = prep_layout(L, k).total * kPrepWarps;
-    cudaError_t e = cudaFuncSetAttribute(k_lanes_prep, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    if (e != cudaSuccess) return e;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     int64_t blocks = (B + kPrepWarps - 1) / kPrepWarps;
     if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
-    k_lanes_prep<<<(unsigned)blocks, kPrepWarps * 32, sm, s>>>(t, B, L, k, bits, mem, cap, bw);
-    return cudaGetLastError();
+    const int ufull = k * (k - 1), uhalf = ufull / 2;
+    for (int pass = 0; pass < 2; ++pass) {
+        const int ucap = pass ? ufull : uhalf;
+        const size_t sm = prep_layout(L, ucap).total * kPrepWarps;
+        // the attribute is set to the larger size both times: it belongs to the function, and another
+        // host thread may be between its own two launches
+        cudaError_t e = cudaFuncSetAttribute(k_lanes_prep, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(prep_layout(L, ufull).total * kPrepWarps));
+        if (e != cudaSuccess) return e;
+        k_lanes_prep<<<(unsigned)blocks, kPrepWarps * 32, sm, s>>>(t, B, L, k, bits, mem, cap, bw, ucap, pass);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_batch_lanes(int64_t B, int L, int k, const uint64_t *bits, const uint32_t *bw,
@@ -605,7 +650,7 @@ cudaError_t launch_batch_lanes(int64_t B, int L, int k, const uint64_t *bits, co
     }
     int64_t blocks = (B + kBackWarps - 1) / kBackWarps;
     if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
-    return launch_dependent(k_lanes_back, (unsigned)blocks, kBackWarps * 32, s, t, B, L, k, bits, bw, beta, m, cuts,
+    return launch_dependent(k_lanes_back, (unsigned)blocks, kBackWarps * 32, 0, s, t, B, L, k, bits, bw, beta, m, cuts,
                             placement, status);
 }
 

@@ -95,6 +95,8 @@ struct BatchLanes {
     uint32_t *table;          // [group][compact row][LH][32]: states, two cut positions per word
     uint32_t *rank;           // [group][v * k + w][LH][32]: gamma ranks, same packing
     uint32_t *len;            // [group][w][LH][32]: window lengths c' - lo_w(c'), same packing
+    uint32_t *win;            // [group][w][2 LH][32]: per cut position the two sparse-table cells whose minimum
+                              // is the window minimum, as byte offsets into a warp's table (see pp_batch_lanes.cu)
     unsigned long long *key;  // [group][32]: smallest final state so far (value, popcount, mask, node)
     int8_t *flag;             // [group][32]: 1 = an input beyond the limits
     const uint32_t *rowoff;   // [2^k]: compact row of (S, lowest node of S), rows ordered by (popcount, mask, node)
