@@ -454,7 +454,11 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
     const int lane = threadIdx.x & 31;
     const int LH = t.LH;
     const double kInf = __longlong_as_double(0x7FF0000000000000ll);
-    __shared__ uint32_t s_len[kBackWarps][kLanesMaxK * 16];  // the instance's window lengths: one load fewer per step
+    // the instance's rank table and window lengths, fetched in one go: the winning rank is looked up and
+    // every backtrack step reads them, and only the states are left to come from global memory
+    __shared__ uint32_t s_rank[kBackWarps][kLanesMaxK * kLanesMaxK * 16];
+    __shared__ uint32_t s_len[kBackWarps][kLanesMaxK * 16];
+    uint32_t *myrank = s_rank[threadIdx.x >> 5];
     uint32_t *mylen = s_len[threadIdx.x >> 5];
     for (int64_t inst = (int64_t)blockIdx.x * kBackWarps + (threadIdx.x >> 5); inst < B;
          inst += (int64_t)gridDim.x * kBackWarps) {
@@ -470,6 +474,8 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
         if (lane < k) place[lane] = -1;
         if (cuts && lane < k - 1) cuts[lane] = -1;
         __syncwarp();
+#pragma unroll 8
+        for (int e = lane; e < k * k * LH; e += 32) myrank[e] = rk[(size_t)e * 32];
         for (int e = lane; e < k * LH; e += 32) mylen[e] = ln[(size_t)e * 32];
         __syncwarp();
         if (bad || key == kNoBest) {
@@ -490,7 +496,7 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
             // quotient is beta* (equal ranks hold equal doubles)
             int found = -1;
             for (int e = lane; e < k * k * LH; e += 32) {
-                const uint32_t x = rk[(size_t)e * 32];
+                const uint32_t x = myrank[e];
                 if ((x & 0xFFFFu) == rstar) found = 2 * e;
                 if ((x >> 16) == rstar) found = 2 * e + 1;
             }
@@ -515,24 +521,23 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
             const uint32_t P = S & ~(1u << w);
             const int l0 = c2 - (int)((mylen[w * LH + (c2 >> 1)] >> ((c2 & 1) * 16)) & 0xFFFFu);
             const uint32_t prow = t.rowoff[P];
+            const int np = __popc(P), total = (c2 - l0) * np;
+            // candidates (position, node of P), lanes over all of them at once: the loads of a step are
+            // independent, the smallest (position, node) that meets the threshold wins
             unsigned int pick = 0xFFFFFFFFu;
-            for (int base = 0; base < (c2 - l0) * k && pick == 0xFFFFFFFFu; base += 32) {
-                const int it = base + lane;
-                if (it < (c2 - l0) * k) {
-                    const int c = l0 + it / k, v = it - (it / k) * k;
-                    if ((P >> v) & 1u) {
-                        const uint32_t a = lanes_elem(tab, (size_t)prow + __popc(P & ((1u << v) - 1u)), LH, c);
-                        const uint32_t b = lanes_elem(rk, (size_t)(v * k + w), LH, c);
-                        const uint32_t mx = a > b ? a : b;
-                        if (mx <= rstar) pick = ((unsigned)c << 5) | (unsigned)v;
-                    }
-                }
-                // candidates ascend with the lane (position first, then node): the first hit of the
-                // earliest chunk that has one is the smallest (position, node)
-                for (int o = 16; o; o >>= 1) {
-                    const unsigned int other = __shfl_xor_sync(0xFFFFFFFFu, pick, o);
-                    pick = other < pick ? other : pick;
-                }
+#pragma unroll 2
+            for (int it = lane; it < total; it += 32) {
+                const int ci = it / np, vi = it - ci * np;
+                const int c = l0 + ci, v = (int)__fns(P, 0, vi + 1);
+                const uint32_t a = lanes_elem(tab, (size_t)prow + vi, LH, c);
+                const uint32_t b = (myrank[(v * k + w) * LH + (c >> 1)] >> ((c & 1) * 16)) & 0xFFFFu;
+                const uint32_t mx = a > b ? a : b;
+                const unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
+                if (mx <= rstar && kk < pick) pick = kk;
+            }
+            for (int o = 16; o; o >>= 1) {
+                const unsigned int other = __shfl_xor_sync(0xFFFFFFFFu, pick, o);
+                pick = other < pick ? other : pick;
             }
             if (pick == 0xFFFFFFFFu) {  // inconsistent table: flag the instance, keep going
                 if (lane == 0) o_status[inst] = (int8_t)PP_ERR_CUDA;
