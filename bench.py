@@ -240,7 +240,10 @@ def run_ours(args):
         ms_total = max_over_ranks(ms_local)
         clk = clocks.summary()
         prof = prob.last_solve_profile()
-        launches_per_step = prof.total_launches + 2
+        # the batched solve of this shape: two preparing passes, one kernel per popcount level from 2 up,
+        # the backtrack; the evaluator is one launch
+        batch_launches = 2 + (min(BATCH_K, BATCH_L) - 1) + 1
+        launches_per_step = prof.total_launches + batch_launches + 1
         if args.step_only:  # for a profiler's launch list: the warm-up and the timed steps, nothing else
             if rank == 0:
                 print("step only: %d steps, %.4f ms per step, %d launches per step"

@@ -222,6 +222,9 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
                         const int sl = 31 - __clz((int)len);
                         code = win_cell(sl, lane - 1, LH) | (win_cell(sl, lo + (1 << sl) - 1, LH) << 16);
                     }
+                    // position 0 has no window: its entry carries the highest level this node's windows read
+                    const uint32_t longest = __reduce_max_sync(FULL, len);
+                    if (lane == 0) code = longest > 1u ? (uint32_t)(31 - __clz((int)longest)) : 0u;
                     if (lane < 2 * LH) wT[(size_t)(w * 2 * LH + lane) * 32] = code;
                 }
                 if (lane < LH) {
@@ -328,7 +331,18 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
     extern __shared__ __align__(16) unsigned char smem_level[];
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem_level) +
                            (uint32_t)((threadIdx.x >> 5) * win_bytes_per_warp(LH)) + (uint32_t)lane * 4u;
+    // A state of j segments ends at layer j - 1 at the earliest: rows of this level's sources (NV
+    // nodes) are +inf before position NV - 1 and the rows written here before position NV.  Words
+    // that hold only such positions are neither read, computed nor written, here and in the next
+    // level alike; their cells of the sparse table are set to +inf once.
+    constexpr int W0 = (NV - 1) / 2;  // first word of a source row that can hold a state
+    constexpr int C0 = NV;            // first position of a target row that can
+    constexpr int O0 = NV / 2;        // its word: the first one stored (the next level's W0)
     st_shared_u32(sbase + win_cell(kWinLevels, 0, LH), 0xFFFFFFFFu);
+#pragma unroll
+    for (int sl = 0; sl < kWinLevels; ++sl)
+#pragma unroll
+        for (int wd = 0; wd < W0; ++wd) st_shared_u32(sbase + win_cell(sl, 2 * wd, LH), 0xFFFFFFFFu);
     const uint32_t nmasks = t.moff[NV + 1] - t.moff[NV];
     const int64_t G = (B + 31) >> 5;
     // a level with few source masks gives the targets of one mask to `split` warps
@@ -359,7 +373,7 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
                 vs[vi] = __ffs(rem) - 1;
                 rem &= rem - 1;
 #pragma unroll
-                for (int wd = 0; wd < LH; ++wd) d[vi][wd] = tab[((size_t)(row0 + vi) * LH + wd) * 32];
+                for (int wd = W0; wd < LH; ++wd) d[vi][wd] = tab[((size_t)(row0 + vi) * LH + wd) * 32];
             }
         }
         unsigned long long key = kNoBest;
@@ -368,63 +382,72 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
             if (turn-- != 0) continue;  // another warp's target
             turn = split - 1;
             const int w = __ffs(wrem) - 1;
-            uint32_t cw[2 * LH];  // the window cells of this node, asked for before anything else
+            // the window cells of this node, asked for before anything else; position 0 has no window
+            // and its entry carries the highest level of the sparse table this (instance, node) reads
+            uint32_t cw[2 * LH];
+            const uint32_t lvl = wn[(size_t)(w * 2 * LH) * 32];
 #pragma unroll
-            for (int c2 = 0; c2 < 2 * LH; ++c2) cw[c2] = wn[(size_t)(w * 2 * LH + c2) * 32];
+            for (int c2 = C0; c2 < 2 * LH; ++c2) cw[c2] = wn[(size_t)(w * 2 * LH + c2) * 32];
             uint32_t gg[LH];
             {
                 const uint32_t *r0 = rk + (size_t)((vs[0] * k + w) * LH) * 32;
 #pragma unroll
-                for (int wd = 0; wd < LH; ++wd) gg[wd] = __vmaxu2(d[0][wd], r0[wd * 32]);
+                for (int wd = W0; wd < LH; ++wd) gg[wd] = __vmaxu2(d[0][wd], r0[wd * 32]);
             }
 #pragma unroll
             for (int vi = 1; vi + 1 < NV; vi += 2) {
                 const uint32_t *r1 = rk + (size_t)((vs[vi] * k + w) * LH) * 32;
                 const uint32_t *r2 = rk + (size_t)((vs[vi + 1] * k + w) * LH) * 32;
 #pragma unroll
-                for (int wd = 0; wd < LH; ++wd)
+                for (int wd = W0; wd < LH; ++wd)
                     gg[wd] = __vimin3_u16x2(gg[wd], __vmaxu2(d[vi][wd], r1[wd * 32]),
                                             __vmaxu2(d[vi + 1][wd], r2[wd * 32]));
             }
             if (!(NV & 1)) {
                 const uint32_t *r1 = rk + (size_t)((vs[NV - 1] * k + w) * LH) * 32;
 #pragma unroll
-                for (int wd = 0; wd < LH; ++wd) gg[wd] = __vminu2(gg[wd], __vmaxu2(d[NV - 1][wd], r1[wd * 32]));
+                for (int wd = W0; wd < LH; ++wd) gg[wd] = __vminu2(gg[wd], __vmaxu2(d[NV - 1][wd], r1[wd * 32]));
             }
             // Window minimum over [lo_w(c2), c2 - 1] for every c2: the sparse table of g goes to the
             // lane's column of shared memory, level s from level s - 1 by one packed minimum per word
-            // (level 1 needs the row shifted by one position), and every cut position then reads the
-            // two cells the preparing kernel named for it.
+            // (level 1 needs the row shifted by one position), up to the highest level a lane of this
+            // warp reads; every cut position then reads the two cells the preparing kernel named for it.
             {
+                const int top = (int)__reduce_max_sync(0xFFFFFFFFu, lvl);
                 uint32_t cur[LH];
 #pragma unroll
-                for (int wd = 0; wd < LH; ++wd) {
+                for (int wd = W0; wd < LH; ++wd) {
                     st_shared_u32(sbase + win_cell(0, 2 * wd, LH), gg[wd]);
-                    const uint32_t prev = wd ? gg[wd - 1] : 0xFFFFFFFFu;
+                    const uint32_t prev = wd > W0 ? gg[wd - 1] : 0xFFFFFFFFu;
                     cur[wd] = __vminu2(gg[wd], __byte_perm(prev, gg[wd], 0x5432));  // positions 2wd-1, 2wd
                     st_shared_u32(sbase + win_cell(1, 2 * wd, LH), cur[wd]);
                 }
 #pragma unroll
                 for (int sl = 2; sl < kWinLevels; ++sl) {
+                    if (sl > top) break;
                     const int shift = 1 << (sl - 2);  // words
 #pragma unroll
-                    for (int wd = LH - 1; wd >= 0; --wd) {  // downwards: cur[wd - shift] is still the level below
-                        if (wd >= shift) cur[wd] = __vminu2(cur[wd], cur[wd - shift]);
+                    for (int wd = LH - 1; wd >= W0; --wd) {  // downwards: cur[wd - shift] is still the level below
+                        if (wd - shift >= W0) cur[wd] = __vminu2(cur[wd], cur[wd - shift]);
                         st_shared_u32(sbase + win_cell(sl, 2 * wd, LH), cur[wd]);
                     }
                 }
             }
             uint32_t ob[2 * LH];
 #pragma unroll
-            for (int c2 = 0; c2 < 2 * LH; ++c2) {
-                const uint32_t a = ld_shared_u16(sbase + (cw[c2] & 0xFFFFu)), b2 = ld_shared_u16(sbase + (cw[c2] >> 16));
-                ob[c2] = min(a, b2);
+            for (int c2 = 2 * O0; c2 < 2 * LH; ++c2) {
+                ob[c2] = 0xFFFFu;
+                if (c2 >= C0) {
+                    const uint32_t a = ld_shared_u16(sbase + (cw[c2] & 0xFFFFu));
+                    const uint32_t b2 = ld_shared_u16(sbase + (cw[c2] >> 16));
+                    ob[c2] = min(a, b2);
+                }
             }
             const uint32_t S2 = P | (1u << w);
             const uint32_t row = t.rowoff[S2] + (uint32_t)__popc(S2 & ((1u << w) - 1u));
             uint32_t xw = 0xFFFFFFFFu;
 #pragma unroll
-            for (int wd = 0; wd < LH; ++wd) {
+            for (int wd = O0; wd < LH; ++wd) {
                 const uint32_t o = ob[2 * wd] | (ob[2 * wd + 1] << 16);
                 tabw[((size_t)row * LH + wd) * 32] = o;
                 if (wd == wfin) xw = o;
@@ -529,7 +552,8 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
             for (int it = lane; it < total; it += 32) {
                 const int ci = it / np, vi = it - ci * np;
                 const int c = l0 + ci, v = (int)__fns(P, 0, vi + 1);
-                const uint32_t a = lanes_elem(tab, (size_t)prow + vi, LH, c);
+                // a state of np segments ends at layer np - 1 at the earliest; earlier positions were never written
+                const uint32_t a = c >= np - 1 ? lanes_elem(tab, (size_t)prow + vi, LH, c) : 0xFFFFu;
                 const uint32_t b = (myrank[(v * k + w) * LH + (c >> 1)] >> ((c & 1) * 16)) & 0xFFFFu;
                 const uint32_t mx = a > b ? a : b;
                 const unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
