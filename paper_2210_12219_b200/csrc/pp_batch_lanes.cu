@@ -477,11 +477,7 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
     const int lane = threadIdx.x & 31;
     const int LH = t.LH;
     const double kInf = __longlong_as_double(0x7FF0000000000000ll);
-    // the instance's rank table and window lengths, fetched in one go: the winning rank is looked up and
-    // every backtrack step reads them, and only the states are left to come from global memory
-    __shared__ uint32_t s_rank[kBackWarps][kLanesMaxK * kLanesMaxK * 16];
-    __shared__ uint32_t s_len[kBackWarps][kLanesMaxK * 16];
-    uint32_t *myrank = s_rank[threadIdx.x >> 5];
+    __shared__ uint32_t s_len[kBackWarps][kLanesMaxK * 16];  // the instance's window lengths: one load fewer per step
     uint32_t *mylen = s_len[threadIdx.x >> 5];
     for (int64_t inst = (int64_t)blockIdx.x * kBackWarps + (threadIdx.x >> 5); inst < B;
          inst += (int64_t)gridDim.x * kBackWarps) {
@@ -497,8 +493,6 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
         if (lane < k) place[lane] = -1;
         if (cuts && lane < k - 1) cuts[lane] = -1;
         __syncwarp();
-#pragma unroll 8
-        for (int e = lane; e < k * k * LH; e += 32) myrank[e] = rk[(size_t)e * 32];
         for (int e = lane; e < k * LH; e += 32) mylen[e] = ln[(size_t)e * 32];
         __syncwarp();
         if (bad || key == kNoBest) {
@@ -518,8 +512,9 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
             // an entry of the rank table that carries the winning rank names a (node pair, layer) whose
             // quotient is beta* (equal ranks hold equal doubles)
             int found = -1;
+#pragma unroll 8
             for (int e = lane; e < k * k * LH; e += 32) {
-                const uint32_t x = myrank[e];
+                const uint32_t x = rk[(size_t)e * 32];
                 if ((x & 0xFFFFu) == rstar) found = 2 * e;
                 if ((x >> 16) == rstar) found = 2 * e + 1;
             }
@@ -554,7 +549,7 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
                 const int c = l0 + ci, v = (int)__fns(P, 0, vi + 1);
                 // a state of np segments ends at layer np - 1 at the earliest; earlier positions were never written
                 const uint32_t a = c >= np - 1 ? lanes_elem(tab, (size_t)prow + vi, LH, c) : 0xFFFFu;
-                const uint32_t b = (myrank[(v * k + w) * LH + (c >> 1)] >> ((c & 1) * 16)) & 0xFFFFu;
+                const uint32_t b = lanes_elem(rk, (size_t)(v * k + w), LH, c);
                 const uint32_t mx = a > b ? a : b;
                 const unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
                 if (mx <= rstar && kk < pick) pick = kk;
