@@ -181,15 +181,21 @@ pp_status pp_eval_plans_packed_dev(pp_problem *p, int64_t B, int64_t total, cons
 
 /*
  * Many independent instances of the same shape (L, k) in one call; each instance is the
- * exact search above, done by one thread block with its whole state table in shared memory.
+ * exact search above.
  *   out_bits [B*L], mem [B*L], node_mem [B*k], bw [B*k*k]   inputs, instance-major
  *   beta_ms [B], m [B], cuts [B*(k-1)], placement [B*k], status [B] (PP_OK / PP_INFEASIBLE,
  *   or PP_ERR_LIMIT for an instance with a value above the limits)
+ * Two device paths give the same results.  From 64 instances on, with 2 <= k <= 8 and L <= 32, a
+ * warp sweeps 32 instances at once (one per lane); the state, rank and window tables of up to 4096
+ * instances at a time live in scratch memory that the call takes from the library's own memory pool
+ * and gives back, both ordered on the stream (k = 8, L = 24: 53 KB per instance; PP_ERR_NOMEM if
+ * the pool cannot supply it; longer batches are worked off in pieces of 4096 on the same stream).
+ * Otherwise one thread block solves one instance with its whole state table in shared memory.
  * Returns PP_ERR_LIMIT without touching outputs when the instance shape does not fit one block:
  * k > 12, k*(k-1)*L + 1 > 65534 (ranks are 16-bit), or k * 2^(k-1) * L 16-bit states plus the
- * rank tables beyond the shared memory of a block (k = 8, L = 24 needs 73 KB).  Host variant is synchronous and uses the
- * legacy default stream; the _dev variant takes device pointers and a stream and is
- * asynchronous.  cuts may be NULL when k == 1.
+ * rank tables beyond the shared memory of a block (k = 8, L = 24 needs 73 KB).  Host variant is
+ * synchronous and uses the legacy default stream; the _dev variant takes device pointers and a
+ * stream and is asynchronous.  cuts may be NULL when k == 1.
  */
 pp_status pp_solve_exact_batch(int64_t B, int32_t L, int32_t k, const uint64_t *out_bits,
                                const uint64_t *mem, const uint64_t *node_mem, const uint32_t *bw,
