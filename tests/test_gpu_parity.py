@@ -455,6 +455,36 @@ def test_batched_solve_instance_per_lane_shapes():
         assert got.plan(b) == oracle.dp_naive(insts[b]).plan()
 
 
+def test_batched_solve_asymmetric_links_and_pieces():
+    # a network whose two directions differ has up to k (k - 1) distinct bandwidths: such instances are
+    # ranked by the second preparing pass, symmetric ones by the first, in one batch
+    rng = np.random.Generator(np.random.PCG64(20240607))
+    for L, k, n in ((11, 5, 96), (24, 8, 70), (32, 7, 65)):
+        insts = [W.random_small(63000 + 100 * L + i, L, k, tight=(i % 5 == 1), dead_links=0.2 if i % 4 == 3 else 0.0)
+                 for i in range(n)]
+        bits, mem, cap, bw = _stack(insts)
+        for i in range(0, n, 2):  # every other instance: independent draws per direction, some links dead
+            m = rng.integers(1000, 12000, size=(k, k)).astype(np.uint32)
+            m[rng.random((k, k)) < 0.1] = 0
+            np.fill_diagonal(m, 0)
+            bw[i] = m
+            insts[i] = W.Instance(L, k, bits[i], mem[i], cap[i], bw[i], "asymmetric")
+        got = pp.solve_exact_batch(L, k, bits, mem, cap, bw)
+        for b, inst in enumerate(insts):
+            want = oracle.dp_naive(inst)
+            assert got.status[b] == want.status, (L, k, b)
+            assert got.plan(b) == want.plan(), (L, k, b)
+            assert got.beta_ms[b] == want.beta_ms or np.isinf(want.beta_ms)
+    # more instances than share the scratch tables at a time: worked off in pieces on the same stream
+    L, k, n = 5, 3, 4096 + 45
+    insts = [W.random_small(64000 + i, L, k, tight=(i % 3 == 1), ties=(i % 7 == 2)) for i in range(n)]
+    got = pp.solve_exact_batch(L, k, *_stack(insts))
+    for b in list(range(0, n, 17)) + list(range(4090, n)):
+        want = oracle.dp_naive(insts[b])
+        assert got.status[b] == want.status and got.plan(b) == want.plan(), b
+        assert got.beta_ms[b] == want.beta_ms or np.isinf(want.beta_ms)
+
+
 def test_workspace_and_stream_from_torch():
     import torch
     inst = W.config_resnet50_shaped()
