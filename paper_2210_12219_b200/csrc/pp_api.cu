@@ -746,15 +746,29 @@ pp_status pp_solve_exact_batch_dev(int64_t B, int32_t L, int32_t k, const uint64
     const size_t line = (size_t)t.LH * 32 * sizeof(uint32_t);
     const size_t b_table = G * t.rows * line, b_rank = G * (size_t)(k * k) * line, b_len = G * (size_t)k * line;
     const size_t b_win = 2 * b_len;
-    const size_t b_key = G * 32 * sizeof(unsigned long long), b_flag = align_up(G * 32, 256);
+    const size_t b_key = G * 32 * sizeof(unsigned long long), b_flag = align_up(G * 32, 256), b_err = 256;
     unsigned char *buf = nullptr;
-    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), b_table + b_rank + b_len + b_win + b_key + b_flag, s));
+    PP_CUDA(staging_alloc(reinterpret_cast<void **>(&buf), b_table + b_rank + b_len + b_win + b_key + b_flag + b_err, s));
     t.table = reinterpret_cast<uint32_t *>(buf);
     t.rank = reinterpret_cast<uint32_t *>(buf + b_table);
     t.len = reinterpret_cast<uint32_t *>(buf + b_table + b_rank);
     t.win = reinterpret_cast<uint32_t *>(buf + b_table + b_rank + b_len);
     t.key = reinterpret_cast<unsigned long long *>(buf + b_table + b_rank + b_len + b_win);
     t.flag = reinterpret_cast<int8_t *>(buf + b_table + b_rank + b_len + b_win + b_key);
+    t.err = reinterpret_cast<int32_t *>(buf + b_table + b_rank + b_len + b_win + b_key + b_flag);
+    t.table_words = b_table / 4;
+    t.rank_words = b_rank / 4;
+    t.len_words = b_len / 4;
+    t.win_words = b_win / 4;
+#ifdef PP_DEBUG_BOUNDS
+    {  // the bounds-checking build records violations here; k_lanes_back turns them into PP_ERR_CUDA
+        cudaError_t ez = cudaMemsetAsync(t.err, 0, sizeof(int32_t), s);
+        if (ez != cudaSuccess) {
+            cudaFreeAsync(buf, s);
+            return from_cuda(ez);
+        }
+    }
+#endif
     cudaError_t e = cudaSuccess;
     for (int64_t b0 = 0; b0 < B && e == cudaSuccess; b0 += chunk) {
         const int64_t n = std::min<int64_t>(chunk, B - b0);

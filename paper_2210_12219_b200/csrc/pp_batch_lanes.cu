@@ -49,6 +49,18 @@ __host__ __device__ inline uint32_t win_cell(int s, int pos, int LH)
 }
 __host__ __device__ inline size_t win_bytes_per_warp(int LH) { return (size_t)(kWinLevels * LH + 1) * 128; }
 
+// Checked access to one of the tables of BatchLanes: in the bounds-checking build an address outside
+// [base, base + words) is recorded in the error word and the access skipped (a load gives +inf); in
+// the normal build PP_IN_BOUNDS is `true` and these are plain loads and stores.
+__device__ __forceinline__ uint32_t ld_table(const BatchLanes &t, const uint32_t *p, const uint32_t *base, size_t words)
+{
+    return PP_IN_BOUNDS(t, (size_t)(p - base), words) ? *p : 0xFFFFFFFFu;
+}
+__device__ __forceinline__ void st_table(const BatchLanes &t, uint32_t *p, const uint32_t *base, size_t words, uint32_t v)
+{
+    if (PP_IN_BOUNDS(t, (size_t)(p - base), words)) *p = v;
+}
+
 // Shared memory of one warp of the preparing kernel (byte offsets; every part 16-byte aligned).
 struct PrepLayout {
     size_t K, M, bits, sorted, cap, bw, ubw, rk, pair_u, rowu, pos, total;
@@ -225,11 +237,12 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
                     // position 0 has no window: its entry carries the highest level this node's windows read
                     const uint32_t longest = __reduce_max_sync(FULL, len);
                     if (lane == 0) code = longest > 1u ? (uint32_t)(31 - __clz((int)longest)) : 0u;
-                    if (lane < 2 * LH) wT[(size_t)(w * 2 * LH + lane) * 32] = code;
+                    if (lane < 2 * LH) st_table(t, wT + (size_t)(w * 2 * LH + lane) * 32, t.win, t.win_words, code);
                 }
                 if (lane < LH) {
-                    lT[(size_t)(w * LH + lane) * 32] = lane < 16 ? len0 | (len1 << 16) : 0u;
-                    tT[((size_t)t.rowoff[1u << w] * LH + lane) * 32] = lane < 16 ? inf0 | (inf1 << 16) : 0xFFFFFFFFu;
+                    st_table(t, lT + (size_t)(w * LH + lane) * 32, t.len, t.len_words, lane < 16 ? len0 | (len1 << 16) : 0u);
+                    st_table(t, tT + ((size_t)t.rowoff[1u << w] * LH + lane) * 32, t.table, t.table_words,
+                             lane < 16 ? inf0 | (inf1 << 16) : 0xFFFFFFFFu);
                 }
             }
             if (lane == 0) {
@@ -302,7 +315,7 @@ k_lanes_prep(const BatchLanes t, const int64_t B, const int L, const int k, cons
                     const uint32_t c = c1 < L ? rk[u * L + q1] : 0xFFFFu;
                     word = a | (c << 16);
                 }
-                if (lane < LH) rT[(size_t)(pr * LH + lane) * 32] = word;
+                if (lane < LH) st_table(t, rT + (size_t)(pr * LH + lane) * 32, t.rank, t.rank_words, word);
             }
         }
     }
@@ -373,7 +386,8 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
                 vs[vi] = __ffs(rem) - 1;
                 rem &= rem - 1;
 #pragma unroll
-                for (int wd = W0; wd < LH; ++wd) d[vi][wd] = tab[((size_t)(row0 + vi) * LH + wd) * 32];
+                for (int wd = W0; wd < LH; ++wd)
+                    d[vi][wd] = ld_table(t, tab + ((size_t)(row0 + vi) * LH + wd) * 32, t.table, t.table_words);
             }
         }
         unsigned long long key = kNoBest;
@@ -385,14 +399,15 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
             // the window cells of this node, asked for before anything else; position 0 has no window
             // and its entry carries the highest level of the sparse table this (instance, node) reads
             uint32_t cw[2 * LH];
-            const uint32_t lvl = wn[(size_t)(w * 2 * LH) * 32];
+            const uint32_t lvl = ld_table(t, wn + (size_t)(w * 2 * LH) * 32, t.win, t.win_words);
 #pragma unroll
-            for (int c2 = C0; c2 < 2 * LH; ++c2) cw[c2] = wn[(size_t)(w * 2 * LH + c2) * 32];
+            for (int c2 = C0; c2 < 2 * LH; ++c2)
+                cw[c2] = ld_table(t, wn + (size_t)(w * 2 * LH + c2) * 32, t.win, t.win_words);
             uint32_t gg[LH];
             {
                 const uint32_t *r0 = rk + (size_t)((vs[0] * k + w) * LH) * 32;
 #pragma unroll
-                for (int wd = W0; wd < LH; ++wd) gg[wd] = __vmaxu2(d[0][wd], r0[wd * 32]);
+                for (int wd = W0; wd < LH; ++wd) gg[wd] = __vmaxu2(d[0][wd], ld_table(t, r0 + wd * 32, t.rank, t.rank_words));
             }
 #pragma unroll
             for (int vi = 1; vi + 1 < NV; vi += 2) {
@@ -400,13 +415,13 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
                 const uint32_t *r2 = rk + (size_t)((vs[vi + 1] * k + w) * LH) * 32;
 #pragma unroll
                 for (int wd = W0; wd < LH; ++wd)
-                    gg[wd] = __vimin3_u16x2(gg[wd], __vmaxu2(d[vi][wd], r1[wd * 32]),
-                                            __vmaxu2(d[vi + 1][wd], r2[wd * 32]));
+                    gg[wd] = __vimin3_u16x2(gg[wd], __vmaxu2(d[vi][wd], ld_table(t, r1 + wd * 32, t.rank, t.rank_words)),
+                                            __vmaxu2(d[vi + 1][wd], ld_table(t, r2 + wd * 32, t.rank, t.rank_words)));
             }
             if (!(NV & 1)) {
                 const uint32_t *r1 = rk + (size_t)((vs[NV - 1] * k + w) * LH) * 32;
 #pragma unroll
-                for (int wd = W0; wd < LH; ++wd) gg[wd] = __vminu2(gg[wd], __vmaxu2(d[NV - 1][wd], r1[wd * 32]));
+                for (int wd = W0; wd < LH; ++wd) gg[wd] = __vminu2(gg[wd], __vmaxu2(d[NV - 1][wd], ld_table(t, r1 + wd * 32, t.rank, t.rank_words)));
             }
             // Window minimum over [lo_w(c2), c2 - 1] for every c2: the sparse table of g goes to the
             // lane's column of shared memory, level s from level s - 1 by one packed minimum per word
@@ -438,8 +453,12 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
             for (int c2 = 2 * O0; c2 < 2 * LH; ++c2) {
                 ob[c2] = 0xFFFFu;
                 if (c2 >= C0) {
-                    const uint32_t a = ld_shared_u16(sbase + (cw[c2] & 0xFFFFu));
-                    const uint32_t b2 = ld_shared_u16(sbase + (cw[c2] >> 16));
+                    // (bounds-checking build: a cell outside the warp's table reads the +inf cell instead)
+                    const uint32_t o1 = PP_IN_BOUNDS(t, cw[c2] & 0xFFFFu, win_bytes_per_warp(LH) - 126) ? cw[c2] & 0xFFFFu
+                                                                                                       : win_cell(kWinLevels, 0, LH);
+                    const uint32_t o2 = PP_IN_BOUNDS(t, cw[c2] >> 16, win_bytes_per_warp(LH) - 126) ? cw[c2] >> 16
+                                                                                                 : win_cell(kWinLevels, 0, LH);
+                    const uint32_t a = ld_shared_u16(sbase + o1), b2 = ld_shared_u16(sbase + o2);
                     ob[c2] = min(a, b2);
                 }
             }
@@ -449,7 +468,7 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
 #pragma unroll
             for (int wd = O0; wd < LH; ++wd) {
                 const uint32_t o = ob[2 * wd] | (ob[2 * wd + 1] << 16);
-                tabw[((size_t)row * LH + wd) * 32] = o;
+                st_table(t, tabw + ((size_t)row * LH + wd) * 32, t.table, t.table_words, o);
                 if (wd == wfin) xw = o;
             }
             const uint32_t x = (xw >> sfin) & 0xFFFFu;
@@ -463,9 +482,10 @@ k_lanes_level(const BatchLanes t, const int64_t B, const int k, const int L, con
 }
 
 // state or rank of one (row, position) of one instance's column
-__device__ __forceinline__ uint32_t lanes_elem(const uint32_t *base, size_t row, int LH, int c)
+__device__ __forceinline__ uint32_t lanes_elem(const BatchLanes &t, const uint32_t *col, const uint32_t *base, size_t words,
+                                               size_t row, int LH, int c)
 {
-    return (base[(row * LH + (size_t)(c >> 1)) * 32] >> ((c & 1) * 16)) & 0xFFFFu;
+    return (ld_table(t, col + (row * LH + (size_t)(c >> 1)) * 32, base, words) >> ((c & 1) * 16)) & 0xFFFFu;
 }
 
 __global__ void __launch_bounds__(kBackWarps * 32)
@@ -493,7 +513,7 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
         if (lane < k) place[lane] = -1;
         if (cuts && lane < k - 1) cuts[lane] = -1;
         __syncwarp();
-        for (int e = lane; e < k * LH; e += 32) mylen[e] = ln[(size_t)e * 32];
+        for (int e = lane; e < k * LH; e += 32) mylen[e] = ld_table(t, ln + (size_t)e * 32, t.len, t.len_words);
         __syncwarp();
         if (bad || key == kNoBest) {
             if (lane == 0) {
@@ -514,7 +534,7 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
             int found = -1;
 #pragma unroll 8
             for (int e = lane; e < k * k * LH; e += 32) {
-                const uint32_t x = rk[(size_t)e * 32];
+                const uint32_t x = ld_table(t, rk + (size_t)e * 32, t.rank, t.rank_words);
                 if ((x & 0xFFFFu) == rstar) found = 2 * e;
                 if ((x >> 16) == rstar) found = 2 * e + 1;
             }
@@ -529,6 +549,9 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
             o_beta[inst] = bstar;
             o_m[inst] = m;
             o_status[inst] = (int8_t)PP_OK;
+#ifdef PP_DEBUG_BOUNDS
+            if (*t.err != 0) o_status[inst] = (int8_t)PP_ERR_CUDA;  // an index left its table somewhere in this piece
+#endif
         }
         for (int j = m - 1; j >= 0; --j) {
             if (lane == 0) {
@@ -548,8 +571,8 @@ k_lanes_back(const BatchLanes t, const int64_t B, const int L, const int k, cons
                 const int ci = it / np, vi = it - ci * np;
                 const int c = l0 + ci, v = (int)__fns(P, 0, vi + 1);
                 // a state of np segments ends at layer np - 1 at the earliest; earlier positions were never written
-                const uint32_t a = c >= np - 1 ? lanes_elem(tab, (size_t)prow + vi, LH, c) : 0xFFFFu;
-                const uint32_t b = lanes_elem(rk, (size_t)(v * k + w), LH, c);
+                const uint32_t a = c >= np - 1 ? lanes_elem(t, tab, t.table, t.table_words, (size_t)prow + vi, LH, c) : 0xFFFFu;
+                const uint32_t b = lanes_elem(t, rk, t.rank, t.rank_words, (size_t)(v * k + w), LH, c);
                 const uint32_t mx = a > b ? a : b;
                 const unsigned int kk = ((unsigned)c << 5) | (unsigned)v;
                 if (mx <= rstar && kk < pick) pick = kk;

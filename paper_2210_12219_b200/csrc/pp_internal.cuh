@@ -99,6 +99,8 @@ struct BatchLanes {
                               // is the window minimum, as byte offsets into a warp's table (see pp_batch_lanes.cu)
     unsigned long long *key;  // [group][32]: smallest final state so far (value, popcount, mask, node)
     int8_t *flag;             // [group][32]: 1 = an input beyond the limits
+    int32_t *err;             // device error word (bounds-checking build: kErrBounds when an index left its table)
+    size_t table_words, rank_words, len_words, win_words;  // sizes of the four tables in 32-bit words
     const uint32_t *rowoff;   // [2^k]: compact row of (S, lowest node of S), rows ordered by (popcount, mask, node)
     const uint32_t *mlist;    // masks by (popcount, value)
     const uint32_t *moff;     // [k + 2]: first entry of each popcount in mlist

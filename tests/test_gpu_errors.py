@@ -48,6 +48,18 @@ def test_bounds_checking_build_runs_the_parity_cases_clean():
         nseg, ends, nodes = W.random_plans(inst, 500, seed=2)
         with pp.Problem.from_instance(inst) as p:
             assert np.array_equal(p.eval_plans(nseg, ends, nodes)[0], oracle.eval_plans(inst, nseg, ends, nodes)[0])
+        # the batched search, both device paths (64 instances and more take the instance-per-lane
+        # kernels); a recorded violation would come back as PP_ERR_CUDA in the instance's status
+        for L, k, n in ((24, 8, 70), (7, 8, 65), (32, 4, 66), (13, 5, 20)):
+            insts = [W.random_small(82000 + 100 * L + i, L, k, tight=(i % 3 == 1), dead_links=0.25 if i % 4 == 3 else 0.0)
+                     for i in range(n)]
+            got = pp.solve_exact_batch(L, k, np.stack([i.layer_out_bits for i in insts]),
+                                       np.stack([i.layer_mem_bytes for i in insts]),
+                                       np.stack([i.node_mem_bytes for i in insts]),
+                                       np.stack([i.bw_kbps for i in insts]))
+            for b, inst in enumerate(insts):
+                want = oracle.dp_naive(inst)
+                assert got.status[b] == want.status and got.plan(b) == want.plan(), (L, k, b)
     assert binding.LIB_PATH.endswith("libpp.so")
 
 
