@@ -411,8 +411,8 @@ def test_batched_solve_full_config():
 
 
 def test_batched_solve_odd_shapes():
-    # L <= 32 ranks the quotients from sorted runs of the next power of two (L itself a power of
-    # two included), longer chains from single keys
+    # batches too small for the instance-per-lane kernels: one block per instance, chains shorter and
+    # longer than a warp, a power of two long, more nodes than layers
     for L, k, n in ((1, 1, 3), (2, 3, 6), (5, 2, 9), (13, 5, 40), (3, 6, 12), (16, 3, 8), (30, 7, 10),
                     (32, 4, 8), (33, 4, 8), (70, 3, 6)):
         insts = [W.random_small(60000 + 100 * L + i, L, k, tight=(i % 3 == 1), ties=(i % 3 == 2),
