@@ -421,6 +421,52 @@ def run_ours(args):
                      "setting": "ResNet50-shaped chain, 14 devices of 32 MB, geometric graph (pairwise Eq. 12), "
                                 "3 classes, 24 colourings per probe"}
 
+        # the kernels behind the two stages, timed in bulk on the device (not part of the timed step):
+        # Algorithm 1 on 4096 copies of the ResNet50-shaped chain with capacities of 16..271 MB, and the
+        # colour-coding k-path query (paths of 8 vertices) 4096 times on a 50-node geometric graph
+        def timed(fn, reps=7):
+            ts = []
+            for _ in range(reps):
+                a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b2.record(stream)
+                b2.synchronize()
+                ts.append(a.elapsed_time(b2))
+            return statistics.median(ts[2:])
+
+        chain = W.config_resnet50_shaped()
+        n_ch, Lc = 4096, chain.L
+        c_w = tt(np.tile(chain.layer_out_bits, (n_ch, 1)))
+        c_m = tt(np.tile(chain.layer_mem_bytes, (n_ch, 1)))
+        c_kap = tt((np.arange(n_ch, dtype=np.uint64) % 256 + 16) * np.uint64(1 << 20))
+        c_cost = torch.empty(n_ch, dtype=torch.int64, device=dev)
+        c_m_out = torch.empty(n_ch, dtype=torch.int32, device=dev)
+        c_cuts = torch.empty(n_ch * Lc, dtype=torch.int32, device=dev)
+        c_sizes = torch.empty(n_ch * Lc, dtype=torch.int64, device=dev)
+        c_stat = torch.empty(n_ch, dtype=torch.int8, device=dev)
+        part_ms = timed(lambda: pp.partition_minsum_batch_dev(
+            n_ch, Lc, c_w.data_ptr(), c_m.data_ptr(), c_kap.data_ptr(), Lc, c_cost.data_ptr(), c_m_out.data_ptr(),
+            c_cuts.data_ptr(), c_sizes.data_ptr(), c_stat.data_ptr(), stream.cuda_stream))
+        g50, _ = W.geometric_bandwidths(50, 5, link="pairwise")
+        n_q, kk_path = 4096, 8
+        q_rng = np.random.default_rng(4242)
+        q_thr = tt(np.full(n_q, int(np.median(g50[g50 > 0])), dtype=np.uint32))
+        q_any = tt(np.full(n_q, -1, dtype=np.int32))
+        q_alive = tt(np.full(n_q, (1 << 50) - 1, dtype=np.uint64).view(np.int64))
+        q_col = tt(q_rng.integers(0, kk_path, size=(n_q, 50), dtype=np.uint8))
+        q_bw = tt(g50.astype(np.uint32))
+        q_found = torch.empty(n_q, dtype=torch.uint8, device=dev)
+        q_path = torch.empty(n_q * kk_path, dtype=torch.int32, device=dev)
+        kpath_ms = timed(lambda: pp.kpath_colour_batch_dev(
+            50, q_bw.data_ptr(), n_q, kk_path, q_thr.data_ptr(), q_any.data_ptr(), q_any.data_ptr(),
+            q_alive.data_ptr(), q_col.data_ptr(), q_found.data_ptr(), q_path.data_ptr(), stream.cuda_stream))
+        heuristic["stage_kernels"] = {
+            "partition_minsum": {"chains": n_ch, "L": Lc, "ms": part_ms, "chains_per_s": n_ch / (part_ms * 1e-3),
+                                 "feasible": int((c_stat == 0).sum().item())},
+            "kpath_colour": {"queries": n_q, "nodes": 50, "path_vertices": kk_path, "ms": kpath_ms,
+                             "queries_per_s": n_q / (kpath_ms * 1e-3), "found": int(q_found.sum().item())}}
+
     sol_rec = pp.pp_solution.from_buffer_copy(d_sol.cpu().numpy().tobytes())
     ms_per_step = ms_total / args.steps
     value, _ = aggregate_over_ranks(relax_step * args.steps, ms_local * 1e-3, dist, dev)

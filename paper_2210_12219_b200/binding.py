@@ -381,6 +381,14 @@ def kpath_colour_batch(bw, kk: int, threshold, start, end, alive, colours):
     return found, path
 
 
+def kpath_colour_batch_dev(n, bw_ptr, Q, kk, threshold_ptr, start_ptr, end_ptr, alive_ptr, colours_ptr, found_ptr,
+                           path_ptr, cuda_stream: int = 0):
+    st = lib().pp_kpath_colour_batch_dev(int(n), ctypes.c_void_p(bw_ptr), int(Q), int(kk),
+                                         *(ctypes.c_void_p(x) for x in (threshold_ptr, start_ptr, end_ptr, alive_ptr,
+                                                                       colours_ptr, found_ptr, path_ptr, cuda_stream)))
+    _check(st, "pp_kpath_colour_batch_dev")
+
+
 def kpath_matching(bw, sizes, n_classes: int, draws, cuda_stream: int = 0):
     """pp_kpath_matching: bw uint32 [n, n], sizes uint64 [n_cuts], draws uint32 [trials, n] ->
     (status, nodes int32 [n_cuts + 1], cut_threshold uint32 [n_cuts])."""
