@@ -694,6 +694,25 @@ def run_only(args):
             got = entry(BATCH_L, BATCH_K, b_bits, b_mem, b_cap, b_bw)
         print("%s of %d: %d with a plan" % (args.only, args.batch, int((got.status == 0).sum())))
         return
+    if args.only == "partition":  # Algorithm 1 on --batch copies of the ResNet50-shaped chain
+        chain = W.config_resnet50_shaped()
+        kap = (np.arange(args.batch, dtype=np.uint64) % 256 + 16) * np.uint64(1 << 20)
+        for _ in range(args.solves):
+            got = pp.partition_minsum_batch(np.tile(chain.layer_out_bits, (args.batch, 1)),
+                                            np.tile(chain.layer_mem_bytes, (args.batch, 1)), kap, chain.L)
+        print("partition of %d chains: %d feasible" % (args.batch, int((got.status == 0).sum())))
+        return
+    if args.only == "kpath":  # colour-coding k-path, --batch random colourings on a 50-node geometric graph
+        g50, _ = W.geometric_bandwidths(50, 5, link="pairwise")
+        rng = np.random.default_rng(4242)
+        Q, kk = args.batch, 8
+        for _ in range(args.solves):
+            found, _ = pp.kpath_colour_batch(g50, kk, np.full(Q, int(np.median(g50[g50 > 0])), np.uint32),
+                                             np.full(Q, -1, np.int32), np.full(Q, -1, np.int32),
+                                             np.full(Q, (1 << 50) - 1, np.uint64),
+                                             rng.integers(0, kk, size=(Q, 50), dtype=np.uint8))
+        print("k-path of %d queries: %d found" % (Q, int(found.sum())))
+        return
     large = W.config_large()
     k = args.k
     inst = W.Instance(large.L, k, large.layer_out_bits, large.layer_mem_bytes,
@@ -729,12 +748,12 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--step-only", action="store_true",
                     help="run the warm-up and the timed steps and exit (for a profiler's launch list)")
-    ap.add_argument("--only", choices=["sweep", "unequal", "batch", "greedy", "random"],
+    ap.add_argument("--only", choices=["sweep", "unequal", "batch", "greedy", "random", "partition", "kpath"],
                     help="profiler helper: run one part a few times and exit (see run_only)")
     ap.add_argument("--k", type=int, default=16, help="--only sweep/unequal/random: nodes kept of the Large instance")
     ap.add_argument("--solves", type=int, default=2, help="--only: repetitions")
     ap.add_argument("--mode", type=int, default=None, help="--only sweep: pp_problem_force_generic mode")
-    ap.add_argument("--batch", type=int, default=N_BATCH, help="--only batch/greedy: instances")
+    ap.add_argument("--batch", type=int, default=N_BATCH, help="--only batch/greedy/partition/kpath: instances, chains or queries")
     ap.add_argument("--plans", type=int, default=N_PLANS, help="--only random: plans")
     args = ap.parse_args()
     if args.only:
