@@ -486,12 +486,15 @@ def run_ours(args):
         pin(p_ends.view(np.int16)).view(np.uint16), pin(p_nodes)
     hb_bits, hb_mem, hb_cap, hb_bw = pin(b_bits), pin(b_mem), pin(b_cap), pin(b_bw)
 
+    h_beta = torch.empty(N_PLANS, dtype=torch.float64).pin_memory().numpy()  # results land in pinned memory too
+    h_pstat = torch.empty(N_PLANS, dtype=torch.uint8).pin_memory().numpy()
+
     def step_host():
         with pp.Problem(L, h_bits, h_mem, k, h_cap, h_bw) as p2:
             p2.set_workspace(ws)
             s = p2.solve_exact()
             bsol = pp.solve_exact_batch(BATCH_L, BATCH_K, hb_bits, hb_mem, hb_cap, hb_bw)
-            beta, pstat = p2.eval_plans_packed(h_nseg, h_off, h_pends, h_pnodes)
+            beta, pstat = p2.eval_plans_packed(h_nseg, h_off, h_pends, h_pnodes, out=(h_beta, h_pstat))
         return s, bsol, beta, pstat
 
     for _ in range(2):

@@ -237,17 +237,19 @@ class Problem:
                                        (nseg_ptr, ends_ptr, nodes_ptr, beta_ptr, status_ptr))),
                "pp_eval_plans_dev")
 
-    def eval_plans_packed(self, nseg, plan_off, ends, nodes):
+    def eval_plans_packed(self, nseg, plan_off, ends, nodes, out=None):
         """pp_eval_plans_packed: uint8 [B], uint32 [B + 1], uint16 [total], uint8 [total] (host) ->
-        (beta_ms float64 [B], plan_status uint8 [B])."""
+        (beta_ms float64 [B], plan_status uint8 [B]).  out = (beta, status): arrays of the caller to
+        write into (page-locked ones make the copy back a plain DMA)."""
         nseg, p0 = _host(nseg, np.uint8)
         B = nseg.shape[0]
         plan_off, p1 = _host(plan_off, np.uint32)
         ends, p2 = _host(ends, np.uint16)
         nodes, p3 = _host(nodes, np.uint8)
         assert plan_off.size == B + 1 and ends.size == nodes.size
-        beta = np.empty(B, dtype=np.float64)
-        status = np.empty(B, dtype=np.uint8)
+        beta, status = out if out is not None else (np.empty(B, dtype=np.float64), np.empty(B, dtype=np.uint8))
+        assert beta.dtype == np.float64 and status.dtype == np.uint8 and beta.size == B and status.size == B
+        assert beta.flags.c_contiguous and status.flags.c_contiguous
         _check(lib().pp_eval_plans_packed(self._h, B, ends.size, p0, p1, p2, p3, ctypes.c_void_p(beta.ctypes.data),
                                           ctypes.c_void_p(status.ctypes.data)), "pp_eval_plans_packed")
         return beta, status
