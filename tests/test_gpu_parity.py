@@ -434,7 +434,7 @@ def test_batched_solve_instance_per_lane_shapes():
     # from 64 instances on, chains of up to 32 layers on up to 8 nodes are solved 32 instances to a
     # warp: every row width of that path (4, 8, 12, 16 words), batches that end inside a group of 32,
     # more nodes than layers, and the degenerate inputs
-    for L, k, n in ((2, 3, 64), (5, 2, 97), (7, 8, 65), (13, 5, 130), (16, 3, 96), (17, 6, 71), (24, 8, 100),
+    for L, k, n in ((1, 4, 64), (2, 3, 64), (5, 2, 97), (7, 8, 65), (13, 5, 130), (16, 3, 96), (17, 6, 71), (24, 8, 100),
                     (25, 4, 64), (30, 7, 70), (32, 4, 89)):
         insts = [W.random_small(61000 + 100 * L + i, L, k, tight=(i % 3 == 1), ties=(i % 3 == 2),
                                 dead_links=0.25 if i % 4 == 3 else 0.0) for i in range(n)]
