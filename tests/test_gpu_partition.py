@@ -20,9 +20,10 @@ def _built():
     pp.lib()
 
 
-def _check(weights, mem, kappa, cap_seg):
+def _check(weights, mem, kappa, cap_seg, every=1):
     got = pp.partition_minsum_batch(weights, mem, kappa, cap_seg)
-    for b in range(weights.shape[0]):
+    B = weights.shape[0]
+    for b in sorted(set(range(0, B, every)) | set(range(max(B - 40, 0), B))):
         want = OP.minsum_partition(weights[b].tolist(), mem[b].tolist(), int(kappa[b]))
         if want.status == OP.INFEASIBLE:
             assert got.status[b] == pp.PP_INFEASIBLE and got.m[b] == 0 and got.cost[b] == 0
@@ -49,20 +50,25 @@ def test_hand_worked_partitions_on_gpu():
             assert (int(got.cost[0]), int(got.m[0]), tuple(got.cuts[0, :m - 1].tolist())) == (cost, m, cuts)
 
 
+# 60 chains: one warp per chain; 8200 chains of up to 64 points: one lane per chain, the last group of
+# 32 not full, every 41st chain and the last 40 compared
+@pytest.mark.parametrize("B", [60, 8200])
 @pytest.mark.parametrize("L", [1, 2, 7, 31, 32, 33, 64, 100, 257])
-def test_random_chains(L):
-    rng = np.random.default_rng(100 + L)
-    B = 60
+def test_random_chains(L, B):
+    if B > 60 and L > 64:
+        pytest.skip("chains this long take the warp-per-chain kernel at any batch size")
+    rng = np.random.default_rng(100 + L + B)
+    every = 1 if B == 60 else 41
     mem = rng.integers(1, 40, size=(B, L)).astype(np.uint64)
     kappa = rng.integers(30, 160, size=B).astype(np.uint64)
     kappa[::7] = 20  # some chains hold a point that fits nowhere
     weights = rng.integers(0, 10**7, size=(B, L)).astype(np.uint64)
     weights[1::3] = rng.integers(0, 4, size=weights[1::3].shape)  # tie-heavy: class numbers
-    got = _check(weights, mem, kappa, L)
+    got = _check(weights, mem, kappa, L, every)
     assert (got.status == pp.PP_OK).sum() > 10
     # rows shorter than the plan: refused per chain, cost and m still reported
     if L >= 31:
-        _check(weights, mem, kappa, 2)
+        _check(weights, mem, kappa, 2, every)
 
 
 def test_model_shaped_chains_and_limits():
