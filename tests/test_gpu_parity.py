@@ -449,8 +449,11 @@ def test_batched_solve_instance_per_lane_shapes():
     insts = [W.random_small(62000 + i, 12, 4) for i in range(80)]
     bits, mem, cap, bw = _stack(insts)
     bits[17, 3] = np.uint64(1) << np.uint64(41)
+    mem[20, :2] = np.uint64(1) << np.uint64(63)  # the 64-bit sum of the memory wraps
+    bw[23, 1, 2] = np.uint32(1) << np.uint32(24)
     got = pp.solve_exact_batch(12, 4, bits, mem, cap, bw)
-    assert got.status[17] == pp.PP_ERR_LIMIT and got.m[17] == 0 and np.isinf(got.beta_ms[17])
+    for b in (17, 20, 23):
+        assert got.status[b] == pp.PP_ERR_LIMIT and got.m[b] == 0 and np.isinf(got.beta_ms[b]), b
     for b in (16, 18, 79):
         assert got.plan(b) == oracle.dp_naive(insts[b]).plan()
 
