@@ -6,77 +6,119 @@
 // vertices whose vertices carry kk different colours (the colouring is an input: the caller draws
 // it), from `start` to `end` when those are given; a walk that reaches `end` early is not continued.
 // The table of the colour-coding method, reach[C] = set of vertices at which a colourful path with
-// colour set C ends, is a 64-bit vertex mask per colour set and lives in shared memory.  One block
-// per query sweeps the colour sets by popcount, like the node sets of the exact search: a set C
-// hands N(reach[C]), the neighbours of its end vertices, to every set C + c, restricted to the
-// vertices of colour c.  The path is rebuilt from the table, lowest predecessor first.
+// colour set C ends, is a 64-bit vertex mask per colour set and lives in shared memory.  One warp
+// per query sweeps the colour sets: a set C hands N(reach[C]), the neighbours of its end vertices,
+// to every set C + c, restricted to the vertices of colour c.  The path is rebuilt from the table,
+// lowest predecessor first.
 #include "pp_internal.cuh"
 
 namespace pp {
 
 namespace {
 
-constexpr int kKpathThreads = 128;
+// One warp per query, lane <-> vertices lane and lane + 32 (n <= 64); the table of a query is the
+// warp's slice of shared memory.  The colour sets are taken in numerical order: a set only receives
+// from its subsets, which are smaller numbers, so no level structure and no block barrier is needed.
+// For a set C the neighbours of reach[C] are the OR of the adjacency masks of its end vertices (each
+// lane offers the masks of its two vertices, one warp-wide OR), and lane c hands the neighbours of
+// colour c to the set C + c: every lane writes a word of its own.
+struct KpathLayout {
+    size_t reach, radj, cls, col, total;
+};
+__host__ __device__ inline KpathLayout kpath_layout(int kk)
+{
+    KpathLayout l;
+    l.reach = 0;
+    l.radj = ((size_t)1 << kk) * 8;
+    l.cls = l.radj + 64 * 8;
+    l.col = l.cls + 16 * 8;
+    l.total = l.col + 64;
+    return l;
+}
+__host__ __device__ inline int kpath_warps_per_block(int kk) { return kk <= 9 ? 4 : kk <= 11 ? 2 : 1; }
 
-__global__ void __launch_bounds__(kKpathThreads)
+__device__ __forceinline__ unsigned long long warp_or_u64(unsigned long long x)
+{
+    const uint32_t lo = __reduce_or_sync(0xFFFFFFFFu, (uint32_t)x);
+    const uint32_t hi = __reduce_or_sync(0xFFFFFFFFu, (uint32_t)(x >> 32));
+    return ((unsigned long long)hi << 32) | lo;
+}
+
+__global__ void __launch_bounds__(128)
 k_kpath_colour(int n, int kk, int64_t Q, const uint32_t *__restrict__ bw, const uint32_t *__restrict__ threshold,
                const int32_t *__restrict__ start, const int32_t *__restrict__ end,
                const unsigned long long *__restrict__ alive_q, const uint8_t *__restrict__ colours,
                uint8_t *__restrict__ found, int32_t *__restrict__ path)
 {
-    extern __shared__ unsigned long long reach[];  // [2^kk]
-    __shared__ unsigned long long adj[64], radj[64], cls[16];
-    __shared__ uint8_t col[64];
-    const int tid = threadIdx.x;
+    extern __shared__ __align__(16) unsigned char smem_kpath[];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    const KpathLayout lay = kpath_layout(kk);
+    unsigned char *base = smem_kpath + (size_t)wid * lay.total;
+    unsigned long long *reach = reinterpret_cast<unsigned long long *>(base + lay.reach);  // [2^kk]
+    unsigned long long *radj = reinterpret_cast<unsigned long long *>(base + lay.radj);    // [64]
+    unsigned long long *cls = reinterpret_cast<unsigned long long *>(base + lay.cls);      // [16]
+    uint8_t *col = base + lay.col;                                                         // [64]
     const uint32_t nsets = 1u << kk, full = nsets - 1u;
-    for (int64_t q = blockIdx.x; q < Q; q += gridDim.x) {
+    for (int64_t q = (int64_t)blockIdx.x * warps + wid; q < Q; q += (int64_t)gridDim.x * warps) {
         const uint32_t t = threshold[q];
         const int s = start[q], u = end[q];
         const unsigned long long alive = alive_q[q] & (n == 64 ? ~0ull : ((1ull << n) - 1ull));
-        __syncthreads();
-        for (uint32_t C = tid; C < nsets; C += kKpathThreads) reach[C] = 0ull;
-        if (tid < 16) cls[tid] = 0ull;
-        if (tid < 64) {
+        __syncwarp();
+        for (uint32_t C = lane; C < nsets; C += 32) reach[C] = 0ull;
+        // adjacency of the class-X subgraph among the available nodes, two vertices per lane
+        unsigned long long adj2[2];
+        int colv[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int v = lane + 32 * h;
             unsigned long long out = 0ull, in = 0ull;
-            if (tid < n && ((alive >> tid) & 1ull)) {
+            if (v < n && ((alive >> v) & 1ull)) {
                 for (int w = 0; w < n; ++w) {
-                    if (w == tid || !((alive >> w) & 1ull)) continue;
-                    const uint32_t fwd = bw[tid * n + w], back = bw[w * n + tid];
+                    if (w == v || !((alive >> w) & 1ull)) continue;
+                    const uint32_t fwd = bw[v * n + w], back = bw[w * n + v];
                     if (fwd > 0 && fwd >= t) out |= 1ull << w;
                     if (back > 0 && back >= t) in |= 1ull << w;
                 }
             }
-            adj[tid] = out;
-            radj[tid] = in;
-            col[tid] = tid < n ? colours[q * n + tid] : (uint8_t)255;
+            adj2[h] = out;
+            radj[v] = in;
+            colv[h] = v < n ? colours[q * n + v] : 255;
+            col[v] = (uint8_t)colv[h];
         }
-        __syncthreads();
-        if (tid < n && ((alive >> tid) & 1ull) && col[tid] < kk) {
-            atomicOr(&cls[col[tid]], 1ull << tid);                                           // vertices of each colour
-            if (s < 0 || s == tid) atomicOr(&reach[1u << col[tid]], 1ull << tid);  // paths of one vertex
-        }
-        __syncthreads();
-        const unsigned long long not_end = (u >= 0 && u < 64) ? ~(1ull << u) : ~0ull;
-        for (int level = 1; level < kk; ++level) {
-            for (uint32_t C = 1 + tid; C < nsets; C += kKpathThreads) {
-                if (__popc(C) != level) continue;
-                unsigned long long X = reach[C] & not_end;  // a walk that has reached the end vertex stops
-                if (!X) continue;
-                unsigned long long N = 0ull;
-                while (X) {
-                    const int v = __ffsll((long long)X) - 1;
-                    X &= X - 1ull;
-                    N |= adj[v];
-                }
-                for (uint32_t rem = full & ~C; rem; rem &= rem - 1u) {
-                    const int c = __ffs(rem) - 1;
-                    const unsigned long long add = N & cls[c];
-                    if (add) atomicOr(&reach[C | (1u << c)], add);
-                }
+        // vertices of each colour, and the paths of one vertex
+        unsigned long long mine = 0ull;  // lane c: the vertices of colour c
+        for (int c = 0; c < kk; ++c) {
+            unsigned long long x = 0ull;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int v = lane + 32 * h;
+                if (v < n && ((alive >> v) & 1ull) && colv[h] == c) x |= 1ull << v;
             }
-            __syncthreads();
+            x = warp_or_u64(x);
+            if (lane == c) mine = x;
         }
-        if (tid == 0) {
+        if (lane < 16) cls[lane] = lane < kk ? mine : 0ull;
+        __syncwarp();
+        if (lane < kk) {
+            unsigned long long first = mine;
+            if (s >= 0) first &= (s < 64) ? (1ull << s) : 0ull;
+            reach[1u << lane] = first;
+        }
+        __syncwarp();
+        const unsigned long long not_end = (u >= 0 && u < 64) ? ~(1ull << u) : ~0ull;
+        const bool my_colour = lane < kk;
+        for (uint32_t C = 1; C < full; ++C) {
+            const unsigned long long X = reach[C] & not_end;  // a walk that has reached the end vertex stops
+            if (!X) continue;
+            unsigned long long N = (((X >> lane) & 1ull) ? adj2[0] : 0ull) | (((X >> (lane + 32)) & 1ull) ? adj2[1] : 0ull);
+            N = warp_or_u64(N);
+            if (my_colour && !((C >> lane) & 1u)) {
+                const unsigned long long add = N & mine;
+                if (add) reach[C | (1u << lane)] |= add;
+            }
+            __syncwarp();
+        }
+        if (lane == 0) {
             unsigned long long ends = reach[full];
             if (u >= 0) ends &= (u < 64) ? (1ull << u) : 0ull;
             int32_t *out = path + q * kk;
@@ -101,7 +143,7 @@ k_kpath_colour(int n, int kk, int64_t Q, const uint32_t *__restrict__ bw, const 
 
 }  // namespace
 
-size_t kpath_smem_bytes(int kk) { return ((size_t)1 << kk) * sizeof(unsigned long long); }
+size_t kpath_smem_bytes(int kk) { return kpath_layout(kk).total * kpath_warps_per_block(kk); }
 
 cudaError_t launch_kpath(int n, int kk, int64_t Q, const uint32_t *bw, const uint32_t *threshold, const int32_t *start,
                          const int32_t *end, const unsigned long long *alive, const uint8_t *colours, uint8_t *found,
@@ -111,11 +153,12 @@ cudaError_t launch_kpath(int n, int kk, int64_t Q, const uint32_t *bw, const uin
     const size_t sm = kpath_smem_bytes(kk);
     cudaError_t e = cudaFuncSetAttribute(k_kpath_colour, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    int64_t blocks = Q;
+    const int warps = kpath_warps_per_block(kk);
+    int64_t blocks = (Q + warps - 1) / warps;
     const int64_t cap = 148 * 16;
     if (blocks > cap) blocks = cap;
-    k_kpath_colour<<<(unsigned)blocks, kKpathThreads, sm, s>>>(n, kk, Q, bw, threshold, start, end, alive, colours,
-                                                                found, path);
+    k_kpath_colour<<<(unsigned)blocks, warps * 32, sm, s>>>(n, kk, Q, bw, threshold, start, end, alive, colours, found,
+                                                            path);
     return cudaGetLastError();
 }
 
